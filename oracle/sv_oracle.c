@@ -1,0 +1,377 @@
+/*
+ * sv_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, fp64 CPU statement of the importance-based sparse
+ * verification attention of the paper "Accelerate Speculative Decoding with
+ * Sparse Computation in Verification" (Section 3.1 "Sparse Attention",
+ * Section 3.2 "Piecewise Budget Control", Section 3.3 "Inter-layer Retrieval
+ * Reuse").  Only the tests, the smoke check and the CPU-baseline leg of the
+ * benchmark may call it.  It shares no code with the CUDA library and is
+ * written so that each function can be checked against the paper by eye:
+ * no blocking, no fusion, no reordering beyond what the definitions state.
+ *
+ * Every floating-point quantity is fp64.  Tensor inputs arrive as bfloat16
+ * bit patterns (uint16) and are widened exactly.
+ *
+ * KV-cache layout (Eq. 4: one block = one KV head x B consecutive tokens):
+ *   pool[page][h][t_in_block][d], page = block_table[s][t / B].
+ *
+ * Parity pins (see tests/test_oracle_pins.py):
+ *   svo_block_reps / svo_group_query / svo_scores : Eq. 5 evaluated literally
+ *       in numpy; planted-shift closed form.
+ *   svo_select  : brute-force enumeration of all subsets on tiny inputs.
+ *   svo_verify_attn : budget = all blocks equals svo_dense_verify_attn and a
+ *       library scaled-dot-product attention with an explicit mask; prefix
+ *       truncation; softmax weights sum to one; log-sum-exp split merge.
+ *   svo_budget_blocks : closed form of Eq. 6 and the sparsity column of Table 2.
+ *   Approximation quality of sparse vs dense attention: parity unpinned (the
+ *       paper bounds nothing; reported as information only).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_f64(uint16_t bits)
+{
+    uint32_t u = (uint32_t)bits << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int svo_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* element d of the cached key/value of token t, kv head h, sequence s */
+static double kv_at(const uint16_t *pool, const int32_t *block_table, int s, int h, int64_t t, int d,
+                    int Hkv, int D, int B, int NBmax)
+{
+    int64_t page = block_table[(int64_t)s * NBmax + t / B];
+    int64_t off = ((page * Hkv + h) * B + (t % B)) * D + d;
+    return bf16_to_f64(pool[off]);
+}
+
+/*
+ * Block representative (Eq. 5 by linearity: s = q0 . mean(k)): the mean key of
+ * the block.  The last block of a sequence may hold fewer than B tokens; its
+ * mean is taken over the tokens it holds.
+ * reps[s][h][b][d], b < ceil(L_s / B); other entries are left untouched.
+ */
+int svo_block_reps(int S, int Hkv, int D, int B, int NBmax, const uint16_t *k_pool, const int32_t *block_table,
+                   const int32_t *seq_lens, double *reps)
+{
+    for (int s = 0; s < S; ++s) {
+        int64_t L = seq_lens[s];
+        int nb = (int)((L + B - 1) / B);
+        if (nb > NBmax) return 1;
+#pragma omp parallel for collapse(2)
+        for (int h = 0; h < Hkv; ++h) {
+            for (int b = 0; b < nb; ++b) {
+                int64_t t0 = (int64_t)b * B;
+                int64_t cnt = (L - t0 < B) ? (L - t0) : B;
+                for (int d = 0; d < D; ++d) {
+                    double sum = 0.0;
+                    for (int64_t t = t0; t < t0 + cnt; ++t)
+                        sum += kv_at(k_pool, block_table, s, h, t, d, Hkv, D, B, NBmax);
+                    reps[(((int64_t)s * Hkv + h) * NBmax + b) * D + d] = sum / (double)cnt;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/*
+ * Retrieval query (Section 2.2: only the first draft token retrieves).  Blocks
+ * belong to KV heads, queries to query heads; the G = Hq / Hkv query heads
+ * hq = h*G .. h*G+G-1 share KV head h, and the retrieval query of KV head h is
+ * their mean.  q[s][i][hq][d], row i = 0 is the first draft token.
+ * qbar[s][h][d].
+ */
+int svo_group_query(int S, int T, int Hq, int Hkv, int D, const uint16_t *q, double *qbar)
+{
+    if (Hq % Hkv) return 1;
+    int G = Hq / Hkv;
+    for (int s = 0; s < S; ++s)
+        for (int h = 0; h < Hkv; ++h)
+            for (int d = 0; d < D; ++d) {
+                double sum = 0.0;
+                for (int g = 0; g < G; ++g)
+                    sum += bf16_to_f64(q[(((int64_t)s * T + 0) * Hq + h * G + g) * D + d]);
+                qbar[((int64_t)s * Hkv + h) * D + d] = sum / (double)G;
+            }
+    return 0;
+}
+
+/* Importance score (Eq. 5): scores[s][h][b] = qbar[s][h] . reps[s][h][b].  No 1/sqrt(D), no softmax. */
+int svo_scores(int S, int Hkv, int D, int B, int NBmax, const double *qbar, const double *reps,
+               const int32_t *seq_lens, double *scores)
+{
+    for (int s = 0; s < S; ++s) {
+        int nb = (int)(((int64_t)seq_lens[s] + B - 1) / B);
+        for (int h = 0; h < Hkv; ++h)
+            for (int b = 0; b < nb; ++b) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d)
+                    acc += qbar[((int64_t)s * Hkv + h) * D + d] * reps[(((int64_t)s * Hkv + h) * NBmax + b) * D + d];
+                scores[((int64_t)s * Hkv + h) * NBmax + b] = acc;
+            }
+    }
+    return 0;
+}
+
+/*
+ * Block selection (Section 3.1): keep the first n_sink and the last n_local
+ * blocks without eviction, then the highest-scoring blocks of the rest until
+ * budget[s] blocks are kept (the forced blocks count against the budget).
+ * Equal scores: the smaller block index wins.  A budget >= the number of
+ * blocks keeps every block (Section 3.2: no eviction).  One set per
+ * (sequence, KV head), shared by every draft token (Section 2.2).
+ * idx[s][h][0..cnt) ascending block indices, cnt[s][h].
+ * Returns 2 when the forced blocks alone exceed the budget, 3 when the set
+ * does not fit max_sel.
+ */
+int svo_select(int S, int Hkv, int B, int NBmax, const double *scores, const int32_t *seq_lens,
+               const int32_t *budget, int n_sink, int n_local, int max_sel, int32_t *idx, int32_t *cnt)
+{
+    for (int s = 0; s < S; ++s) {
+        int nb = (int)(((int64_t)seq_lens[s] + B - 1) / B);
+        int N = budget[s];
+        for (int h = 0; h < Hkv; ++h) {
+            const double *sc = scores + ((int64_t)s * Hkv + h) * NBmax;
+            int32_t *out = idx + ((int64_t)s * Hkv + h) * max_sel;
+            char *keep = (char *)calloc((size_t)(nb > 0 ? nb : 1), 1);
+            int kept = 0;
+            if (N >= nb) {
+                for (int b = 0; b < nb; ++b) keep[b] = 1;
+                kept = nb;
+            } else {
+                for (int b = 0; b < nb; ++b)
+                    if (b < n_sink || b >= nb - n_local) {
+                        keep[b] = 1;
+                        ++kept;
+                    }
+                if (kept > N) {
+                    free(keep);
+                    return 2;
+                }
+                while (kept < N) {
+                    int best = -1;
+                    for (int b = 0; b < nb; ++b)
+                        if (!keep[b] && (best < 0 || sc[b] > sc[best])) best = b;
+                    keep[best] = 1;
+                    ++kept;
+                }
+            }
+            if (kept > max_sel) {
+                free(keep);
+                return 3;
+            }
+            int n = 0;
+            for (int b = 0; b < nb; ++b)
+                if (keep[b]) out[n++] = b;
+            cnt[(int64_t)s * Hkv + h] = n;
+            free(keep);
+        }
+    }
+    return 0;
+}
+
+/* is draft token j visible to draft token i?  chain: j <= i; tree: j is i or an ancestor of i. */
+static int draft_visible(const int32_t *parent, int s, int T, int i, int j)
+{
+    if (!parent) return j <= i;
+    for (int a = i; a >= 0; a = parent[(int64_t)s * T + a])
+        if (a == j) return 1;
+    return 0;
+}
+
+/*
+ * softmax(scale * q . k) weighted sum of v over a list of (z, value-row) pairs,
+ * the textbook three steps: max, exponentials, normalised sum.
+ */
+static void softmax_weighted_sum(int n, const double *z, const double *vals, int D, double *o, double *lse)
+{
+    double m = -INFINITY, l = 0.0;
+    for (int j = 0; j < n; ++j)
+        if (z[j] > m) m = z[j];
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    for (int j = 0; j < n; ++j) {
+        double p = exp(z[j] - m);
+        l += p;
+        for (int d = 0; d < D; ++d) o[d] += p * vals[(int64_t)j * D + d];
+    }
+    for (int d = 0; d < D; ++d) o[d] /= l;
+    *lse = m + log(l);
+}
+
+/*
+ * Sparse verification attention (Fig. 1; the 4B(1-s_a)T^2 d term of Table 1):
+ * every draft token i of every query head hq attends to the cached tokens of
+ * the selected blocks of its KV head hq / G (tokens t < L_s only) and to the
+ * draft tokens visible to it (itself and its ancestors; a causal chain when
+ * parent is NULL).  Standard scaled dot-product attention.
+ *
+ * samples: NULL -> all (s, i, hq) rows; otherwise n_samples triples
+ * (s, i, hq) and out/lse hold n_samples rows in that order.
+ * out[s][i][hq][d] fp64, lse[s][i][hq] = log of the softmax denominator.
+ */
+int svo_verify_attn(int S, int T, int Hq, int Hkv, int D, int B, int NBmax, const uint16_t *q,
+                    const uint16_t *k_pool, const uint16_t *v_pool, const int32_t *block_table,
+                    const int32_t *seq_lens, const uint16_t *draft_k, const uint16_t *draft_v,
+                    const int32_t *parent, const int32_t *sel_idx, const int32_t *sel_cnt, int max_sel,
+                    double scale, int n_samples, const int32_t *samples, double *out, double *lse)
+{
+    int G = Hq / Hkv;
+    int64_t n_rows = samples ? n_samples : (int64_t)S * T * Hq;
+    int err = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        int s, i, hq;
+        if (samples) {
+            s = samples[3 * r], i = samples[3 * r + 1], hq = samples[3 * r + 2];
+        } else {
+            s = (int)(r / ((int64_t)T * Hq)), i = (int)((r / Hq) % T), hq = (int)(r % Hq);
+        }
+        int h = hq / G;
+        int64_t L = seq_lens[s];
+        const int32_t *sel = sel_idx + ((int64_t)s * Hkv + h) * max_sel;
+        int n_sel = sel_cnt[(int64_t)s * Hkv + h];
+        int64_t cap = (int64_t)n_sel * B + T;
+        double *z = (double *)malloc(sizeof(double) * (size_t)cap);
+        double *vals = (double *)malloc(sizeof(double) * (size_t)cap * D);
+        double qi[1024];
+        if (!z || !vals || D > 1024) {
+            err = 1;
+            free(z);
+            free(vals);
+            continue;
+        }
+        for (int d = 0; d < D; ++d) qi[d] = bf16_to_f64(q[(((int64_t)s * T + i) * Hq + hq) * D + d]);
+        int n = 0;
+        for (int j = 0; j < n_sel; ++j) {
+            int64_t b = sel[j];
+            for (int64_t t = b * B; t < (b + 1) * B && t < L; ++t) {
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d) dot += qi[d] * kv_at(k_pool, block_table, s, h, t, d, Hkv, D, B, NBmax);
+                z[n] = scale * dot;
+                for (int d = 0; d < D; ++d)
+                    vals[(int64_t)n * D + d] = kv_at(v_pool, block_table, s, h, t, d, Hkv, D, B, NBmax);
+                ++n;
+            }
+        }
+        for (int j = 0; j < T; ++j) {
+            if (!draft_visible(parent, s, T, i, j)) continue;
+            const uint16_t *kj = draft_k + (((int64_t)s * T + j) * Hkv + h) * D;
+            const uint16_t *vj = draft_v + (((int64_t)s * T + j) * Hkv + h) * D;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += qi[d] * bf16_to_f64(kj[d]);
+            z[n] = scale * dot;
+            for (int d = 0; d < D; ++d) vals[(int64_t)n * D + d] = bf16_to_f64(vj[d]);
+            ++n;
+        }
+        softmax_weighted_sum(n, z, vals, D, out + r * D, lse + r);
+        free(z);
+        free(vals);
+    }
+    return err;
+}
+
+/*
+ * Dense ("strict") verification attention: the same attention over the whole
+ * cached prefix 0..L_s-1, written as its own contiguous loop with no block
+ * list.  Fixed point of the sparse path when nothing is evicted, and the dense
+ * CPU baseline.  Same sampling convention as svo_verify_attn.
+ */
+int svo_dense_verify_attn(int S, int T, int Hq, int Hkv, int D, int B, int NBmax, const uint16_t *q,
+                          const uint16_t *k_pool, const uint16_t *v_pool, const int32_t *block_table,
+                          const int32_t *seq_lens, const uint16_t *draft_k, const uint16_t *draft_v,
+                          const int32_t *parent, double scale, int n_samples, const int32_t *samples,
+                          double *out, double *lse)
+{
+    int G = Hq / Hkv;
+    int64_t n_rows = samples ? n_samples : (int64_t)S * T * Hq;
+    int err = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        int s, i, hq;
+        if (samples) {
+            s = samples[3 * r], i = samples[3 * r + 1], hq = samples[3 * r + 2];
+        } else {
+            s = (int)(r / ((int64_t)T * Hq)), i = (int)((r / Hq) % T), hq = (int)(r % Hq);
+        }
+        int h = hq / G;
+        int64_t L = seq_lens[s];
+        int64_t n = L + T;
+        double *z = (double *)malloc(sizeof(double) * (size_t)n);
+        if (!z) {
+            err = 1;
+            continue;
+        }
+        const uint16_t *qi = q + (((int64_t)s * T + i) * Hq + hq) * D;
+        for (int64_t t = 0; t < L; ++t) {
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d)
+                dot += bf16_to_f64(qi[d]) * kv_at(k_pool, block_table, s, h, t, d, Hkv, D, B, NBmax);
+            z[t] = scale * dot;
+        }
+        for (int j = 0; j < T; ++j) {
+            if (!draft_visible(parent, s, T, i, j)) {
+                z[L + j] = -INFINITY;
+                continue;
+            }
+            const uint16_t *kj = draft_k + (((int64_t)s * T + j) * Hkv + h) * D;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += bf16_to_f64(qi[d]) * bf16_to_f64(kj[d]);
+            z[L + j] = scale * dot;
+        }
+        double m = -INFINITY;
+        for (int64_t t = 0; t < n; ++t)
+            if (z[t] > m) m = z[t];
+        double l = 0.0;
+        for (int64_t t = 0; t < n; ++t) {
+            z[t] = exp(z[t] - m); /* z now holds the unnormalised softmax weights */
+            l += z[t];
+        }
+        double *o = out + r * D;
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int64_t t = 0; t < L; ++t)
+                acc += z[t] / l * kv_at(v_pool, block_table, s, h, t, d, Hkv, D, B, NBmax);
+            for (int j = 0; j < T; ++j)
+                acc += z[L + j] / l * bf16_to_f64(draft_v[(((int64_t)s * T + j) * Hkv + h) * D + d]);
+            o[d] = acc;
+        }
+        lse[r] = m + log(l);
+        free(z);
+    }
+    return err;
+}
+
+/*
+ * Piecewise budget (Section 3.2, Eq. 6) per KV head: a cache of at most L0
+ * tokens is not evicted; a longer one keeps ((L - L0) * rho + L0) / B blocks
+ * per head, rounded up, and never fewer than the forced blocks nor more than
+ * the blocks that exist.
+ */
+int svo_budget_blocks(int64_t L, int64_t L0, double rho, int B, int n_sink, int n_local)
+{
+    int nb = (int)((L + B - 1) / B);
+    if (L <= L0) return nb;
+    double tokens = ((double)(L - L0)) * rho + (double)L0;
+    int n = (int)ceil(tokens / (double)B);
+    int forced = n_sink + n_local;
+    if (n < forced) n = forced;
+    if (n > nb) n = nb;
+    return n;
+}

@@ -1,0 +1,433 @@
+"""Pins of the fp64 CPU oracle to what the paper and the mathematics fix (no GPU needed).
+
+Each test ties one oracle function to something other than itself: a hand-worked fixture under
+tests/golden/, a closed form, brute force on tiny inputs, a library routine, or an invariant of
+the definition.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import sv_inputs as si
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_fixture(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = np.array([float(v) for v in vals])
+    return out
+
+
+def _bits(x):
+    return si.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def _tiny_case(S=2, Hq=4, Hkv=2, D=8, B=4, T=3, lens=(13, 6), seed=0, tree=False, scale=1.0):
+    """Small random case with an out-of-order page table (values rounded to bf16)."""
+    g = np.random.default_rng(seed)
+    lens = np.array(lens, dtype=np.int32)
+    nb = (lens + B - 1) // B
+    n_pages = int(nb.sum()) + 2
+    perm = g.permutation(n_pages)
+    bt = np.zeros((S, int(nb.max())), dtype=np.int32)
+    o = 0
+    for s in range(S):
+        bt[s, :nb[s]] = perm[o:o + nb[s]]
+        o += nb[s]
+    c = dict(
+        q=_bits(g.standard_normal((S, T, Hq, D)) * scale),
+        k_pool=_bits(g.standard_normal((n_pages, Hkv, B, D)) * scale),
+        v_pool=_bits(g.standard_normal((n_pages, Hkv, B, D))),
+        draft_k=_bits(g.standard_normal((S, T, Hkv, D)) * scale),
+        draft_v=_bits(g.standard_normal((S, T, Hkv, D))),
+        block_table=bt, seq_lens=lens, n_blocks=nb, B=B, Hkv=Hkv, parent=None)
+    if tree:
+        par = np.full((S, T), -1, dtype=np.int32)
+        for s in range(S):
+            for i in range(1, T):
+                par[s, i] = g.integers(0, i)
+        c["parent"] = par
+    return c
+
+
+def _gather_tokens(pool, bt, s, h, L, B):
+    """[L][D] fp64 rows of one (sequence, KV head), gathered with numpy indexing (independent of the C code)."""
+    t = np.arange(L)
+    return si.bf16_bits_to_f64(pool[bt[s, t // B], h, t % B, :])
+
+
+# --------------------------------------------------------------------------- O1-O3: Eq. 5
+
+def test_eq5_hand_worked_fixture():
+    fx = _read_fixture("eq5_block_scores.txt")
+    q = _bits(fx["q_heads"].reshape(1, 1, 2, 2))
+    k_pool = np.zeros((3, 1, 2, 2), dtype=np.uint16)
+    keys = fx["keys"].reshape(5, 2)
+    bt = np.array([[2, 0, 1]], dtype=np.int32)          # pages out of order on purpose
+    for t in range(5):
+        k_pool[bt[0, t // 2], 0, t % 2] = _bits(keys[t])
+    k_pool[bt[0, 2], 0, 1] = _bits([99.0, 99.0])        # slot past the end of the sequence: must be ignored
+    lens = np.array([5], dtype=np.int32)
+    reps = oracle.block_reps(k_pool, bt, lens)
+    np.testing.assert_array_equal(reps[0, 0], fx["reps"].reshape(3, 2))
+    qbar = oracle.group_query(q, 1)
+    np.testing.assert_array_equal(qbar[0, 0], [2.0, 0.0])
+    sc = oracle.scores(qbar, reps, lens, 2)
+    np.testing.assert_array_equal(sc[0, 0], fx["scores"])
+
+
+def test_eq5_literal_sum_matches_representative_form():
+    """Eq. 5 as printed (mean over the block of q0.k) against the oracle's q0 . mean(k)."""
+    c = _tiny_case(seed=3)
+    B, Hkv = c["B"], c["Hkv"]
+    reps = oracle.block_reps(c["k_pool"], c["block_table"], c["seq_lens"])
+    qbar = oracle.group_query(c["q"], Hkv)
+    sc = oracle.scores(qbar, reps, c["seq_lens"], B)
+    G = c["q"].shape[2] // Hkv
+    for s in range(2):
+        L = int(c["seq_lens"][s])
+        for h in range(Hkv):
+            keys = _gather_tokens(c["k_pool"], c["block_table"], s, h, L, B)
+            q0 = si.bf16_bits_to_f64(c["q"][s, 0, h * G:(h + 1) * G]).sum(axis=0) / G
+            dots = keys @ q0
+            for b in range(int(c["n_blocks"][s])):
+                lit = dots[b * B:min((b + 1) * B, L)].mean()
+                assert abs(sc[s, h, b] - lit) < 1e-12
+            assert np.all(np.isneginf(sc[s, h, int(c["n_blocks"][s]):]))
+
+
+def test_planted_shift_closed_form():
+    """A block whose keys are all c*u (u = q0/|q0|), others zero: score is exactly c*|q0|, others 0."""
+    D, B = 4, 4
+    q = _bits(np.array([3.0, 0.0, 4.0, 0.0]).reshape(1, 1, 1, D))     # |q0| = 5, u = (0.6, 0, 0.8, 0)
+    k_pool = np.zeros((4, 1, B, D), dtype=np.uint16)
+    u = np.array([0.75, 0.0, 1.0, 0.0])                                # 1.25*u, exactly representable
+    k_pool[2, 0] = _bits(np.tile(u, (B, 1)))
+    bt = np.array([[0, 1, 2, 3]], dtype=np.int32)
+    lens = np.array([16], dtype=np.int32)
+    idx, cnt, sc = oracle.select_blocks(q, k_pool, bt, lens, np.array([1], np.int32), 0, 0, 4)
+    np.testing.assert_array_equal(sc[0, 0], [0.0, 0.0, 1.25 * 5.0, 0.0])
+    assert cnt[0, 0] == 1 and idx[0, 0, 0] == 2
+
+
+# --------------------------------------------------------------------------- O4: selection
+
+def _brute_force_select(sc, nb, N, n_sink, n_local):
+    if N >= nb:
+        return list(range(nb))
+    forced = [b for b in range(nb) if b < n_sink or b >= nb - n_local]
+    rest = [b for b in range(nb) if b not in forced]
+    best, best_sum = None, -math.inf
+    for comb in itertools.combinations(rest, N - len(forced)):     # lexicographic: smaller indices first
+        tot = sum(sc[b] for b in comb)
+        if tot > best_sum:
+            best, best_sum = comb, tot
+    return sorted(forced + list(best))
+
+
+@pytest.mark.parametrize("n_sink,n_local", [(0, 0), (1, 1), (2, 3)])
+def test_select_equals_brute_force(n_sink, n_local):
+    g = np.random.default_rng(11)
+    B = 4
+    for trial in range(12):
+        nb = int(g.integers(n_sink + n_local + 1, 13))
+        N = int(g.integers(n_sink + n_local, nb + 2))
+        L = nb * B - int(g.integers(0, B))
+        sc = np.full((1, 1, 12), -np.inf)
+        sc[0, 0, :nb] = g.standard_normal(nb)
+        idx, cnt = oracle.select(sc, np.array([L], np.int32), np.array([N], np.int32), B, n_sink, n_local, 12)
+        want = _brute_force_select(sc[0, 0], nb, N, n_sink, n_local)
+        assert cnt[0, 0] == len(want) == min(N, nb)
+        assert idx[0, 0, :cnt[0, 0]].tolist() == want
+
+
+def test_select_ties_prefer_smaller_index_and_errors():
+    sc = np.zeros((1, 1, 8))
+    idx, cnt = oracle.select(sc, np.array([32], np.int32), np.array([4], np.int32), 4, 1, 1, 8)
+    assert idx[0, 0, :4].tolist() == [0, 1, 2, 7]
+    with pytest.raises(ValueError):
+        oracle.select(sc, np.array([32], np.int32), np.array([1], np.int32), 4, 1, 1, 8)
+    with pytest.raises(ValueError):
+        oracle.select(sc, np.array([32], np.int32), np.array([5], np.int32), 4, 1, 1, 4)
+
+
+def test_selection_ignores_later_draft_tokens_and_is_shared():
+    """Only the first draft token retrieves (Section 2.2): other query rows cannot change the set."""
+    geom = si.make_geometry(si.WORKLOADS["cfg0"])
+    c = si.make_layer(geom)
+    a = oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
+    q2 = c["q"].copy()
+    q2[:, 1:] = _bits(np.random.default_rng(5).standard_normal(q2[:, 1:].shape))
+    b = oracle.select_blocks(q2, c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
+    np.testing.assert_array_equal(a[0], b[0])
+    assert a[0].shape == (1, 2, 16)        # one list per (sequence, KV head), none per draft token
+
+
+def test_generator_plants_and_repairs_gap():
+    geom = si.make_geometry(si.WORKLOADS["cfg0"])
+    c = si.make_layer(geom)
+    idx, cnt, sc = oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
+    assert c["min_gap"] >= c["delta"] > 0
+    for (s, h), planted in c["planted"].items():
+        sel = set(idx[s, h, :cnt[s, h]].tolist())
+        assert set(planted.tolist()) <= sel and {0, 63} <= sel
+        rest = np.setdiff1d(np.arange(64), list(sel))
+        assert sc[s, h, list(sel - {0, 63})].min() - sc[s, h, rest].max() >= c["delta"] * 0.999
+
+
+# --------------------------------------------------------------------------- O5: inter-layer reuse (Eq. 9)
+
+def test_reuse_copies_nearest_preceding_anchor():
+    w = si.shrink(si.WORKLOADS["cfg0"], seq_len=(1024, 1024), budget_blocks=6, planted=3)
+    geom = si.make_geometry(w)
+    layers = [si.make_layer(geom, layer=l) for l in range(5)]
+    anchors = [True, False, True, False, False]
+    res = oracle.select_layers(layers, anchors, geom["budget"], 1, 1, geom["max_sel"])
+    ind = oracle.select_layers(layers, [True] * 5, geom["budget"], 1, 1, geom["max_sel"])
+    for l, a in enumerate([0, 0, 2, 2, 2]):
+        np.testing.assert_array_equal(res[l][0], ind[a][0])
+        np.testing.assert_array_equal(res[l][1], ind[a][1])
+    for l in range(5):      # all anchors == independent per-layer retrieval
+        one = oracle.select_blocks(layers[l]["q"], layers[l]["k_pool"], geom["block_table"], geom["seq_lens"],
+                                   geom["budget"], 1, 1, geom["max_sel"])
+        np.testing.assert_array_equal(ind[l][0], one[0])
+    assert any(not np.array_equal(ind[0][0], ind[l][0]) for l in range(1, 5))
+
+
+# --------------------------------------------------------------------------- O6: attention
+
+def _all_blocks(c, max_sel=None):
+    S, Hkv = c["block_table"].shape[0], c["Hkv"]
+    nbmax = int(c["n_blocks"].max())
+    max_sel = max_sel or nbmax
+    idx = np.full((S, Hkv, max_sel), -1, dtype=np.int32)
+    cnt = np.zeros((S, Hkv), dtype=np.int32)
+    for s in range(S):
+        idx[s, :, :c["n_blocks"][s]] = np.arange(c["n_blocks"][s])
+        cnt[s] = c["n_blocks"][s]
+    return idx, cnt
+
+
+def _attn(c, idx, cnt, **kw):
+    return oracle.verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"],
+                              c["draft_v"], c["parent"], idx, cnt, **kw)
+
+
+def _dense(c, **kw):
+    return oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                    c["draft_k"], c["draft_v"], c["parent"], **kw)
+
+
+def test_attention_hand_worked_fixture():
+    fx = _read_fixture("softmax_attention.txt")
+    k_pool = np.zeros((2, 1, 2, 2), np.uint16)
+    v_pool = np.zeros((2, 1, 2, 2), np.uint16)
+    bt = np.array([[1, 0]], np.int32)
+    for t in range(3):
+        k_pool[bt[0, t // 2], 0, t % 2] = _bits(fx["keys"].reshape(3, 2)[t])
+        v_pool[bt[0, t // 2], 0, t % 2] = _bits(fx["values"].reshape(3, 2)[t])
+    k_pool[bt[0, 1], 0, 1] = _bits([40.0, 40.0])      # past the end: must not contribute
+    v_pool[bt[0, 1], 0, 1] = _bits([1e4, 1e4])
+    args = (_bits(fx["q"].reshape(1, 1, 1, 2)), k_pool, v_pool, bt, np.array([3], np.int32),
+            _bits(fx["draft_k"].reshape(1, 1, 1, 2)), _bits(fx["draft_v"].reshape(1, 1, 1, 2)), None)
+    ln2 = math.log(2.0)
+    cases = [([0, 1], [1.0, 14.0], math.log(15.0)), ([0], [-105.0 / 11, 270.0 / 11], math.log(11.0)),
+             ([1], [0.0, 15.0], math.log(12.0))]
+    for sel, o_want, lse_want in cases:
+        idx = np.array([[sel + [-1] * (2 - len(sel))]], np.int32)
+        cnt = np.array([[len(sel)]], np.int32)
+        o, lse = oracle.verify_attn(*args, idx, cnt, scale=ln2)
+        np.testing.assert_allclose(o[0, 0, 0], o_want, rtol=0, atol=1e-13)
+        assert abs(lse[0, 0, 0] - lse_want) < 1e-13
+    o, lse = oracle.dense_verify_attn(*args, scale=ln2)
+    np.testing.assert_allclose(o[0, 0, 0], [1.0, 14.0], rtol=0, atol=1e-13)
+    assert abs(lse[0, 0, 0] - math.log(15.0)) < 1e-13
+
+
+@pytest.mark.parametrize("tree", [False, True])
+def test_all_blocks_equals_dense_and_library_sdpa(tree):
+    c = _tiny_case(S=2, Hq=4, Hkv=2, D=8, B=4, T=5, lens=(13, 8), seed=7, tree=tree)
+    idx, cnt = _all_blocks(c)
+    o, lse = _attn(c, idx, cnt)
+    od, lsed = _dense(c)
+    np.testing.assert_allclose(o, od, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, lsed, rtol=0, atol=1e-12)
+    # library routine: torch scaled_dot_product_attention in fp64 with an explicit boolean mask
+    S, T, Hq, D = c["q"].shape
+    G = Hq // c["Hkv"]
+    for s in range(S):
+        L = int(c["seq_lens"][s])
+        for hq in range(Hq):
+            h = hq // G
+            K = np.concatenate([_gather_tokens(c["k_pool"], c["block_table"], s, h, L, 4),
+                                si.bf16_bits_to_f64(c["draft_k"][s, :, h])])
+            V = np.concatenate([_gather_tokens(c["v_pool"], c["block_table"], s, h, L, 4),
+                                si.bf16_bits_to_f64(c["draft_v"][s, :, h])])
+            Q = si.bf16_bits_to_f64(c["q"][s, :, hq])
+            mask = np.ones((T, L + T), dtype=bool)
+            for i in range(T):
+                vis = set()
+                a = i
+                while a >= 0:
+                    vis.add(a)
+                    a = (a - 1) if c["parent"] is None else int(c["parent"][s, a])
+                for j in range(T):
+                    mask[i, L + j] = j in vis
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                torch.from_numpy(Q)[None], torch.from_numpy(K)[None], torch.from_numpy(V)[None],
+                attn_mask=torch.from_numpy(mask)[None]).numpy()[0]
+            np.testing.assert_allclose(o[s, :, hq], ref, rtol=0, atol=1e-12)
+
+
+def test_prefix_blocks_equal_dense_on_truncated_prefix():
+    c = _tiny_case(S=1, Hq=2, Hkv=1, D=8, B=4, T=2, lens=(19,), seed=9)
+    idx = np.array([[[0, 1, 2, -1, -1]]], np.int32)
+    cnt = np.array([[3]], np.int32)
+    o, lse = _attn(c, idx, cnt)
+    c2 = dict(c)
+    c2["seq_lens"] = np.array([12], np.int32)
+    od, lsed = _dense(c2)
+    np.testing.assert_allclose(o, od, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, lsed, rtol=0, atol=1e-12)
+
+
+def test_softmax_weights_sum_to_one():
+    """With every value vector equal to ones the output is the sum of the softmax weights."""
+    c = _tiny_case(seed=13, tree=True, scale=3.0)
+    c["v_pool"][...] = _bits(1.0)
+    c["draft_v"][...] = _bits(1.0)
+    idx = np.array([[[0, 2, -1, -1]] * 2, [[1, -1, -1, -1]] * 2], np.int32)
+    cnt = np.array([[2, 2], [1, 1]], np.int32)
+    o, _ = _attn(c, idx, cnt)
+    np.testing.assert_allclose(o, 1.0, rtol=0, atol=1e-12)
+
+
+def test_single_draft_token_is_plain_decode_attention():
+    c = _tiny_case(S=1, Hq=2, Hkv=1, D=8, B=4, T=1, lens=(10,), seed=17)
+    idx, cnt = _all_blocks(c)
+    o, lse = _attn(c, idx, cnt)
+    K = np.concatenate([_gather_tokens(c["k_pool"], c["block_table"], 0, 0, 10, 4), si.bf16_bits_to_f64(c["draft_k"][0, :, 0])])
+    V = np.concatenate([_gather_tokens(c["v_pool"], c["block_table"], 0, 0, 10, 4), si.bf16_bits_to_f64(c["draft_v"][0, :, 0])])
+    for hq in range(2):
+        z = K @ si.bf16_bits_to_f64(c["q"][0, 0, hq]) / math.sqrt(8)
+        p = np.exp(z - z.max())
+        np.testing.assert_allclose(o[0, 0, hq], (p / p.sum()) @ V, rtol=0, atol=1e-12)
+        assert abs(lse[0, 0, hq] - (z.max() + math.log(p.sum()))) < 1e-12
+
+
+def test_tree_with_linear_parents_is_chain():
+    c = _tiny_case(seed=19, T=4)
+    idx, cnt = _all_blocks(c)
+    o_chain, _ = _attn(c, idx, cnt)
+    c["parent"] = np.tile(np.arange(-1, 3, dtype=np.int32), (2, 1))
+    o_tree, _ = _attn(c, idx, cnt)
+    np.testing.assert_array_equal(o_chain, o_tree)
+
+
+def test_tree_siblings_do_not_see_each_other():
+    """Two children of the root: each equals a 2-token chain made of the root and itself."""
+    c = _tiny_case(S=1, Hq=2, Hkv=1, D=8, B=4, T=3, lens=(8,), seed=23)
+    idx, cnt = _all_blocks(c)
+    c["parent"] = np.array([[-1, 0, 0]], np.int32)
+    o, _ = _attn(c, idx, cnt)
+    c2 = dict(c)
+    keep = [0, 2]
+    c2.update(q=c["q"][:, keep].copy(), draft_k=c["draft_k"][:, keep].copy(), draft_v=c["draft_v"][:, keep].copy(),
+              parent=None)
+    o2, _ = _attn(c2, idx, cnt)
+    np.testing.assert_allclose(o[:, 2], o2[:, 1], rtol=0, atol=1e-13)
+
+
+def test_split_merge_by_log_sum_exp():
+    """Attention over Sel1 u Sel2 equals the log-sum-exp merge of attention over each half
+    (the draft tokens go with one half only; the other half is computed with T-less inputs via lse)."""
+    c = _tiny_case(S=1, Hq=2, Hkv=1, D=8, B=4, T=1, lens=(16,), seed=29, scale=2.0)
+    full_idx, full_cnt = _all_blocks(c)
+    o, lse = _attn(c, full_idx, full_cnt)
+    # half A: blocks {0,1} + draft token; half B: blocks {2,3} + draft token.  The draft token is in both,
+    # so remove its contribution once: w_draft = exp(z_draft - lse_X).
+    oa, la = _attn(c, np.array([[[0, 1, -1, -1]]], np.int32), np.array([[2]], np.int32))
+    ob, lb = _attn(c, np.array([[[2, 3, -1, -1]]], np.int32), np.array([[2]], np.int32))
+    on, ln_ = _attn(c, np.array([[[-1, -1, -1, -1]]], np.int32), np.array([[0]], np.int32))   # draft token only
+    for hq in range(2):
+        # sums of exponentials: E_A = e^{la}, E_B = e^{lb}, E_draft = e^{ln}; union = E_A + E_B - E_draft
+        m = max(la[0, 0, hq], lb[0, 0, hq])
+        ea, eb, en = (math.exp(x - m) for x in (la[0, 0, hq], lb[0, 0, hq], ln_[0, 0, hq]))
+        tot = ea + eb - en
+        merged = (ea * oa[0, 0, hq] + eb * ob[0, 0, hq] - en * on[0, 0, hq]) / tot
+        np.testing.assert_allclose(o[0, 0, hq], merged, rtol=0, atol=1e-11)
+        assert abs(lse[0, 0, hq] - (m + math.log(tot))) < 1e-11
+
+
+def test_sampled_rows_match_full_output():
+    c = _tiny_case(seed=31, tree=True)
+    idx = np.array([[[0, 3, -1, -1]] * 2, [[0, 1, -1, -1]] * 2], np.int32)
+    cnt = np.array([[2, 2], [2, 2]], np.int32)
+    o, lse = _attn(c, idx, cnt)
+    smp = [(1, 2, 3), (0, 0, 0), (0, 1, 2)]
+    os_, ls = _attn(c, idx, cnt, samples=smp)
+    od, ld = _dense(c)
+    ods, lds = _dense(c, samples=smp)
+    for r, (s, i, hq) in enumerate(smp):
+        np.testing.assert_array_equal(os_[r], o[s, i, hq])
+        assert ls[r] == lse[s, i, hq]
+        np.testing.assert_array_equal(ods[r], od[s, i, hq])
+        assert lds[r] == ld[s, i, hq]
+
+
+def test_full_budget_selection_gives_dense_attention_on_workload_shape():
+    """The paper's fixed point on a generator-made case: budget = all blocks => dense verification."""
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=2, seq_len=(300, 700), n_q_heads=8, n_kv_heads=2, budget_blocks=10**6)
+    geom = si.make_geometry(w)
+    c = si.make_layer(geom, sharp=True)
+    idx, cnt, _ = oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1,
+                                       geom["max_blocks"])
+    np.testing.assert_array_equal(cnt, np.repeat(geom["n_blocks"][:, None], 2, axis=1))
+    o, lse = oracle.verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"],
+                                c["draft_v"], None, idx, cnt)
+    od, lsed = oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                        c["draft_k"], c["draft_v"], None)
+    np.testing.assert_allclose(o, od, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, lsed, rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- O7: budget (Eq. 6)
+
+def test_budget_closed_form():
+    assert oracle.budget_blocks(4096, 4096, 0.1, 64) == 64           # L <= L0: nothing evicted
+    assert oracle.budget_blocks(1000, 4096, 0.1, 64) == 16
+    assert oracle.budget_blocks(32768, 4096, 0.1, 64) == 109         # (28672*0.1 + 4096)/64 = 108.8
+    assert oracle.budget_blocks(131072, 4096, 0.5, 128) == 528       # (126976*0.5 + 4096)/128 = 528
+    assert oracle.budget_blocks(5000, 64, 0.001, 64, 2, 4) == 6      # never fewer than the forced blocks
+    assert oracle.budget_blocks(4097, 4096, 0.999, 64) == 65         # never more than the blocks that exist
+    for L in (5000, 20000, 77777):
+        for rho in (0.05, 0.1, 0.3):
+            n = oracle.budget_blocks(L, 2048, rho, 1)
+            assert n == math.ceil((L - 2048) * rho + 2048)
+
+
+def test_budget_reproduces_table2_sparsity_column():
+    """Weak cross-check: one effective length per dataset reproduces the printed s_a at all three L0."""
+    rows = []
+    with open(os.path.join(GOLDEN, "table2_sparsity.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, L0, sa = line.split()
+                rows.append((name, int(L0), float(sa)))
+    for name, L in (("GovReport", 6300), ("2WikiMQA", 6900)):
+        for n, L0, sa in rows:
+            if n == name:
+                kept = oracle.budget_blocks(L, L0, 0.1, 1)
+                assert abs((1 - kept / L) - sa) < 0.035, (name, L0, 1 - kept / L, sa)
