@@ -1,0 +1,176 @@
+/*
+ * sv.h -- C ABI of the sparse verification attention library (CUDA, sm_100a).
+ *
+ * The library implements the importance-based sparse attention that a target
+ * model runs when it verifies draft tokens against a long KV cache (paper:
+ * "Accelerate Speculative Decoding with Sparse Computation in Verification",
+ * Section 3.1 "Sparse Attention", Section 3.2 "Piecewise Budget Control",
+ * Section 3.3 "Inter-layer Retrieval Reuse"):
+ *
+ *   sv_block_reps     one representative (the mean key) per KV block       (Eq. 5)
+ *   sv_select_blocks  score the representatives against the first draft
+ *                     token's query, keep the top-N blocks plus the first /
+ *                     last few; or reuse the previous layer's set  (Eq. 5, Eq. 9)
+ *   sv_verify_attn    attention of all draft tokens over the kept blocks
+ *                     and the draft tokens' own K/V                       (Fig. 1)
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are device memory owned by the caller; the library never
+ *     allocates, frees or synchronises.  Work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream) of the
+ *     current device and the call returns at once.
+ *   - Tensor bases must be 16-byte aligned (the K/V pools 128-byte aligned).
+ *   - bf16 tensors are passed as const void*.
+ *   - Arguments are validated on the host; a bad argument returns an sv_status
+ *     and launches nothing.  A failed launch returns SV_ERR_CUDA.
+ *   - head_dim must be 128; block_size 64 or 128; n_q_heads a multiple of
+ *     n_kv_heads; query head hq uses KV head hq / (n_q_heads / n_kv_heads).
+ */
+#ifndef SV_H_
+#define SV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define SV_API __attribute__((visibility("default")))
+#else
+#define SV_API
+#endif
+
+typedef enum {
+    SV_OK = 0,
+    SV_ERR_NULL = 1,        /* a required pointer is NULL */
+    SV_ERR_SHAPE = 2,       /* a size is out of range or inconsistent */
+    SV_ERR_ALIGN = 3,       /* a pointer is not aligned as required */
+    SV_ERR_BUDGET = 4,      /* n_sink + n_local exceeds max_sel */
+    SV_ERR_WORKSPACE = 5,   /* workspace_bytes is smaller than sv_workspace_bytes() */
+    SV_ERR_UNSUPPORTED = 6, /* head_dim != 128, block_size not 64/128, more than 128 query rows per KV head ... */
+    SV_ERR_CUDA = 7         /* a CUDA call or kernel launch failed */
+} sv_status;
+
+/* Static, human-readable text for a status code. */
+SV_API const char *sv_strerror(sv_status st);
+
+/* Geometry shared by all calls. */
+typedef struct {
+    int32_t n_seq;      /* S: sequences in the batch */
+    int32_t n_q_heads;  /* Hq */
+    int32_t n_kv_heads; /* Hkv */
+    int32_t head_dim;   /* D, must be 128 */
+    int32_t block_size; /* B: tokens per KV block (Eq. 4), 64 or 128 */
+    int32_t max_blocks; /* NBmax: row stride of block_table / reps / scores */
+    int32_t n_draft;    /* T: draft tokens verified per sequence, 1..32, with G*T <= 128 */
+} sv_geom;
+
+/*
+ * Paged KV cache; one page holds one block (Eq. 4: one KV head x B consecutive
+ * tokens) of every KV head:  pool[page][kv_head][token_in_block][dim], bf16.
+ * Token t of sequence s lives in page block_table[s][t / B].  Slots past
+ * seq_lens[s] inside the last page may hold anything (they are never used).
+ */
+typedef struct {
+    const void *k_pool;         /* dev bf16 [n_pages][Hkv][B][D] */
+    const void *v_pool;         /* dev bf16 [n_pages][Hkv][B][D] */
+    const int32_t *block_table; /* dev int32 [S][NBmax] page ids */
+    const int32_t *seq_lens;    /* dev int32 [S]: cached prefix tokens L_s (draft tokens not counted) */
+    int32_t n_pages;            /* pages in each pool */
+} sv_kv;
+
+/*
+ * Piecewise budget (Section 3.2, Eq. 6), host arithmetic only: the number of
+ * blocks to keep per KV head for a cache of L_seq tokens.  L_seq <= L0 keeps
+ * every block; otherwise ceil(((L_seq - L0) * rho + L0) / block_size), clamped
+ * to [n_sink + n_local, number of blocks].
+ */
+SV_API int32_t sv_budget_blocks(int64_t L_seq, int64_t L0, double rho, int32_t block_size, int32_t n_sink,
+                         int32_t n_local);
+
+/*
+ * Bytes of scratch that sv_verify_attn needs for this geometry when at most
+ * max_sel blocks are kept per (sequence, KV head) (pass max_blocks for dense
+ * attention).  Holds the per-split partial results of the split-KV kernel.
+ */
+SV_API size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel);
+
+/*
+ * Block representatives (Eq. 5: s = q0 . mean(k), so the representative of a
+ * block is its mean key).  Recomputes blocks block_begin <= b < block_end of
+ * every sequence (block_end < 0: up to the last block; blocks past a
+ * sequence's end are skipped).  The last block of a sequence is averaged over
+ * the tokens it holds.  Full blocks never change, so a decoding loop only
+ * needs to refresh the tail block.
+ *   reps: dev fp32 [S][Hkv][NBmax][D], written for the recomputed blocks only.
+ */
+SV_API sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
+                        float *reps, void *stream);
+
+/*
+ * Block selection (Section 3.1; Section 2.2: only the first draft token
+ * retrieves, every draft token shares its set; Section 3.3, Eq. 9: a
+ * non-anchor layer reuses the preceding layer's set).
+ *
+ * reuse_prev == 0: score[s][h][b] = mean_g(q[s][0][h*G+g]) . reps[s][h][b] in
+ *   fp32; the first n_sink and last n_local blocks are always kept (they count
+ *   against the budget); then the highest scores until budget_blocks[s] blocks
+ *   are kept (equal scores: smaller block index first).  A budget >= the
+ *   number of blocks keeps all of them.  The effective budget is clamped to
+ *   [forced blocks, max_sel].
+ * reuse_prev != 0: out_idx / out_cnt become copies of prev_idx / prev_cnt
+ *   (same shapes); q, reps and budget_blocks are not read.
+ *
+ *   q             dev bf16 [S][T][Hq][D]; only row 0 (the first draft token) is read
+ *   reps          dev fp32 [S][Hkv][NBmax][D] from sv_block_reps
+ *   seq_lens      dev int32 [S]
+ *   budget_blocks dev int32 [S]: N, blocks to keep per KV head
+ *   out_idx       dev int32 [S][Hkv][max_sel]: kept block indices, ascending; entries >= cnt untouched
+ *   out_cnt       dev int32 [S][Hkv]
+ *   out_scores    dev fp32 [S][Hkv][NBmax] or NULL (diagnostic copy of the scores)
+ * NBmax <= 32768.
+ */
+SV_API sv_status sv_select_blocks(const sv_geom *geom, const void *q, const float *reps, const int32_t *seq_lens,
+                           const int32_t *budget_blocks, int32_t n_sink, int32_t n_local, int32_t reuse_prev,
+                           const int32_t *prev_idx, const int32_t *prev_cnt, int32_t *out_idx,
+                           int32_t *out_cnt, int32_t max_sel, float *out_scores, void *stream);
+
+/*
+ * Sparse verification attention (Fig. 1; the 4B(1-s_a)T^2 d term of Table 1).
+ * For every sequence s, draft token i and query head hq (KV head h = hq / G):
+ * softmax(softmax_scale * q . k) . v over the cached tokens t < seq_lens[s] of
+ * the kept blocks sel_idx[s][h][0..sel_cnt[s][h]) and over the draft tokens
+ * visible to i: i itself and its ancestors through `parent` (parent[s][0] = -1,
+ * parent[s][i] < i), or tokens j <= i when parent is NULL (a chain).
+ * fp32 softmax and accumulation; probabilities are rounded to bf16 for the PV
+ * product.
+ *
+ *   q               dev bf16 [S][T][Hq][D]
+ *   draft_k/draft_v dev bf16 [S][T][Hkv][D]
+ *   parent          dev int32 [S][T] or NULL
+ *   sel_idx/sel_cnt as written by sv_select_blocks (ascending); sel_idx == NULL
+ *                   means dense verification: every block of every sequence
+ *                   (max_sel is then ignored, sel_cnt may be NULL)
+ *   softmax_scale   0 selects 1/sqrt(D)
+ *   out             dev bf16 [S][T][Hq][D]
+ *   lse             dev fp32 [S][T][Hq] natural-log softmax denominators, or NULL
+ *   workspace       dev scratch of at least sv_workspace_bytes(geom, max_sel)
+ *                   bytes, 16-byte aligned; contents are overwritten.  Calls
+ *                   that may overlap on the GPU need distinct workspaces.
+ *   status_word     dev int32 or NULL: set non-zero if a kernel gave up on a
+ *                   bounded wait (the output is then invalid)
+ */
+SV_API sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                         const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                         const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
+                         void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
+
+/* Number of KV splits (CTAs per (sequence, KV head)) sv_verify_attn uses for this geometry. */
+SV_API int32_t sv_verify_attn_splits(const sv_geom *geom, int32_t max_sel);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SV_H_ */

@@ -1,0 +1,9 @@
+"""Sparse verification attention for speculative decoding on B200 (sm_100a).
+
+CUDA library (csrc/, built into libsv.so) + a ctypes binding with the names of include/sv.h +
+``SparseVerifier``, a small driver that runs the per-layer select -> attention sequence for a stack of
+layers.  Importing the package loads the compiled library and fails if it is missing.
+"""
+from .binding import (SvError, make_geom, make_kv, sv_block_reps, sv_budget_blocks, sv_geom, sv_kv,  # noqa: F401
+                      sv_select_blocks, sv_verify_attn, sv_verify_attn_splits, sv_workspace_bytes, LIB_PATH, EXPORTS)
+from .engine import SparseVerifier  # noqa: F401

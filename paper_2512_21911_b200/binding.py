@@ -1,0 +1,147 @@
+"""ctypes binding of libsv.so: the same entry points as include/sv.h, taking torch CUDA tensors.
+
+Argument marshalling only -- every step of the path runs in the library's CUDA kernels.  torch is
+used for device memory and streams.  There is no CPU fallback: importing this module fails if the
+compiled library is missing.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsv.so")
+
+SV_OK = 0
+STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIGN", 4: "SV_ERR_BUDGET",
+                5: "SV_ERR_WORKSPACE", 6: "SV_ERR_UNSUPPORTED", 7: "SV_ERR_CUDA"}
+
+EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
+           "sv_verify_attn", "sv_verify_attn_splits")
+
+
+class SvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({_strerror(status)})")
+
+
+class sv_geom(ctypes.Structure):
+    _fields_ = [("n_seq", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("block_size", ctypes.c_int32), ("max_blocks", ctypes.c_int32),
+                ("n_draft", ctypes.c_int32)]
+
+
+class sv_kv(ctypes.Structure):
+    _fields_ = [("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p), ("block_table", ctypes.c_void_p),
+                ("seq_lens", ctypes.c_void_p), ("n_pages", ctypes.c_int32)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_21911_b200.build` "
+                          "(there is no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, f64, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_double,
+                                  ctypes.c_size_t)
+    gp, kp = ctypes.POINTER(sv_geom), ctypes.POINTER(sv_kv)
+    lib.sv_strerror.restype = ctypes.c_char_p
+    lib.sv_strerror.argtypes = [ctypes.c_int]
+    lib.sv_budget_blocks.restype = i32
+    lib.sv_budget_blocks.argtypes = [i64, i64, f64, i32, i32, i32]
+    lib.sv_workspace_bytes.restype = sz
+    lib.sv_workspace_bytes.argtypes = [gp, i32]
+    lib.sv_verify_attn_splits.restype = i32
+    lib.sv_verify_attn_splits.argtypes = [gp, i32]
+    lib.sv_block_reps.restype = ctypes.c_int
+    lib.sv_block_reps.argtypes = [gp, kp, i32, i32, vp, vp]
+    lib.sv_select_blocks.restype = ctypes.c_int
+    lib.sv_select_blocks.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
+    lib.sv_verify_attn.restype = ctypes.c_int
+    lib.sv_verify_attn.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
+    return lib
+
+
+_lib = _load()
+
+
+def _strerror(status: int) -> str:
+    return _lib.sv_strerror(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str) -> Optional[int]:
+    """Device pointer of a contiguous CUDA tensor of the given dtype (None -> NULL)."""
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != SV_OK:
+        raise SvError(status, where)
+
+
+def make_geom(n_seq, n_q_heads, n_kv_heads, head_dim, block_size, max_blocks, n_draft) -> sv_geom:
+    return sv_geom(n_seq, n_q_heads, n_kv_heads, head_dim, block_size, max_blocks, n_draft)
+
+
+def make_kv(k_pool: torch.Tensor, v_pool: Optional[torch.Tensor], block_table: torch.Tensor,
+            seq_lens: torch.Tensor) -> sv_kv:
+    """Paged KV descriptor.  Pools are bf16 [n_pages][Hkv][B][D]; the tensors must outlive the calls."""
+    return sv_kv(_ptr(k_pool, torch.bfloat16, "k_pool"), _ptr(v_pool, torch.bfloat16, "v_pool"),
+                 _ptr(block_table, torch.int32, "block_table"), _ptr(seq_lens, torch.int32, "seq_lens"),
+                 int(k_pool.shape[0]))
+
+
+def sv_budget_blocks(L_seq: int, L0: int, rho: float, block_size: int, n_sink: int = 0, n_local: int = 0) -> int:
+    return int(_lib.sv_budget_blocks(L_seq, L0, rho, block_size, n_sink, n_local))
+
+
+def sv_workspace_bytes(geom: sv_geom, max_sel: int) -> int:
+    return int(_lib.sv_workspace_bytes(ctypes.byref(geom), max_sel))
+
+
+def sv_verify_attn_splits(geom: sv_geom, max_sel: int) -> int:
+    return int(_lib.sv_verify_attn_splits(ctypes.byref(geom), max_sel))
+
+
+def sv_block_reps(geom: sv_geom, kv: sv_kv, reps: torch.Tensor, block_begin: int = 0, block_end: int = -1,
+                  stream=None) -> None:
+    _check(_lib.sv_block_reps(ctypes.byref(geom), ctypes.byref(kv), block_begin, block_end,
+                              _ptr(reps, torch.float32, "reps"), _stream(stream)), "sv_block_reps")
+
+
+def sv_select_blocks(geom: sv_geom, q, reps, seq_lens, budget_blocks, n_sink: int, n_local: int, out_idx, out_cnt,
+                     reuse_prev: bool = False, prev_idx=None, prev_cnt=None, out_scores=None, stream=None) -> None:
+    max_sel = int(out_idx.shape[-1])
+    _check(_lib.sv_select_blocks(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), _ptr(reps, torch.float32, "reps"),
+                                 _ptr(seq_lens, torch.int32, "seq_lens"),
+                                 _ptr(budget_blocks, torch.int32, "budget_blocks"), n_sink, n_local,
+                                 1 if reuse_prev else 0, _ptr(prev_idx, torch.int32, "prev_idx"),
+                                 _ptr(prev_cnt, torch.int32, "prev_cnt"), _ptr(out_idx, torch.int32, "out_idx"),
+                                 _ptr(out_cnt, torch.int32, "out_cnt"), max_sel,
+                                 _ptr(out_scores, torch.float32, "out_scores"), _stream(stream)), "sv_select_blocks")
+
+
+def sv_verify_attn(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=None,
+                   workspace=None, softmax_scale: float = 0.0, status_word=None, stream=None) -> None:
+    max_sel = int(sel_idx.shape[-1]) if sel_idx is not None else int(geom.max_blocks)
+    ws_ptr = workspace.data_ptr() if workspace is not None else None
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    if workspace is not None and not workspace.is_cuda:
+        raise TypeError("workspace must be a CUDA tensor")
+    _check(_lib.sv_verify_attn(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), ctypes.byref(kv),
+                               _ptr(draft_k, torch.bfloat16, "draft_k"), _ptr(draft_v, torch.bfloat16, "draft_v"),
+                               _ptr(parent, torch.int32, "parent"), _ptr(sel_idx, torch.int32, "sel_idx"),
+                               _ptr(sel_cnt, torch.int32, "sel_cnt"), max_sel, float(softmax_scale),
+                               _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"), ws_ptr, ws_bytes,
+                               _ptr(status_word, torch.int32, "status_word"), _stream(stream)), "sv_verify_attn")

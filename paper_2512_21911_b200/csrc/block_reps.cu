@@ -1,0 +1,90 @@
+// sv_block_reps: mean key of every KV block (the block representative implied by Eq. 5).
+//
+// Pure streaming reduction, bound by HBM bandwidth: one CTA per (block, KV head,
+// sequence) reads the contiguous B x 128 bf16 tile of the block with 128-bit loads
+// (all of a thread's loads are issued before the first use), accumulates in fp32 in a
+// fixed order and writes 128 fp32 values.  Algorithmic traffic: B*256 bytes read +
+// 512 bytes written per block.
+#include <cuda_bf16.h>
+
+#include "sv_host.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRowGroups = kThreads / 16;   // 16 threads cover one 256-byte key row
+
+template <int B>
+__global__ void __launch_bounds__(kThreads) block_reps_kernel(const uint4 *__restrict__ k_pool,
+                                                              const int32_t *__restrict__ block_table,
+                                                              const int32_t *__restrict__ seq_lens,
+                                                              float *__restrict__ reps, int Hkv, int NBmax,
+                                                              int block_begin, int block_end)
+{
+    const int s = blockIdx.z, h = blockIdx.y;
+    const int b = block_begin + blockIdx.x;
+    const int L = seq_lens[s];
+    const int nb = (L + B - 1) / B;
+    if (b >= nb || (block_end >= 0 && b >= block_end)) return;
+    const int cnt = min(B, L - b * B);
+    const int page = block_table[(size_t)s * NBmax + b];
+    const uint4 *tile = k_pool + ((size_t)page * Hkv + h) * (B * 16);
+
+    const int chunk = threadIdx.x & 15;     // 8 dims = one 16-byte chunk of the row
+    const int rg = threadIdx.x >> 4;
+    constexpr int kIter = B / kRowGroups;
+    uint4 v[kIter];
+#pragma unroll
+    for (int i = 0; i < kIter; ++i) {
+        const int row = rg + i * kRowGroups;
+        v[i] = row < cnt ? __ldg(tile + row * 16 + chunk) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < kIter; ++i) {
+        const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&v[i]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __bfloat1622float2(p[j]);
+            acc[2 * j] += f.x;
+            acc[2 * j + 1] += f.y;
+        }
+    }
+    __shared__ float part[kRowGroups][128];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) part[rg][chunk * 8 + j] = acc[j];
+    __syncthreads();
+    if (threadIdx.x < 128) {
+        float sum = 0.f;
+#pragma unroll
+        for (int g = 0; g < kRowGroups; ++g) sum += part[g][threadIdx.x];
+        reps[(((size_t)s * Hkv + h) * NBmax + b) * 128 + threadIdx.x] = sum / (float)cnt;
+    }
+}
+
+}  // namespace
+
+extern "C" sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
+                                   float *reps, void *stream)
+{
+    sv_status st = svh::check_geom(geom);
+    if (st != SV_OK) return st;
+    st = svh::check_kv(geom, kv, false);
+    if (st != SV_OK) return st;
+    if (!reps) return SV_ERR_NULL;
+    if (!svh::aligned(reps, 16)) return SV_ERR_ALIGN;
+    if (block_begin < 0) return SV_ERR_SHAPE;
+    const int hi = (block_end < 0 || block_end > geom->max_blocks) ? geom->max_blocks : block_end;
+    if (hi <= block_begin) return SV_OK;   // empty range: nothing to do
+    dim3 grid(hi - block_begin, geom->n_kv_heads, geom->n_seq);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (geom->block_size == 64)
+        block_reps_kernel<64><<<grid, kThreads, 0, cs>>>(static_cast<const uint4 *>(kv->k_pool), kv->block_table,
+                                                         kv->seq_lens, reps, geom->n_kv_heads, geom->max_blocks,
+                                                         block_begin, block_end);
+    else
+        block_reps_kernel<128><<<grid, kThreads, 0, cs>>>(static_cast<const uint4 *>(kv->k_pool), kv->block_table,
+                                                          kv->seq_lens, reps, geom->n_kv_heads, geom->max_blocks,
+                                                          block_begin, block_end);
+    return svh::launch_status();
+}

@@ -1,0 +1,46 @@
+// Host-side helpers shared by the entry points: argument checks and launch-error mapping.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sv.h"
+
+namespace svh {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxRows = 128;      // G * T rows packed per KV head
+constexpr int kMaxDraft = 32;      // ancestor masks are 32-bit
+constexpr int kMaxBlocksSelect = 32768;
+
+inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+inline sv_status check_geom(const sv_geom *g)
+{
+    if (!g) return SV_ERR_NULL;
+    if (g->n_seq < 1 || g->n_q_heads < 1 || g->n_kv_heads < 1 || g->max_blocks < 1 || g->n_draft < 1)
+        return SV_ERR_SHAPE;
+    if (g->n_q_heads % g->n_kv_heads) return SV_ERR_SHAPE;
+    if (g->head_dim != kHeadDim) return SV_ERR_UNSUPPORTED;
+    if (g->block_size != 64 && g->block_size != 128) return SV_ERR_UNSUPPORTED;
+    if (g->n_draft > kMaxDraft) return SV_ERR_UNSUPPORTED;
+    if ((g->n_q_heads / g->n_kv_heads) * g->n_draft > kMaxRows) return SV_ERR_UNSUPPORTED;
+    if (g->n_seq > 65535 || g->n_kv_heads > 65535) return SV_ERR_SHAPE;
+    return SV_OK;
+}
+
+inline sv_status check_kv(const sv_geom *g, const sv_kv *kv, bool need_v)
+{
+    if (!kv || !kv->k_pool || !kv->block_table || !kv->seq_lens || (need_v && !kv->v_pool)) return SV_ERR_NULL;
+    if (kv->n_pages < 1) return SV_ERR_SHAPE;
+    if ((int64_t)kv->n_pages * g->n_kv_heads * g->block_size >= (int64_t)1 << 31) return SV_ERR_SHAPE;
+    if (!aligned(kv->k_pool, 128) || (need_v && !aligned(kv->v_pool, 128))) return SV_ERR_ALIGN;
+    if (!aligned(kv->block_table, 4) || !aligned(kv->seq_lens, 4)) return SV_ERR_ALIGN;
+    return SV_OK;
+}
+
+inline sv_status launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? SV_OK : SV_ERR_CUDA;
+}
+
+}  // namespace svh

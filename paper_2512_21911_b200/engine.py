@@ -1,0 +1,74 @@
+"""SparseVerifier: runs block selection and sparse verification attention for a stack of layers.
+
+A thin driver over the C-ABI calls: it owns the per-layer representatives, the shared block list,
+the split-KV workspace and the outputs, and enqueues, per layer, ``sv_select_blocks`` (anchor
+layers) or the reuse of the previous layer's list (Eq. 9), then ``sv_verify_attn``.  All compute is in
+the library's kernels; this class only holds buffers and calls them in order.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import binding as sv
+
+
+class SparseVerifier:
+    def __init__(self, *, n_seq: int, n_q_heads: int, n_kv_heads: int, head_dim: int, block_size: int,
+                 max_blocks: int, n_draft: int, n_layers: int, block_table: torch.Tensor, seq_lens: torch.Tensor,
+                 budget_blocks: torch.Tensor, max_sel: int, n_sink: int = 1, n_local: int = 1,
+                 anchors: Optional[Sequence[bool]] = None, parent: Optional[torch.Tensor] = None,
+                 device: str = "cuda"):
+        self.geom = sv.make_geom(n_seq, n_q_heads, n_kv_heads, head_dim, block_size, max_blocks, n_draft)
+        self.n_layers = n_layers
+        self.block_table, self.seq_lens, self.budget, self.parent = block_table, seq_lens, budget_blocks, parent
+        self.n_sink, self.n_local, self.max_sel = n_sink, n_local, max_sel
+        self.anchors = list(anchors) if anchors is not None else [True] * n_layers
+        assert self.anchors[0], "layer 0 has no preceding layer to reuse"
+        dev = torch.device(device)
+        self.reps = torch.zeros((n_layers, n_seq, n_kv_heads, max_blocks, head_dim), dtype=torch.float32, device=dev)
+        self.sel_idx = torch.zeros((n_seq, n_kv_heads, max_sel), dtype=torch.int32, device=dev)
+        self.sel_cnt = torch.zeros((n_seq, n_kv_heads), dtype=torch.int32, device=dev)
+        self.workspace = torch.empty(max(16, sv.sv_workspace_bytes(self.geom, max_sel)), dtype=torch.uint8, device=dev)
+        self.dense_workspace = None
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.kv: List[Optional[sv.sv_kv]] = [None] * n_layers
+        self._pools = [None] * n_layers   # keep the tensors alive
+
+    def set_layer_kv(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
+        self._pools[layer] = (k_pool, v_pool)
+        self.kv[layer] = sv.make_kv(k_pool, v_pool, self.block_table, self.seq_lens)
+
+    def build_reps(self, layer: int, block_begin: int = 0, block_end: int = -1) -> None:
+        """(Re)compute block representatives of a layer; a decoding loop only refreshes the tail block."""
+        sv.sv_block_reps(self.geom, self.kv[layer], self.reps[layer], block_begin, block_end)
+
+    def verify_layer(self, layer: int, q, draft_k, draft_v, out, lse=None) -> None:
+        """select (anchor) or reuse (non-anchor), then sparse verification attention, on the current stream."""
+        if self.anchors[layer]:
+            sv.sv_select_blocks(self.geom, q, self.reps[layer], self.seq_lens, self.budget, self.n_sink,
+                                self.n_local, self.sel_idx, self.sel_cnt)
+        else:   # Eq. 9: same list as the preceding layer; in place, so nothing is launched
+            sv.sv_select_blocks(self.geom, None, None, None, None, self.n_sink, self.n_local, self.sel_idx,
+                                self.sel_cnt, reuse_prev=True, prev_idx=self.sel_idx, prev_cnt=self.sel_cnt)
+        sv.sv_verify_attn(self.geom, q, self.kv[layer], draft_k, draft_v, self.parent, self.sel_idx, self.sel_cnt,
+                          out, lse=lse, workspace=self.workspace, status_word=self.status)
+
+    def dense_layer(self, layer: int, q, draft_k, draft_v, out, lse=None) -> None:
+        """Dense ("strict") verification attention over every cached block, for comparison."""
+        if self.dense_workspace is None:
+            n = max(16, sv.sv_workspace_bytes(self.geom, self.geom.max_blocks))
+            self.dense_workspace = torch.empty(n, dtype=torch.uint8, device=self.workspace.device)
+        sv.sv_verify_attn(self.geom, q, self.kv[layer], draft_k, draft_v, self.parent, None, None, out, lse=lse,
+                          workspace=self.dense_workspace, status_word=self.status)
+
+    def verify_step(self, q, draft_k, draft_v, out) -> None:
+        """One verification step of the whole stack.  q/out: [layers][S][T][Hq][D]; draft_k/v: [layers][S][T][Hkv][D]."""
+        for l in range(self.n_layers):
+            self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l])
+
+    def kernels_per_step(self) -> int:
+        """Kernel launches of one verify_step (select per anchor layer; attention (+ merge) per layer)."""
+        splits = sv.sv_verify_attn_splits(self.geom, self.max_sel)
+        return sum(self.anchors) + self.n_layers * (2 if splits > 1 else 1)

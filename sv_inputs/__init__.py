@@ -147,7 +147,8 @@ def make_layer(geom: dict, layer: int = 0, sharp: bool = False, tail_fill: Optio
     """Tensors of one layer of a case (see the module docstring for the recipe).
 
     Returns q, k_pool, v_pool, draft_k, draft_v as uint16 bf16 bits plus the geometry entries,
-    ``min_gap`` (smallest kept-vs-evicted score gap over all (s, h)), ``delta`` and ``planted``.
+    ``min_gap`` (smallest kept-vs-evicted score gap over all (s, h)), ``delta`` (largest per-(s, h) margin
+    asked for), ``min_gap_ratio`` (smallest gap / delta of any (s, h); >= 1 after repair) and ``planted``.
     ``tail_fill``: value written to K and V slots past the end of a sequence inside its last page
     (a correct kernel never lets them contribute); ``None`` writes NaN bit patterns.
     """
@@ -171,6 +172,7 @@ def make_layer(geom: dict, layer: int = 0, sharp: bool = False, tail_fill: Optio
     v_pool[...] = fill_bits
 
     min_gap = np.inf
+    min_ratio = np.inf
     delta_used = 0.0
     planted_sets = {}
     for s in range(S):
@@ -221,7 +223,9 @@ def make_layer(geom: dict, layer: int = 0, sharp: bool = False, tail_fill: Optio
                 else:
                     raise RuntimeError("gap repair did not converge")
                 order = cand[np.argsort(-sc[cand], kind="stable")]
-                min_gap = min(min_gap, float(sc[order[need - 1]] - sc[order[need]]))
+                gap = float(sc[order[need - 1]] - sc[order[need]])
+                min_gap = min(min_gap, gap)
+                min_ratio = min(min_ratio, gap / delta)
             vb = f32_to_bf16_bits(v)
             kb[~tok_valid] = fill_bits
             vb[~tok_valid] = fill_bits
@@ -230,7 +234,7 @@ def make_layer(geom: dict, layer: int = 0, sharp: bool = False, tail_fill: Optio
 
     out = dict(geom)
     out.update(q=q, k_pool=k_pool, v_pool=v_pool, draft_k=draft_k, draft_v=draft_v, layer=layer,
-               min_gap=min_gap, delta=delta_used, planted=planted_sets, sharp=sharp)
+               min_gap=min_gap, delta=delta_used, min_gap_ratio=min_ratio, planted=planted_sets, sharp=sharp)
     return out
 
 

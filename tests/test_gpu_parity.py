@@ -1,0 +1,348 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle, element by element,
+on the same seeded bf16 inputs.
+
+Bars: kept block indices and counts bit-exact; attention outputs within max-abs 1e-2 and mean-abs 1e-3
+(the stated tolerance) and, because those are loose for the N(0,1)/sqrt(128) generator, also a
+per-row relative L2 error <= 1e-2 and |lse - lse*| <= 1e-3; every case also runs with the
+"sharp" generator (logit std ~3), where a wrong mask, a dropped block or a wrong tail bound
+fails by orders of magnitude.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import sv_inputs as si
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sv():
+    import paper_2512_21911_b200 as pkg
+    return pkg
+
+
+def bf16_dev(a):
+    return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def bf16_host(t):
+    return si.bf16_bits_to_f64(t.cpu().view(torch.int16).numpy().view(np.uint16))
+
+
+class Dev:
+    """Device copies of a generated case + the geometry descriptors."""
+
+    def __init__(self, sv, c):
+        w = c["workload"]
+        self.c, self.w = c, w
+        self.geom = sv.make_geom(w.n_seq, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, c["max_blocks"], w.n_draft)
+        self.q, self.k_pool, self.v_pool = bf16_dev(c["q"]), bf16_dev(c["k_pool"]), bf16_dev(c["v_pool"])
+        self.draft_k, self.draft_v = bf16_dev(c["draft_k"]), bf16_dev(c["draft_v"])
+        self.block_table = torch.from_numpy(c["block_table"]).cuda()
+        self.seq_lens = torch.from_numpy(c["seq_lens"]).cuda()
+        self.budget = torch.from_numpy(c["budget"]).cuda()
+        self.parent = torch.from_numpy(c["parent"]).cuda() if c["parent"] is not None else None
+        self.kv = sv.make_kv(self.k_pool, self.v_pool, self.block_table, self.seq_lens)
+        self.reps = torch.full((w.n_seq, w.n_kv_heads, c["max_blocks"], w.head_dim), float("nan"), device="cuda")
+
+
+def gpu_select(sv, d, n_sink, n_local, max_sel, scores=False):
+    sv.sv_block_reps(d.geom, d.kv, d.reps)
+    idx = torch.full((d.w.n_seq, d.w.n_kv_heads, max_sel), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((d.w.n_seq, d.w.n_kv_heads), -7, dtype=torch.int32, device="cuda")
+    sc = torch.full((d.w.n_seq, d.w.n_kv_heads, d.c["max_blocks"]), float("nan"), device="cuda") if scores else None
+    sv.sv_select_blocks(d.geom, d.q, d.reps, d.seq_lens, d.budget, n_sink, n_local, idx, cnt, out_scores=sc)
+    return idx, cnt, sc
+
+
+def gpu_attn(sv, d, idx, cnt):
+    w = d.w
+    out = torch.full((w.n_seq, w.n_draft, w.n_q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((w.n_seq, w.n_draft, w.n_q_heads), float("nan"), device="cuda")
+    max_sel = idx.shape[-1] if idx is not None else d.c["max_blocks"]
+    ws = torch.empty(max(16, sv.sv_workspace_bytes(d.geom, max_sel)), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sv.sv_verify_attn(d.geom, d.q, d.kv, d.draft_k, d.draft_v, d.parent, idx, cnt, out, lse=lse, workspace=ws,
+                      status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return bf16_host(out), lse.cpu().numpy().astype(np.float64)
+
+
+def check_attn(o, lse, o_ref, lse_ref, what=""):
+    assert np.isfinite(o).all() and np.isfinite(lse).all(), what
+    err = np.abs(o - o_ref)
+    scale = max(1.0, float(np.abs(o_ref).max()))
+    assert err.max() <= 1e-2 * scale, (what, err.max())
+    assert err.mean() <= 1e-3 * scale, (what, err.mean())
+    rel = np.linalg.norm(o - o_ref, axis=-1) / np.linalg.norm(o_ref, axis=-1)
+    assert rel.max() <= 1e-2, (what, rel.max())
+    assert np.abs(lse - lse_ref).max() <= 1e-3, (what, np.abs(lse - lse_ref).max())
+
+
+def oracle_select(c, n_sink, n_local, max_sel):
+    return oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], n_sink, n_local, max_sel)
+
+
+def oracle_attn(c, idx, cnt, samples=None):
+    return oracle.verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"],
+                              c["draft_v"], c["parent"], idx, cnt, samples=samples)
+
+
+def run_pipeline(sv, c, n_sink=None, n_local=None, what=""):
+    """reps -> select -> attention on the GPU, compared stage by stage with the oracle."""
+    n_sink = c["n_sink"] if n_sink is None else n_sink
+    n_local = c["n_local"] if n_local is None else n_local
+    d = Dev(sv, c)
+    idx, cnt, sc = gpu_select(sv, d, n_sink, n_local, c["max_sel"], scores=True)
+    torch.cuda.synchronize()
+    idx_ref, cnt_ref, sc_ref = oracle_select(c, n_sink, n_local, c["max_sel"])
+    reps_ref = oracle.block_reps(c["k_pool"], c["block_table"], c["seq_lens"])
+    reps = d.reps.cpu().numpy().astype(np.float64)
+    for s in range(d.w.n_seq):
+        nb = int(c["n_blocks"][s])
+        np.testing.assert_allclose(reps[s, :, :nb], reps_ref[s, :, :nb], rtol=1e-5, atol=1e-6 * max(1.0, np.abs(reps_ref).max()))
+        assert np.isnan(reps[s, :, nb:]).all()                       # blocks past the end are not written
+        tol = 1e-5 * max(1.0, float(np.abs(sc_ref[s, :, :nb]).max()))
+        np.testing.assert_allclose(sc.cpu().numpy()[s, :, :nb], sc_ref[s, :, :nb], rtol=0, atol=tol)
+    cnt_h, idx_h = cnt.cpu().numpy(), idx.cpu().numpy()
+    np.testing.assert_array_equal(cnt_h, cnt_ref)
+    for s in range(d.w.n_seq):
+        for h in range(d.w.n_kv_heads):
+            n = cnt_ref[s, h]
+            np.testing.assert_array_equal(idx_h[s, h, :n], idx_ref[s, h, :n], err_msg=f"{what} s={s} h={h}")
+            assert (idx_h[s, h, n:] == -7).all()
+    o, lse = gpu_attn(sv, d, idx, cnt)
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref)
+    check_attn(o, lse, o_ref, lse_ref, what)
+    return d, idx, cnt, o, lse
+
+
+SMALL = {
+    # rows = G*T: 16 (1 warp row), 32, 20 (ragged batch), 64, 128 (block 128, tree)
+    "cfg0": si.WORKLOADS["cfg0"],
+    "cfg1_small": si.shrink(si.WORKLOADS["cfg1"], seq_len=(4096, 4096), budget_blocks=20, n_layers=1),
+    "cfg2_small": si.shrink(si.WORKLOADS["cfg2"], n_seq=5, seq_len=(700, 3000), budget_blocks=9),
+    "rows64": si.shrink(si.WORKLOADS["cfg1"], seq_len=(2500, 2500), budget_blocks=12, n_draft=16, n_layers=1, tree=True),
+    "cfg3_small": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(5000, 9000), budget_blocks=11, planted=3),
+    "rows4": si.shrink(si.WORKLOADS["cfg1"], seq_len=(2048, 2048), budget_blocks=8, n_draft=1, n_layers=1),
+    "t32": si.shrink(si.WORKLOADS["cfg0"], seq_len=(1000, 1000), budget_blocks=5, n_draft=32, tree=True, planted=2),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+@pytest.mark.parametrize("sharp", [False, True])
+def test_pipeline_parity_small(sv, name, sharp):
+    c = si.make_layer(si.make_geometry(SMALL[name]), sharp=sharp)
+    assert c["min_gap_ratio"] >= 1.0
+    run_pipeline(sv, c, what=f"{name} sharp={sharp}")
+
+
+@pytest.mark.parametrize("forced", [(0, 0), (2, 4)])
+def test_sink_local_variants(sv, forced):
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(900, 2000), budget_blocks=10, n_sink=forced[0], n_local=forced[1])
+    c = si.make_layer(si.make_geometry(w), sharp=True)
+    run_pipeline(sv, c, what=f"forced={forced}")
+
+
+def test_nan_in_unused_tail_slots_is_harmless(sv):
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(900, 2000), budget_blocks=10)
+    c = si.make_layer(si.make_geometry(w), sharp=True, tail_fill=None)
+    run_pipeline(sv, c, what="nan tail")
+
+
+def test_budget_covering_all_blocks_is_dense(sv):
+    """Fixed point: nothing evicted -> the sparse path equals dense verification; sel_idx=NULL is the same."""
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(500, 1500), budget_blocks=10**6)
+    geom = si.make_geometry(w)
+    geom["max_sel"] = geom["max_blocks"]
+    c = si.make_layer(geom, sharp=True)
+    d, idx, cnt, o, lse = run_pipeline(sv, c, what="full budget")
+    np.testing.assert_array_equal(cnt.cpu().numpy(), np.repeat(c["n_blocks"][:, None], w.n_kv_heads, axis=1))
+    od_ref, lsed_ref = oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                                c["draft_k"], c["draft_v"], c["parent"])
+    check_attn(o, lse, od_ref, lsed_ref, "sparse(all) vs dense oracle")
+    o2, lse2 = gpu_attn(sv, d, None, None)
+    check_attn(o2, lse2, od_ref, lsed_ref, "dense entry")
+
+
+def test_selection_ties_and_first_token_only(sv):
+    """All-zero keys: every score ties, smaller indices win.  Other draft rows never change the set."""
+    w = si.shrink(si.WORKLOADS["cfg0"], seq_len=(1500, 1500), budget_blocks=7)
+    c = si.make_layer(si.make_geometry(w))
+    z = dict(c)
+    z["k_pool"] = np.zeros_like(c["k_pool"])
+    d = Dev(sv, z)
+    idx, cnt, _ = gpu_select(sv, d, 1, 1, 7)
+    torch.cuda.synchronize()
+    assert (cnt.cpu().numpy() == 7).all()
+    assert (idx.cpu().numpy() == np.array([0, 1, 2, 3, 4, 5, 23])).all()
+    idx_ref, _, _ = oracle_select(z, 1, 1, 7)
+    np.testing.assert_array_equal(idx.cpu().numpy(), idx_ref)
+    d1 = Dev(sv, c)
+    a, _, _ = gpu_select(sv, d1, 1, 1, 7)
+    c2 = dict(c)
+    c2["q"] = c["q"].copy()
+    c2["q"][:, 1:] = si.f32_to_bf16_bits(np.random.default_rng(1).standard_normal(c["q"][:, 1:].shape).astype(np.float32))
+    b, _, _ = gpu_select(sv, Dev(sv, c2), 1, 1, 7)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_reuse_prev_copies_previous_layer(sv):
+    w = si.shrink(si.WORKLOADS["cfg0"], seq_len=(1500, 1500), budget_blocks=7)
+    c = si.make_layer(si.make_geometry(w))
+    d = Dev(sv, c)
+    idx, cnt, _ = gpu_select(sv, d, 1, 1, 7)
+    idx2, cnt2 = torch.zeros_like(idx), torch.zeros_like(cnt)
+    sv.sv_select_blocks(d.geom, None, None, None, None, 1, 1, idx2, cnt2, reuse_prev=True, prev_idx=idx, prev_cnt=cnt)
+    torch.cuda.synchronize()
+    assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2)
+    with pytest.raises(sv.SvError):
+        sv.sv_select_blocks(d.geom, None, None, None, None, 1, 1, idx2, cnt2, reuse_prev=True)
+
+
+def test_block_reps_range_update(sv):
+    """Only the requested block range is rewritten (a decoding loop refreshes the tail block only)."""
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(900, 2000), budget_blocks=10)
+    c = si.make_layer(si.make_geometry(w))
+    d = Dev(sv, c)
+    sv.sv_block_reps(d.geom, d.kv, d.reps)
+    full = d.reps.clone()
+    d.reps.fill_(123.0)
+    sv.sv_block_reps(d.geom, d.kv, d.reps, 3, 6)
+    torch.cuda.synchronize()
+    assert torch.equal(d.reps[:, :, 3:6], full[:, :, 3:6])
+    assert (d.reps[:, :, :3] == 123.0).all() and (d.reps[:, :, 6:] == 123.0).all()
+
+
+def test_empty_prefix_and_empty_selection(sv):
+    """A sequence with no cached tokens attends to its draft tokens only; so does an empty block list."""
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(300, 900), budget_blocks=4, tree=True)
+    geom = si.make_geometry(w)
+    c = si.make_layer(geom, sharp=True)
+    c["seq_lens"] = c["seq_lens"].copy()
+    c["seq_lens"][1] = 0
+    c["n_blocks"] = ((c["seq_lens"] + 63) // 64).astype(np.int32)
+    d = Dev(sv, c)
+    idx, cnt, _ = gpu_select(sv, d, 1, 1, c["max_sel"])
+    torch.cuda.synchronize()
+    idx_ref, cnt_ref, _ = oracle_select(c, 1, 1, c["max_sel"])
+    np.testing.assert_array_equal(cnt.cpu().numpy(), cnt_ref)
+    assert (cnt_ref[1] == 0).all()
+    o, lse = gpu_attn(sv, d, idx, cnt)
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref)
+    check_attn(o, lse, o_ref, lse_ref, "empty prefix")
+    cnt0 = torch.zeros_like(cnt)
+    o, lse = gpu_attn(sv, d, idx, cnt0)
+    o_ref, lse_ref = oracle_attn(c, idx_ref, np.zeros_like(cnt_ref))
+    check_attn(o, lse, o_ref, lse_ref, "empty selection")
+
+
+def test_more_splits_than_blocks(sv):
+    """One (sequence, KV head) pair: the split count is capped by the block count, some CTAs get one block."""
+    w = si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=1, seq_len=(2000, 2000), budget_blocks=3, planted=1)
+    c = si.make_layer(si.make_geometry(w), sharp=True)
+    d = run_pipeline(sv, c, what="3 blocks")[0]
+    assert sv.sv_verify_attn_splits(d.geom, 3) == 3
+
+
+def test_workspace_too_small_is_rejected(sv):
+    c = si.make_layer(si.make_geometry(SMALL["cfg0"]))
+    d = Dev(sv, c)
+    idx, cnt, _ = gpu_select(sv, d, 1, 1, 16)
+    out = torch.zeros((1, 4, 8, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(sv.SvError) as e:
+        sv.sv_verify_attn(d.geom, d.q, d.kv, d.draft_k, d.draft_v, None, idx, cnt, out, workspace=ws)
+    assert e.value.status == 5
+
+
+def test_layer_stack_with_reuse_matches_oracle(sv):
+    """SparseVerifier over 4 layers, anchors on even layers (Eq. 9), against the oracle's layer loop."""
+    w = si.shrink(si.WORKLOADS["cfg1"], seq_len=(4096, 4096), budget_blocks=12, n_layers=4)
+    geom = si.make_geometry(w)
+    layers = [si.make_layer(geom, layer=l, sharp=True) for l in range(4)]
+    anchors = [True, False, True, False]
+    ref_sel = oracle.select_layers(layers, anchors, geom["budget"], 1, 1, geom["max_sel"])
+    eng = sv.SparseVerifier(n_seq=1, n_q_heads=32, n_kv_heads=8, head_dim=128, block_size=64,
+                            max_blocks=geom["max_blocks"], n_draft=8, n_layers=4,
+                            block_table=torch.from_numpy(geom["block_table"]).cuda(),
+                            seq_lens=torch.from_numpy(geom["seq_lens"]).cuda(),
+                            budget_blocks=torch.from_numpy(geom["budget"]).cuda(), max_sel=geom["max_sel"],
+                            anchors=anchors)
+    q = torch.stack([bf16_dev(c["q"]) for c in layers])
+    dk = torch.stack([bf16_dev(c["draft_k"]) for c in layers])
+    dv = torch.stack([bf16_dev(c["draft_v"]) for c in layers])
+    out = torch.zeros_like(q)
+    for l, c in enumerate(layers):
+        eng.set_layer_kv(l, bf16_dev(c["k_pool"]), bf16_dev(c["v_pool"]))
+        eng.build_reps(l)
+    eng.verify_step(q, dk, dv, out)
+    torch.cuda.synchronize()
+    assert int(eng.status.item()) == 0
+    for l, c in enumerate(layers):
+        o_ref, _ = oracle_attn(c, *ref_sel[l])
+        o = bf16_host(out[l])
+        rel = np.linalg.norm(o - o_ref, axis=-1) / np.linalg.norm(o_ref, axis=-1)
+        assert rel.max() <= 1e-2, (l, rel.max())
+    np.testing.assert_array_equal(eng.sel_idx.cpu().numpy(), ref_sel[2][0])
+    assert eng.kernels_per_step() == 2 + 4 * (2 if sv.sv_verify_attn_splits(eng.geom, geom["max_sel"]) > 1 else 1)
+
+
+# ------------------------------------------------------------------ full-size configurations
+
+def _sampled_check(sv, c, n_samples, what):
+    d = Dev(sv, c)
+    idx, cnt, _ = gpu_select(sv, d, c["n_sink"], c["n_local"], c["max_sel"])
+    torch.cuda.synchronize()
+    idx_ref, cnt_ref, _ = oracle_select(c, c["n_sink"], c["n_local"], c["max_sel"])
+    np.testing.assert_array_equal(cnt.cpu().numpy(), cnt_ref)
+    np.testing.assert_array_equal(idx.cpu().numpy(), idx_ref)
+    o, lse = gpu_attn(sv, d, idx, cnt)
+    w = c["workload"]
+    g = np.random.default_rng(7)
+    smp = np.stack([g.integers(0, w.n_seq, n_samples), g.integers(0, w.n_draft, n_samples),
+                    g.integers(0, w.n_q_heads, n_samples)], axis=1).astype(np.int32)
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref, samples=smp)
+    o_s = np.stack([o[s, i, hq] for s, i, hq in smp])
+    lse_s = np.array([lse[s, i, hq] for s, i, hq in smp])
+    check_attn(o_s, lse_s, o_ref, lse_ref, what)
+    # properties that hold at any size: finite everywhere, and (V rows are random) outputs bounded by max |v|
+    assert np.isfinite(o).all()
+    return d, idx, cnt
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_full_size_cfg1_one_layer(sv, sharp):
+    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg1"]), layer=3, sharp=sharp)
+    run_pipeline(sv, c, what=f"cfg1 sharp={sharp}")
+
+
+def test_full_size_cfg1_dense_sampled(sv):
+    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg1"]), layer=0, sharp=True)
+    d = Dev(sv, c)
+    o, lse = gpu_attn(sv, d, None, None)
+    smp = [(0, 7, 31), (0, 0, 0), (0, 3, 17), (0, 5, 9)]
+    o_ref, lse_ref = oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                              c["draft_k"], c["draft_v"], None, samples=smp)
+    check_attn(np.stack([o[s, i, h] for s, i, h in smp]), np.array([lse[s, i, h] for s, i, h in smp]), o_ref, lse_ref,
+               "cfg1 dense")
+
+
+def test_full_size_cfg2(sv):
+    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg2"]), sharp=True)
+    run_pipeline(sv, c, what="cfg2")
+
+
+def test_full_size_cfg3_sampled(sv):
+    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg3"]), sharp=True)
+    _sampled_check(sv, c, 64, "cfg3")
+
+
+@pytest.mark.parametrize("point", [(8192, 1 / 32, 1), (32768, 1 / 8, 16), (131072, 1 / 4, 4)])
+def test_sweep_points(sv, point):
+    c = si.make_layer(si.make_geometry(si.sweep_workload(*point)), sharp=True)
+    _sampled_check(sv, c, 48, f"sweep {point}")

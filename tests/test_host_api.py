@@ -1,0 +1,86 @@
+"""Host-side checks that need no GPU: the library loads, exports every declared symbol, validates
+arguments before touching the device, and its budget helper follows Eq. 6."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def svb():
+    # build through the file path: importing the package would already load a stale library
+    subprocess.run([sys.executable, os.path.join(ROOT, "paper_2512_21911_b200", "build.py")], check=True,
+                   capture_output=True)
+    import paper_2512_21911_b200.binding as b
+    return b
+
+
+def test_exports_every_declared_symbol(svb):
+    header = open(os.path.join(ROOT, "include", "sv.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(sv_[a-z_]+)\s*\(", header))
+    assert declared == set(svb.EXPORTS)
+    lib = ctypes.CDLL(svb.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_strerror_texts(svb):
+    texts = {svb._strerror(i) for i in range(8)}
+    assert len(texts) == 8 and "ok" in texts
+    assert svb._strerror(99) == "unknown status"
+
+
+def test_budget_matches_eq6_and_oracle(svb):
+    for L in (100, 4096, 4097, 6300, 32768, 131072, 1000003):
+        for L0 in (1024, 4096):
+            for rho in (0.05, 0.1, 0.5):
+                for B in (64, 128):
+                    for forced in ((0, 0), (1, 1), (2, 4)):
+                        assert svb.sv_budget_blocks(L, L0, rho, B, *forced) == oracle.budget_blocks(L, L0, rho, B, *forced)
+    assert svb.sv_budget_blocks(32768, 4096, 0.1, 64) == 109
+
+
+def test_argument_validation_without_device(svb):
+    g = svb.make_geom(1, 8, 2, 128, 64, 64, 4)
+    lib = svb._lib
+    null_kv = svb.sv_kv(None, None, None, None, 1)
+    assert lib.sv_block_reps(ctypes.byref(g), ctypes.byref(null_kv), 0, -1, None, None) == 1      # SV_ERR_NULL
+    bad = svb.make_geom(1, 8, 3, 128, 64, 64, 4)
+    assert lib.sv_block_reps(ctypes.byref(bad), ctypes.byref(null_kv), 0, -1, None, None) == 2    # SV_ERR_SHAPE
+    for kw, code in ((dict(head_dim=64), 6), (dict(block_size=32), 6), (dict(n_draft=33), 6), (dict(n_draft=0), 2)):
+        args = dict(n_seq=1, n_q_heads=8, n_kv_heads=2, head_dim=128, block_size=64, max_blocks=64, n_draft=4)
+        args.update(kw)
+        gg = svb.make_geom(**args)
+        assert lib.sv_block_reps(ctypes.byref(gg), ctypes.byref(null_kv), 0, -1, None, None) == code
+    big = svb.make_geom(1, 64, 2, 128, 64, 64, 8)        # 32 * 8 = 256 query rows per KV head
+    assert lib.sv_block_reps(ctypes.byref(big), ctypes.byref(null_kv), 0, -1, None, None) == 6
+    # misaligned pool pointer
+    kv = svb.sv_kv(0x1008, 0x2000, 0x3000, 0x4000, 4)
+    assert lib.sv_block_reps(ctypes.byref(g), ctypes.byref(kv), 0, -1, 0x5000, None) == 3        # SV_ERR_ALIGN
+    # select: outputs missing, forced blocks above max_sel, reuse without a previous list
+    assert lib.sv_select_blocks(ctypes.byref(g), 0x1000, 0x2000, 0x3000, 0x4000, 1, 1, 0, None, None, None, None,
+                                16, None, None) == 1
+    assert lib.sv_select_blocks(ctypes.byref(g), 0x1000, 0x2000, 0x3000, 0x4000, 9, 9, 0, None, None, 0x5000,
+                                0x6000, 16, None, None) == 4
+    assert lib.sv_select_blocks(ctypes.byref(g), None, None, None, None, 1, 1, 1, None, None, 0x5000, 0x6000, 16,
+                                None, None) == 1
+    # attention: missing output
+    kv = svb.sv_kv(0x1000, 0x2000, 0x3000, 0x4000, 4)
+    assert lib.sv_verify_attn(ctypes.byref(g), 0x1000, ctypes.byref(kv), 0x1000, 0x1000, None, None, None, 0, 0.0,
+                              None, None, None, 0, None, None) == 1
+
+
+def test_workspace_size_formula(svb):
+    g = svb.make_geom(1, 32, 8, 128, 64, 512, 8)
+    splits = svb.sv_verify_attn_splits(g, 64)
+    assert 1 <= splits <= 64
+    assert svb.sv_workspace_bytes(g, 64) == 1 * 8 * splits * 32 * 130 * 4 + 256
+    assert svb.sv_workspace_bytes(svb.make_geom(1, 8, 3, 128, 64, 64, 4), 16) == 0

@@ -179,7 +179,7 @@ def test_generator_plants_and_repairs_gap():
     geom = si.make_geometry(si.WORKLOADS["cfg0"])
     c = si.make_layer(geom)
     idx, cnt, sc = oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
-    assert c["min_gap"] >= c["delta"] > 0
+    assert c["min_gap_ratio"] >= 1.0 and c["delta"] > 0
     for (s, h), planted in c["planted"].items():
         sel = set(idx[s, h, :cnt[s, h]].tolist())
         assert set(planted.tolist()) <= sel and {0, 63} <= sel
