@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse verification attention path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Workload: the Llama-3.1-8B-shaped attention stack (32 layers, 32 query / 8 KV heads, head_dim 128,
+bf16, batch 1, 32768 cached tokens in 64-token blocks, 64 kept blocks, 8 draft tokens as a chain),
+seeded synthetic tensors from sv_inputs.  One step = one pass of the whole hot path over all 32
+layers: refresh of the tail block's representative, block selection (every layer), sparse verification
+attention (split-KV + merge).  The step is captured in a CUDA graph; K replays are timed with CUDA
+events between barriers.  Every layer has its own 128 MiB KV pool and a step gathers 512 MiB from a
+4 GiB working set, so no iteration finds its K/V in the 126 MB L2.
+
+Prints ONE JSON line (rank 0).  `value` is microseconds per layer (whole job: N GPUs run N independent
+replicas, value = step time / (layers * N)); lower is better.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import sv_inputs as si  # noqa: E402
+
+WORKLOAD = "cfg1"
+METRIC = "sparse_verify_attn_us_per_layer"
+UNIT = "us/layer"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def generate_layers(w, geom, n_layers, sharp=False):
+    """Host tensors of every layer (thread pool: numpy's generators release the GIL)."""
+    workers = max(1, min(n_layers, (os.cpu_count() or 8)))
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        return list(ex.map(lambda l: si.make_layer(geom, layer=l, sharp=sharp), range(n_layers)))
+
+
+# ----------------------------------------------------------------------------- reference arm (CPU oracle)
+
+def oracle_layer_seconds(case, n_kv_heads_sample):
+    """Oracle time for block selection of a layer plus sparse attention of the query heads of the
+    first `n_kv_heads_sample` KV heads, scaled to a full layer."""
+    import oracle
+    w = case["workload"]
+    G = w.group
+    t0 = time.perf_counter()
+    idx, cnt, _ = oracle.select_blocks(case["q"], case["k_pool"], case["block_table"], case["seq_lens"], case["budget"],
+                                       w.n_sink, w.n_local, case["max_sel"])
+    t_sel = time.perf_counter() - t0
+    samples = [(s, i, hq) for s in range(w.n_seq) for i in range(w.n_draft) for hq in range(n_kv_heads_sample * G)]
+    t0 = time.perf_counter()
+    oracle.verify_attn(case["q"], case["k_pool"], case["v_pool"], case["block_table"], case["seq_lens"], case["draft_k"],
+                       case["draft_v"], case["parent"], idx, cnt, samples=samples)
+    t_attn = (time.perf_counter() - t0) * (w.n_kv_heads / n_kv_heads_sample)
+    return t_sel + t_attn
+
+
+def run_reference(args):
+    """--impl reference: the fp64 CPU oracle, as it stands, on the host cores, same config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = si.WORKLOADS[WORKLOAD]
+    geom = si.make_geometry(w)
+    case = si.make_layer(geom, layer=0)
+    oracle_layer_seconds(case, 1)   # build + page in
+    t_full = oracle_layer_seconds(case, w.n_kv_heads)
+    # size the per-step sample so that the whole run stays within ~2 minutes
+    total = args.steps + args.warmup
+    nh = w.n_kv_heads
+    while nh > 1 and t_full * nh / w.n_kv_heads * total > 120.0:
+        nh //= 2
+    for _ in range(args.warmup):
+        oracle_layer_seconds(case, nh)
+    times = [oracle_layer_seconds(case, nh) for _ in range(args.steps)]
+    sec_per_layer = sum(times) / len(times)
+    us = sec_per_layer * 1e6
+    sample = (f"one layer per step: block selection of the layer + sparse attention of the query heads of {nh} of "
+              f"{w.n_kv_heads} KV heads, scaled to the layer")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_per_layer * 1e3 * w.n_layers, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, geom),
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, geom):
+    return {"workload": "cfg1: 32-layer Llama-3.1-8B-shaped stack, batch 1, 32 q / 8 kv heads, head_dim 128, "
+                        "32768 cached tokens, block 64, top-64 blocks (4096 tokens), 8 draft tokens (chain), "
+                        "selection recomputed every layer",
+            "layers": w.n_layers, "context": int(geom["seq_lens"][0]), "block": w.block_size,
+            "budget_blocks": w.budget_blocks, "n_draft": w.n_draft, "n_sink": w.n_sink, "n_local": w.n_local,
+            "l2": "inputs larger than L2: every layer has its own 128 MiB K/V pool; a step gathers 512 MiB out of 4 GiB"}
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.sm_max = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if not self.nv:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                     "hw_power_brake_slowdown": 0x80, "sync_boost": 0x10, "applications_clocks_setting": 0x2}
+            for k, bit in names.items():
+                if r & bit:
+                    self.reasons.add(k)
+        except Exception:
+            pass
+
+    def __enter__(self):
+        def loop():
+            while not self._stop.is_set():
+                self.sample()
+                self._stop.wait(0.005)
+        self._thread = threading.Thread(target=loop, daemon=True)
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self.sample()
+        self._stop.set()
+        self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2512_21911_b200 as sv
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = si.WORKLOADS[WORKLOAD]
+    if args.layers:
+        w = si.shrink(w, n_layers=args.layers)
+    geom = si.make_geometry(w)
+    layers = generate_layers(w, geom, w.n_layers)
+    min_ratio = min(c["min_gap_ratio"] for c in layers)
+
+    def bf16_dev(a):
+        return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(dev)
+
+    def make_engine(anchors):
+        e = sv.SparseVerifier(n_seq=w.n_seq, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                              block_size=w.block_size, max_blocks=geom["max_blocks"], n_draft=w.n_draft,
+                              n_layers=w.n_layers, block_table=torch.from_numpy(geom["block_table"]).to(dev),
+                              seq_lens=torch.from_numpy(geom["seq_lens"]).to(dev),
+                              budget_blocks=torch.from_numpy(geom["budget"]).to(dev), max_sel=geom["max_sel"],
+                              n_sink=w.n_sink, n_local=w.n_local, anchors=anchors, device=str(dev))
+        return e
+
+    eng = make_engine([True] * w.n_layers)
+    eng_reuse = make_engine([l % 2 == 0 for l in range(w.n_layers)])   # anchors on even layers (Eq. 9)
+    pools = [(bf16_dev(c["k_pool"]), bf16_dev(c["v_pool"])) for c in layers]
+    for l, (kp, vp) in enumerate(pools):
+        eng.set_layer_kv(l, kp, vp)
+        eng_reuse.set_layer_kv(l, kp, vp)
+        eng.build_reps(l)
+    eng_reuse.reps = eng.reps
+    # per-step inputs: pinned host copies (end-to-end timing) and device-resident copies (kernel timing)
+    q_h = torch.stack([torch.from_numpy(c["q"].view(np.int16)).view(torch.bfloat16) for c in layers]).pin_memory()
+    dk_h = torch.stack([torch.from_numpy(c["draft_k"].view(np.int16)).view(torch.bfloat16) for c in layers]).pin_memory()
+    dv_h = torch.stack([torch.from_numpy(c["draft_v"].view(np.int16)).view(torch.bfloat16) for c in layers]).pin_memory()
+    q, dk, dv = q_h.to(dev), dk_h.to(dev), dv_h.to(dev)
+    out = torch.zeros_like(q)
+    out_h = torch.empty_like(q_h).pin_memory()
+    h2d = q_h.numel() * 2 + dk_h.numel() * 2 + dv_h.numel() * 2
+    d2h = out_h.numel() * 2
+
+    stream = torch.cuda.Stream(device=dev)
+
+    def capture(fn):
+        with torch.cuda.stream(stream):
+            for _ in range(2):      # first calls configure kernels / encode tensor maps: keep them out of the capture
+                fn()
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+        return g
+
+    def time_replays(g, steps, warmup, before=None, after=None, sampler=None):
+        """ms per step of `steps` replays of graph g on `stream` (device time, CUDA events)."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                if before:
+                    before()
+                g.replay()
+                if after:
+                    after()
+            barrier()
+            ctx = sampler if sampler is not None else _Null()
+            with ctx:
+                e0.record(stream)
+                for _ in range(steps):
+                    if before:
+                        before()
+                    g.replay()
+                    if after:
+                        after()
+                e1.record(stream)
+                if sampler is not None:
+                    sampler.sample()
+                stream.synchronize()
+            barrier()
+        return e0.elapsed_time(e1) / steps
+
+    class _Null:
+        def __enter__(self):
+            return self
+
+        def __exit__(self, *a):
+            return False
+
+    g_step = capture(lambda: eng.verify_step(q, dk, dv, out, refresh_tail=True))
+    if args.only_step:
+        ms = time_replays(g_step, args.steps, args.warmup)
+        if rank == 0:
+            print(json.dumps({"only_step": True, "layers": w.n_layers, "us_per_layer": ms * 1e3 / w.n_layers,
+                              "kernels_per_step": eng.kernels_per_step(refresh_tail=True)}))
+        return
+    g_reuse = capture(lambda: eng_reuse.verify_step(q, dk, dv, out, refresh_tail=True))
+    g_attn = capture(lambda: [sv.sv_verify_attn(eng.geom, q[l], eng.kv[l], dk[l], dv[l], None, eng.sel_idx, eng.sel_cnt,
+                                                out[l], workspace=eng.workspace, status_word=eng.status)
+                              for l in range(w.n_layers)])
+    g_dense = capture(lambda: eng.dense_step(q, dk, dv, out))
+
+    sampler = ClockSampler(local)
+    ms_step = time_replays(g_step, args.steps, max(args.warmup, 3), sampler=sampler)
+    side = max(10, min(args.steps, 200))
+    ms_reuse = time_replays(g_reuse, side, 3)
+    ms_attn = time_replays(g_attn, side, 3)
+    ms_dense = time_replays(g_dense, max(5, side // 4), 3)
+
+    def h2d_copy():
+        q.copy_(q_h, non_blocking=True)
+        dk.copy_(dk_h, non_blocking=True)
+        dv.copy_(dv_h, non_blocking=True)
+
+    def d2h_copy():
+        out_h.copy_(out, non_blocking=True)
+
+    ms_e2e = time_replays(g_step, side, 3, before=h2d_copy, after=d2h_copy)
+    assert int(eng.status.item()) == 0 and int(eng_reuse.status.item()) == 0, "a kernel gave up on a bounded wait"
+
+    def allmax(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e = (allmax(x) for x in (ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e))
+
+    # algorithmic bytes of one sv_verify_attn launch (K+V of the kept tokens and draft tokens, Q in, O out)
+    S, T, Hq, Hkv, D, B, N = w.n_seq, w.n_draft, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, w.budget_blocks
+    kv_tokens = sum(min(N * B, int(L)) for L in geom["seq_lens"])
+    gathered = Hkv * kv_tokens * 2 * D * 2
+    attn_bytes = Hkv * (kv_tokens + S * T) * 2 * D * 2 + 2 * S * T * Hq * D * 2
+    dense_bytes = Hkv * (int(geom["seq_lens"].sum()) + S * T) * 2 * D * 2 + 2 * S * T * Hq * D * 2
+    peak, peak_kind = measured_peaks()
+    us_attn = ms_attn * 1e3 / w.n_layers
+    us_dense = ms_dense * 1e3 / w.n_layers
+    achieved = attn_bytes / (us_attn * 1e-6) / 1e9
+    us_layer = ms_step * 1e3 / (w.n_layers * world)
+
+    line = {
+        "metric": METRIC, "value": us_layer, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, geom),
+        "clocks": sampler.summary(),
+        "e2e": {"value": ms_e2e * 1e3 / (w.n_layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h,
+                "note": "per step: Q and draft K/V of all layers copied from pinned host memory, outputs copied back; "
+                        "the KV cache is device-resident state"},
+        "gpu_launches": args.steps * eng.kernels_per_step(refresh_tail=True),
+        "kernels_per_step": eng.kernels_per_step(refresh_tail=True),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "kernel": "sv_verify_attn (split-KV attention + split merge), one launch per layer",
+                     "bytes_per_launch": attn_bytes, "us_per_launch": us_attn},
+        "kv_gathered_gbs": gathered / (us_attn * 1e-6) / 1e9,
+        "pct_of_8tbs": 100.0 * gathered / (us_attn * 1e-6) / 8e12,
+        "tokens_verified_per_s": S * T * world / (ms_step * 1e-3),
+        "reuse_even_anchors": {"us_per_layer": ms_reuse * 1e3 / w.n_layers, "kernels_per_step": eng_reuse.kernels_per_step(True)},
+        "dense_verify": {"us_per_layer": us_dense, "gbs": dense_bytes / (us_dense * 1e-6) / 1e9,
+                         "frac": dense_bytes / (us_dense * 1e-6) / 1e9 / peak, "bytes_per_launch": dense_bytes},
+        "min_score_gap_over_delta": min_ratio,
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle_layer_seconds(layers[0], 1)
+        n_layers_sample = w.n_layers
+        t0 = time.perf_counter()
+        secs = [oracle_layer_seconds(layers[l], w.n_kv_heads) for l in range(n_layers_sample)]
+        line["cpu_baseline"] = {"value": sum(secs) / len(secs) * 1e6, "unit": UNIT, "cores": oracle.num_threads(),
+                                "kind": "oracle",
+                                "sample": f"{n_layers_sample} of {w.n_layers} layers, each in full (block selection + sparse "
+                                          f"attention of all heads), {time.perf_counter() - t0:.1f} s of wall time"}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: run a shorter stack (default: all 32)")
+    ap.add_argument("--only-step", action="store_true",
+                    help="profiling aid: time only the main step graph (no reuse / dense / attention-only / e2e passes)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -103,9 +103,11 @@ SV_API size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel);
  * every sequence (block_end < 0: up to the last block; blocks past a
  * sequence's end are skipped).  The last block of a sequence is averaged over
  * the tokens it holds.  Full blocks never change, so a decoding loop only
- * needs to refresh the tail block.
+ * needs to refresh the tail block: block_begin == SV_TAIL_BLOCK recomputes
+ * just the last block of every sequence (block_end is then ignored).
  *   reps: dev fp32 [S][Hkv][NBmax][D], written for the recomputed blocks only.
  */
+#define SV_TAIL_BLOCK (-1)
 SV_API sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
                         float *reps, void *stream);
 

@@ -16,6 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsv.so")
 
 SV_OK = 0
+SV_TAIL_BLOCK = -1   # sv_block_reps(block_begin=SV_TAIL_BLOCK): refresh only each sequence's last block
 STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIGN", 4: "SV_ERR_BUDGET",
                 5: "SV_ERR_WORKSPACE", 6: "SV_ERR_UNSUPPORTED", 7: "SV_ERR_CUDA"}
 

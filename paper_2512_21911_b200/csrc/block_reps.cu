@@ -22,10 +22,10 @@ __global__ void __launch_bounds__(kThreads) block_reps_kernel(const uint4 *__res
                                                               int block_begin, int block_end)
 {
     const int s = blockIdx.z, h = blockIdx.y;
-    const int b = block_begin + blockIdx.x;
     const int L = seq_lens[s];
-    const int nb = (L + B - 1) / B;
-    if (b >= nb || (block_end >= 0 && b >= block_end)) return;
+    const int nb = min((L + B - 1) / B, NBmax);
+    const int b = block_begin < 0 ? nb - 1 : block_begin + blockIdx.x;   // block_begin < 0: the tail block
+    if (b < 0 || b >= nb || (block_begin >= 0 && block_end >= 0 && b >= block_end)) return;
     const int cnt = min(B, L - b * B);
     const int page = block_table[(size_t)s * NBmax + b];
     const uint4 *tile = k_pool + ((size_t)page * Hkv + h) * (B * 16);
@@ -73,10 +73,10 @@ extern "C" sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t
     if (st != SV_OK) return st;
     if (!reps) return SV_ERR_NULL;
     if (!svh::aligned(reps, 16)) return SV_ERR_ALIGN;
-    if (block_begin < 0) return SV_ERR_SHAPE;
+    if (block_begin < 0 && block_begin != SV_TAIL_BLOCK) return SV_ERR_SHAPE;
     const int hi = (block_end < 0 || block_end > geom->max_blocks) ? geom->max_blocks : block_end;
-    if (hi <= block_begin) return SV_OK;   // empty range: nothing to do
-    dim3 grid(hi - block_begin, geom->n_kv_heads, geom->n_seq);
+    if (block_begin >= 0 && hi <= block_begin) return SV_OK;   // empty range: nothing to do
+    dim3 grid(block_begin < 0 ? 1 : hi - block_begin, geom->n_kv_heads, geom->n_seq);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (geom->block_size == 64)
         block_reps_kernel<64><<<grid, kThreads, 0, cs>>>(static_cast<const uint4 *>(kv->k_pool), kv->block_table,

@@ -35,6 +35,8 @@ class SparseVerifier:
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.kv: List[Optional[sv.sv_kv]] = [None] * n_layers
         self._pools = [None] * n_layers   # keep the tensors alive
+        self._side = None
+        self._events = None
 
     def set_layer_kv(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
         self._pools[layer] = (k_pool, v_pool)
@@ -63,12 +65,39 @@ class SparseVerifier:
         sv.sv_verify_attn(self.geom, q, self.kv[layer], draft_k, draft_v, self.parent, None, None, out, lse=lse,
                           workspace=self.dense_workspace, status_word=self.status)
 
-    def verify_step(self, q, draft_k, draft_v, out) -> None:
-        """One verification step of the whole stack.  q/out: [layers][S][T][Hq][D]; draft_k/v: [layers][S][T][Hkv][D]."""
-        for l in range(self.n_layers):
-            self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l])
+    def verify_step(self, q, draft_k, draft_v, out, refresh_tail: bool = False) -> None:
+        """One verification step of the whole stack.  q/out: [layers][S][T][Hq][D]; draft_k/v: [layers][S][T][Hkv][D].
 
-    def kernels_per_step(self) -> int:
-        """Kernel launches of one verify_step (select per anchor layer; attention (+ merge) per layer)."""
-        splits = sv.sv_verify_attn_splits(self.geom, self.max_sel)
-        return sum(self.anchors) + self.n_layers * (2 if splits > 1 else 1)
+        refresh_tail: first recompute the representative of every sequence's last block in the anchor
+        layers (the block that grew when the previous step's accepted tokens were appended).  These
+        small launches do not depend on the layer chain, so they go to a side stream and each anchor
+        layer waits only for its own."""
+        cur = torch.cuda.current_stream()
+        if refresh_tail:
+            if self._side is None:
+                self._side = torch.cuda.Stream()
+                self._events = [torch.cuda.Event() for _ in range(self.n_layers)]
+            self._side.wait_stream(cur)
+            with torch.cuda.stream(self._side):
+                for l in range(self.n_layers):
+                    if self.anchors[l]:
+                        sv.sv_block_reps(self.geom, self.kv[l], self.reps[l], sv.SV_TAIL_BLOCK)
+                        self._events[l].record(self._side)
+        for l in range(self.n_layers):
+            if refresh_tail and self.anchors[l]:
+                cur.wait_event(self._events[l])
+            self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l])
+        if refresh_tail:
+            cur.wait_stream(self._side)
+
+    def dense_step(self, q, draft_k, draft_v, out) -> None:
+        for l in range(self.n_layers):
+            self.dense_layer(l, q[l], draft_k[l], draft_v[l], out[l])
+
+    def kernels_per_step(self, refresh_tail: bool = False, dense: bool = False) -> int:
+        """Kernel launches of one step: tail refresh and select per anchor layer; attention (+ merge) per layer."""
+        splits = sv.sv_verify_attn_splits(self.geom, self.geom.max_blocks if dense else self.max_sel)
+        attn = self.n_layers * (2 if splits > 1 else 1)
+        if dense:
+            return attn
+        return sum(self.anchors) * (2 if refresh_tail else 1) + attn

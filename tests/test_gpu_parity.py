@@ -216,6 +216,14 @@ def test_block_reps_range_update(sv):
     torch.cuda.synchronize()
     assert torch.equal(d.reps[:, :, 3:6], full[:, :, 3:6])
     assert (d.reps[:, :, :3] == 123.0).all() and (d.reps[:, :, 6:] == 123.0).all()
+    # tail-only refresh: exactly the last block of every (ragged) sequence
+    d.reps.fill_(123.0)
+    sv.sv_block_reps(d.geom, d.kv, d.reps, sv.SV_TAIL_BLOCK)
+    torch.cuda.synchronize()
+    for s in range(3):
+        t = int(c["n_blocks"][s]) - 1
+        assert torch.equal(d.reps[s, :, t], full[s, :, t])
+        assert (d.reps[s, :, :t] == 123.0).all() and (d.reps[s, :, t + 1:] == 123.0).all()
 
 
 def test_empty_prefix_and_empty_selection(sv):
