@@ -1,0 +1,32 @@
+// Shared between the two attention kernels (mma.sync path and tcgen05 path): launch parameters.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace svk {
+
+struct AttnParams {
+    const __nv_bfloat16 *q;
+    const __nv_bfloat16 *draft_k;
+    const __nv_bfloat16 *draft_v;
+    const int32_t *parent;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    const int32_t *sel_idx;
+    const int32_t *sel_cnt;
+    __nv_bfloat16 *out;
+    float *lse;
+    float *ws_o;    // [S][Hkv][splits][rows][128]
+    float *ws_ml;   // [S][Hkv][splits][rows][2]
+    int32_t *status;
+    int T, Hq, Hkv, G, B, NBmax, max_sel, splits;
+    float scale_log2;
+};
+
+// tcgen05 / TMEM attention kernel (verify_attn_tc.cu): rows = G*T <= 128 packed as one M=128 tile.
+cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
+                           cudaStream_t stream);
+
+}  // namespace svk

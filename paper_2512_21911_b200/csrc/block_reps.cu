@@ -8,6 +8,7 @@
 #include <cuda_bf16.h>
 
 #include "sv_host.h"
+#include "sv_ptx.cuh"
 
 namespace {
 
@@ -22,6 +23,8 @@ __global__ void __launch_bounds__(kThreads) block_reps_kernel(const uint4 *__res
                                                               int block_begin, int block_end)
 {
     const int s = blockIdx.z, h = blockIdx.y;
+    svk::grid_dependency_wait();      // the keys may come from the kernel just before (a cache append)
+    svk::grid_launch_dependents();
     const int L = seq_lens[s];
     const int nb = min((L + B - 1) / B, NBmax);
     const int b = block_begin < 0 ? nb - 1 : block_begin + blockIdx.x;   // block_begin < 0: the tail block
@@ -77,14 +80,20 @@ extern "C" sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t
     const int hi = (block_end < 0 || block_end > geom->max_blocks) ? geom->max_blocks : block_end;
     if (block_begin >= 0 && hi <= block_begin) return SV_OK;   // empty range: nothing to do
     dim3 grid(block_begin < 0 ? 1 : hi - block_begin, geom->n_kv_heads, geom->n_seq);
-    cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (geom->block_size == 64)
-        block_reps_kernel<64><<<grid, kThreads, 0, cs>>>(static_cast<const uint4 *>(kv->k_pool), kv->block_table,
-                                                         kv->seq_lens, reps, geom->n_kv_heads, geom->max_blocks,
-                                                         block_begin, block_end);
-    else
-        block_reps_kernel<128><<<grid, kThreads, 0, cs>>>(static_cast<const uint4 *>(kv->k_pool), kv->block_table,
-                                                          kv->seq_lens, reps, geom->n_kv_heads, geom->max_blocks,
-                                                          block_begin, block_end);
-    return svh::launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    svh::pdl_attribute(attr);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint4 *pool = static_cast<const uint4 *>(kv->k_pool);
+    const cudaError_t e =
+        geom->block_size == 64
+            ? cudaLaunchKernelEx(&cfg, block_reps_kernel<64>, pool, kv->block_table, kv->seq_lens, reps,
+                                 (int)geom->n_kv_heads, (int)geom->max_blocks, (int)block_begin, (int)block_end)
+            : cudaLaunchKernelEx(&cfg, block_reps_kernel<128>, pool, kv->block_table, kv->seq_lens, reps,
+                                 (int)geom->n_kv_heads, (int)geom->max_blocks, (int)block_begin, (int)block_end);
+    return e == cudaSuccess ? svh::launch_status() : SV_ERR_CUDA;
 }

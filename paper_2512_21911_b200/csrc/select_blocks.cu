@@ -13,6 +13,7 @@
 #include <cuda_bf16.h>
 
 #include "sv_host.h"
+#include "sv_ptx.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -62,6 +63,29 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     const bool keep_all = N >= nb;
     if (keep_all) N = nb;
 
+    // While the kernel that precedes this one in the stream drains, pull this warp's first batch of
+    // representative rows towards L2 (a prefetch consumes no data, so it is safe even if that kernel
+    // is still writing them); all real loads come after the dependency wait.
+    const bool need_scores = !keep_all || p.out_scores;
+    const int b0 = rank * p.chunk;
+    const int b1 = min(b0 + p.chunk, nb);
+    const float4 *rbase = reinterpret_cast<const float4 *>(p.reps + ((size_t)s * p.Hkv + h) * p.NBmax * 128);
+    float4 r[kRowsPerIter];
+    int b = b0 + warp * kRowsPerIter;
+    auto load_rows = [&](int bb) {
+#pragma unroll
+        for (int i = 0; i < kRowsPerIter; ++i)
+            r[i] = (bb + i < b1) ? __ldg(rbase + (size_t)(bb + i) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    if (need_scores) {
+#pragma unroll
+        for (int i = 0; i < kRowsPerIter; ++i)
+            if (b + i < b1) svk::prefetch_l2(rbase + (size_t)(b + i) * 32 + lane);
+    }
+    svk::grid_dependency_wait();
+    svk::grid_launch_dependents();
+    if (need_scores && b < b1) load_rows(b);
+
     // retrieval query: mean of the first draft token's query over the GQA group
     const int G = p.Hq / p.Hkv;
     if (tid < 128) {
@@ -72,16 +96,9 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     }
     __syncthreads();
 
-    if (!keep_all || p.out_scores) {
+    if (need_scores) {
         const float4 qv = reinterpret_cast<const float4 *>(qbar)[lane];
-        const int b0 = rank * p.chunk;
-        const int b1 = min(b0 + p.chunk, nb);
-        const float4 *rbase = reinterpret_cast<const float4 *>(p.reps + ((size_t)s * p.Hkv + h) * p.NBmax * 128);
-        for (int b = b0 + warp * kRowsPerIter; b < b1; b += kWarps * kRowsPerIter) {
-            float4 r[kRowsPerIter];
-#pragma unroll
-            for (int i = 0; i < kRowsPerIter; ++i)
-                r[i] = (b + i < b1) ? __ldg(rbase + (size_t)(b + i) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (; b < b1; b += kWarps * kRowsPerIter) {
 #pragma unroll
             for (int i = 0; i < kRowsPerIter; ++i) {
                 float d = r[i].x * qv.x + r[i].y * qv.y + r[i].z * qv.z + r[i].w * qv.w;
@@ -94,6 +111,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                     if (p.out_scores) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = d;
                 }
             }
+            if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter);
         }
     }
     cluster.sync();
@@ -256,13 +274,14 @@ extern "C" sv_status sv_select_blocks(const sv_geom *geom, const void *q, const 
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = cs;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CL;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    svh::pdl_attribute(attr + 1);
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, select_kernel, p) != cudaSuccess) return SV_ERR_CUDA;
     return svh::launch_status();
 }

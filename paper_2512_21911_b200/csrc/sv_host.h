@@ -38,6 +38,15 @@ inline sv_status check_kv(const sv_geom *g, const sv_kv *kv, bool need_v)
     return SV_OK;
 }
 
+// Launch attribute for programmatic dependent launch: the kernel may be scheduled while its
+// predecessor in the stream drains; every kernel of the library executes griddepcontrol.wait before it
+// reads anything the predecessor wrote.
+inline void pdl_attribute(cudaLaunchAttribute *attr)
+{
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+}
+
 inline sv_status launch_status()
 {
     return cudaGetLastError() == cudaSuccess ? SV_OK : SV_ERR_CUDA;

@@ -23,11 +23,33 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <mutex>
 #include <unordered_map>
 
+#include "attn_common.cuh"
 #include "sv_host.h"
 #include "sv_ptx.cuh"
+
+#ifdef SV_TRACE
+// Development aid (never compiled into the library): per-CTA cycle stamps of the attention kernel.
+__device__ long long g_sv_trace[256 * 16];
+extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer()
+{
+    long long *p = nullptr;
+    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace);
+    return p;
+}
+#define SV_STAMP(slot)                                                                      \
+    do {                                                                                    \
+        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);    \
+        if (cta_ < 256) g_sv_trace[cta_ * 16 + (slot)] = clock64();                         \
+    } while (0)
+#else
+#define SV_STAMP(slot) \
+    do {               \
+    } while (0)
+#endif
 
 namespace {
 
@@ -43,169 +65,150 @@ constexpr int kDraftBytes = 4 * kDraftRows * 128;
 constexpr int kSmemLimit = 232448;                 // 227 KB per CTA
 constexpr int kMiscBytes = 1024;
 
-struct AttnParams {
-    const __nv_bfloat16 *q;
-    const __nv_bfloat16 *draft_k;
-    const __nv_bfloat16 *draft_v;
-    const int32_t *parent;
-    const int32_t *block_table;
-    const int32_t *seq_lens;
-    const int32_t *sel_idx;
-    const int32_t *sel_cnt;
-    __nv_bfloat16 *out;
-    float *lse;
-    float *ws_o;    // [S][Hkv][splits][rows][128]
-    float *ws_ml;   // [S][Hkv][splits][rows][2]
-    int32_t *status;
-    int T, Hq, Hkv, G, B, NBmax, max_sel, splits;
-    float scale_log2;
-};
 
-// WM warps share a stage (each owns MT 16-row tiles); WT such warp groups work on different stages.
-// The ring length is a multiple of WT, so a stage is always consumed by the same warp group: a group
-// then never waits on an mbarrier phase more than one ahead of the one it last saw complete (the
-// parity wait cannot tell phase n from phase n-2).
-template <int WM, int MT, int WT>
+// Warp layout: WM x KS consumer warps.  Warp (wm, ks) owns MT 16-row tiles of the query rows and the
+// keys [ks*64/KS, (ks+1)*64/KS) of every 64-key stage, so all warps work on a stage as soon as it lands
+// and every warp consumes every stage in order.
+template <int WM, int MT, int KS>
 struct Cfg {
     static constexpr int kRowsPad = WM * MT * 16;
-    static constexpr int kWT = WT;
-    static constexpr int kConsumerWarps = WM * WT;
+    static constexpr int kKeysPerWarp = kUnit / KS;
+    static constexpr int kConsumerWarps = WM * KS;
     static constexpr int kConsumerThreads = kConsumerWarps * 32;
     static constexpr int kQBytes = kRowsPad * 256;
     static constexpr int kMaxStages = (kSmemLimit - 1024 - kQBytes - kDraftBytes - kMiscBytes) / kStageBytes;
-    static constexpr int kStages = kMaxStages / WT * WT;
-    static_assert(kConsumerWarps <= kMathWarps, "too many consumer warps");
+    static constexpr int kStages = kMaxStages > 6 ? 6 : kMaxStages;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kQBytes + kDraftBytes + kMiscBytes;
+    static_assert(kConsumerWarps <= kMathWarps, "too many consumer warps");
     static_assert(kStages >= 3, "pipeline too shallow");
-    // the cross-group merge at the end reuses the ring and, behind it, the Q tile
-    static_assert(kWT * kRowsPad * (128 + 2) * 4 <= kStages * kStageBytes + kQBytes, "merge area does not fit");
+    static_assert(kKeysPerWarp == 16 || kKeysPerWarp == 32, "a warp takes 16 or 32 keys of a stage");
+    // the cross-warp merge at the end reuses the ring and, behind it, the Q tile
+    static_assert(KS * kRowsPad * (128 + 2) * 4 <= kStages * kStageBytes + kQBytes, "merge area does not fit");
 };
 
-// One 64-key (or 32-key draft) unit: S = Q K^T, masked online softmax, O += P V.
-template <int MT, int NKEYS, bool DRAFT>
-__device__ __forceinline__ void process_unit(uint32_t kbase, uint32_t vbase, uint32_t qbase, uint32_t q_half_stride,
+// NK keys (16 or 32) starting at key0 of a tile: S = Q K^T, masked online softmax, O += P V.
+// HALF = bytes between the dim 0-63 and dim 64-127 halves of the tile (rows * 128).
+template <int MT, int NK, uint32_t HALF, bool DRAFT>
+__device__ __forceinline__ void process_keys(uint32_t kbase, uint32_t vbase, uint32_t qbase, uint32_t q_half_stride,
                                              int row_base, const uint32_t (&qf)[8][4], float (&o)[MT][16][4],
-                                             float (&m)[MT][2], float (&l)[MT][2], float scale_log2, int nvalid,
-                                             const uint32_t (&vis)[MT][2], int lane)
+                                             float (&m)[MT][2], float (&l)[MT][2], float scale_log2, int key0,
+                                             int nvalid, const uint32_t (&vis)[MT][2], int lane)
 {
-    constexpr int KCH = (MT == 1) ? NKEYS : 32;   // keys per softmax step
-    constexpr uint32_t kHalf = NKEYS * 128;       // bytes between the dim 0-63 and dim 64-127 halves
-#pragma unroll 1
-    for (int kc = 0; kc < NKEYS; kc += KCH) {
-        float sacc[MT][KCH / 8][4];
+    float sacc[MT][NK / 8][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NK / 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sacc[mt][nt][e] = 0.f;
+
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        uint32_t qa[MT][4];
+        if constexpr (MT == 1) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) qa[0][e] = qf[ks][e];
+        } else {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint32_t row = row_base + mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                const uint32_t chunk = ks * 2 + (lane >> 4);
+                ldsm_x4(qa[mt], qbase + (chunk >> 3) * q_half_stride + swz128(row, chunk & 7));
+            }
+        }
+#pragma unroll
+        for (int np = 0; np < NK / 16; ++np) {
+            const uint32_t key = key0 + np * 16 + (lane >> 4) * 8 + (lane & 7);
+            const uint32_t chunk = ks * 2 + ((lane >> 3) & 1);
+            uint32_t kb[4];
+            ldsm_x4(kb, kbase + (chunk >> 3) * HALF + swz128(key, chunk & 7));
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                mma_bf16_16816(sacc[mt][2 * np], qa[mt], kb[0], kb[1]);
+                mma_bf16_16816(sacc[mt][2 * np + 1], qa[mt], kb[2], kb[3]);
+            }
+        }
+    }
+
+    if (DRAFT || nvalid < key0 + NK) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int nt = 0; nt < KCH / 8; ++nt)
+            for (int nt = 0; nt < NK / 8; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) sacc[mt][nt][e] = 0.f;
-
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            uint32_t qa[MT][4];
-            if constexpr (MT == 1) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) qa[0][e] = qf[ks][e];
-            } else {
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const uint32_t row = row_base + mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-                    const uint32_t chunk = ks * 2 + (lane >> 4);
-                    ldsm_x4(qa[mt], qbase + (chunk >> 3) * q_half_stride + swz128(row, chunk & 7));
+                for (int e = 0; e < 4; ++e) {
+                    const int col = key0 + nt * 8 + 2 * (lane & 3) + (e & 1);
+                    bool ok = col < nvalid;
+                    if (DRAFT) ok = ok && ((vis[mt][e >> 1] >> col) & 1u);
+                    if (!ok) sacc[mt][nt][e] = -INFINITY;
                 }
+    }
+
+    uint32_t pa[MT][NK / 16][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < NK / 8; ++nt) mx = fmaxf(mx, fmaxf(sacc[mt][nt][2 * r], sacc[mt][nt][2 * r + 1]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m[mt][r], mx * scale_log2);
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            const float corr = fast_exp2(m[mt][r] - m_use);
+            m[mt][r] = m_new;
+            float lsum = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < NK / 8; ++nt) {
+                const float p0 = fast_exp2(fmaf(sacc[mt][nt][2 * r], scale_log2, -m_use));
+                const float p1 = fast_exp2(fmaf(sacc[mt][nt][2 * r + 1], scale_log2, -m_use));
+                sacc[mt][nt][2 * r] = p0;
+                sacc[mt][nt][2 * r + 1] = p1;
+                lsum += p0 + p1;
             }
-#pragma unroll
-            for (int np = 0; np < KCH / 16; ++np) {
-                const uint32_t key = kc + np * 16 + (lane >> 4) * 8 + (lane & 7);
-                const uint32_t chunk = ks * 2 + ((lane >> 3) & 1);
-                uint32_t kb[4];
-                ldsm_x4(kb, kbase + (chunk >> 3) * kHalf + swz128(key, chunk & 7));
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    mma_bf16_16816(sacc[mt][2 * np], qa[mt], kb[0], kb[1]);
-                    mma_bf16_16816(sacc[mt][2 * np + 1], qa[mt], kb[2], kb[3]);
-                }
-            }
-        }
-
-        if (DRAFT || nvalid < NKEYS) {
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                for (int nt = 0; nt < KCH / 8; ++nt)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int col = kc + nt * 8 + 2 * (lane & 3) + (e & 1);
-                        bool ok = col < nvalid;
-                        if (DRAFT) ok = ok && ((vis[mt][e >> 1] >> col) & 1u);
-                        if (!ok) sacc[mt][nt][e] = -INFINITY;
-                    }
-        }
-
-        uint32_t pa[MT][KCH / 16][4];
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                float mx = -INFINITY;
-#pragma unroll
-                for (int nt = 0; nt < KCH / 8; ++nt) mx = fmaxf(mx, fmaxf(sacc[mt][nt][2 * r], sacc[mt][nt][2 * r + 1]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m[mt][r], mx * scale_log2);
-                const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                const float corr = fast_exp2(m[mt][r] - m_use);
-                m[mt][r] = m_new;
-                float lsum = 0.f;
-#pragma unroll
-                for (int nt = 0; nt < KCH / 8; ++nt) {
-                    const float p0 = fast_exp2(fmaf(sacc[mt][nt][2 * r], scale_log2, -m_use));
-                    const float p1 = fast_exp2(fmaf(sacc[mt][nt][2 * r + 1], scale_log2, -m_use));
-                    sacc[mt][nt][2 * r] = p0;
-                    sacc[mt][nt][2 * r + 1] = p1;
-                    lsum += p0 + p1;
-                }
-                l[mt][r] = l[mt][r] * corr + lsum;
+            l[mt][r] = l[mt][r] * corr + lsum;
+            if (corr != 1.f) {   // the running maximum moved: rescale the accumulator rows of this thread
 #pragma unroll
                 for (int nt = 0; nt < 16; ++nt) {
                     o[mt][nt][2 * r] *= corr;
                     o[mt][nt][2 * r + 1] *= corr;
                 }
             }
-#pragma unroll
-            for (int kk = 0; kk < KCH / 16; ++kk) {
-                pa[mt][kk][0] = pack_bf16(sacc[mt][2 * kk][0], sacc[mt][2 * kk][1]);
-                pa[mt][kk][1] = pack_bf16(sacc[mt][2 * kk][2], sacc[mt][2 * kk][3]);
-                pa[mt][kk][2] = pack_bf16(sacc[mt][2 * kk + 1][0], sacc[mt][2 * kk + 1][1]);
-                pa[mt][kk][3] = pack_bf16(sacc[mt][2 * kk + 1][2], sacc[mt][2 * kk + 1][3]);
-            }
         }
+#pragma unroll
+        for (int kk = 0; kk < NK / 16; ++kk) {
+            pa[mt][kk][0] = pack_bf16(sacc[mt][2 * kk][0], sacc[mt][2 * kk][1]);
+            pa[mt][kk][1] = pack_bf16(sacc[mt][2 * kk][2], sacc[mt][2 * kk][3]);
+            pa[mt][kk][2] = pack_bf16(sacc[mt][2 * kk + 1][0], sacc[mt][2 * kk + 1][1]);
+            pa[mt][kk][3] = pack_bf16(sacc[mt][2 * kk + 1][2], sacc[mt][2 * kk + 1][3]);
+        }
+    }
 
 #pragma unroll
-        for (int kk = 0; kk < KCH / 16; ++kk) {
-            const uint32_t key = kc + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+    for (int kk = 0; kk < NK / 16; ++kk) {
+        const uint32_t key = key0 + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
-            for (int dp = 0; dp < 8; ++dp) {
-                const uint32_t chunk = dp * 2 + (lane >> 4);
-                uint32_t vb[4];
-                ldsm_x4_trans(vb, vbase + (chunk >> 3) * kHalf + swz128(key, chunk & 7));
+        for (int dp = 0; dp < 8; ++dp) {
+            const uint32_t chunk = dp * 2 + (lane >> 4);
+            uint32_t vb[4];
+            ldsm_x4_trans(vb, vbase + (chunk >> 3) * HALF + swz128(key, chunk & 7));
 #pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    mma_bf16_16816(o[mt][2 * dp], pa[mt][kk], vb[0], vb[1]);
-                    mma_bf16_16816(o[mt][2 * dp + 1], pa[mt][kk], vb[2], vb[3]);
-                }
+            for (int mt = 0; mt < MT; ++mt) {
+                mma_bf16_16816(o[mt][2 * dp], pa[mt][kk], vb[0], vb[1]);
+                mma_bf16_16816(o[mt][2 * dp + 1], pa[mt][kk], vb[2], vb[3]);
             }
         }
     }
 }
 
-template <int WM, int MT, int WT_>
+template <int WM, int MT, int KS>
 __global__ void __launch_bounds__(kThreads, 1)
     verify_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                        const AttnParams p)
 {
-    using C = Cfg<WM, MT, WT_>;
-    constexpr int ROWS_PAD = C::kRowsPad, WT = C::kWT, STAGES = C::kStages;
+    using C = Cfg<WM, MT, KS>;
+    constexpr int ROWS_PAD = C::kRowsPad, STAGES = C::kStages, KW = C::kKeysPerWarp;
     constexpr int kConsumerWarps = C::kConsumerWarps, kConsumerThreads = C::kConsumerThreads;
 
     extern __shared__ uint8_t smem_raw[];
@@ -223,75 +226,38 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int L = p.seq_lens[s];
-    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
-    const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-    const int j0 = (int)((long long)split * n_sel / p.splits);
-    const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
     const int upb = p.B / kUnit;
-    const int n_units = (j1 - j0) * upb;
     const bool has_draft = split == p.splits - 1;
     const int rows = p.G * p.T;
 
-    // ------------------------------------------------------------------ prologue
     if (tid == 0) {
+        SV_STAMP(0);
         for (int i = 0; i < STAGES; ++i) {
             mbar_init(full_bar + 8 * i, 1);
-            mbar_init(empty_bar + 8 * i, WM);
+            mbar_init(empty_bar + 8 * i, kConsumerWarps);
         }
         *abort_flag = 0;
         mbar_fence_init();
     }
-    if (tid < kMathThreads) {
-        // Q rows r = i*G + g  ->  q[s][i][h*G + g][:], zero padded to ROWS_PAD, stored swizzled
-        for (int idx = tid; idx < ROWS_PAD * 16; idx += kMathThreads) {
-            const int r = idx >> 4, c = idx & 15;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < rows) {
-                const int i = r / p.G, g = r - i * p.G;
-                v = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
-            }
-            *reinterpret_cast<uint4 *>(smem + (q_base - smem0) + (c >> 3) * (ROWS_PAD * 128) + swz128(r, c & 7)) = v;
-        }
-        if (has_draft) {
-            for (int idx = tid; idx < 2 * kDraftRows * 16; idx += kMathThreads) {
-                const int which = idx / (kDraftRows * 16);   // 0: K, 1: V
-                const int r = (idx >> 4) % kDraftRows, c = idx & 15;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (r < p.T) {
-                    const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
-                    v = __ldg(reinterpret_cast<const uint4 *>(src) + c);
-                }
-                *reinterpret_cast<uint4 *>(smem + (draft_base - smem0) + which * (2 * kDraftRows * 128) +
-                                           (c >> 3) * (kDraftRows * 128) + swz128(r, c & 7)) = v;
-            }
-            if (tid < kDraftRows) {
-                uint32_t mask = 0;
-                if (tid < p.T) {
-                    if (p.parent) {
-                        int a = tid;
-                        for (int step = 0; step < p.T && a >= 0; ++step) {
-                            mask |= 1u << a;
-                            const int nxt = p.parent[(size_t)s * p.T + a];
-                            a = nxt < a ? nxt : -1;   // parents must precede their children
-                        }
-                    } else {
-                        mask = (tid == 31) ? 0xFFFFFFFFu : ((1u << (tid + 1)) - 1u);
-                    }
-                }
-                anc[tid] = mask;
-            }
-        }
-    } else if (lane == 0) {
-        tma_prefetch_desc(&tm_k);
-        tma_prefetch_desc(&tm_v);
-    }
     __syncthreads();
+    if (tid == 0) SV_STAMP(1);
 
     if (warp >= kMathWarps) {
         // -------------------------------------------------------------- producer warpgroup
         reg_dealloc<40>();   // hand registers to the math warpgroups
         if (warp != kMathWarps) return;
+        if (lane == 0) {
+            tma_prefetch_desc(&tm_k);
+            tma_prefetch_desc(&tm_v);
+        }
+        // The block list is written by the kernel that precedes this one in the stream.
+        grid_dependency_wait();
+        if (lane == 0) SV_STAMP(2);
+        const int L = p.seq_lens[s];
+        const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+        const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
+        const int j0 = (int)((long long)split * n_sel / p.splits);
+        const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
         const uint64_t policy = policy_evict_first();
         bool dead = false;
         for (int base = j0; base < j1; base += 32) {
@@ -308,6 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int i = 0; i < n_here; ++i) {
                 const int r0 = __shfl_sync(0xffffffffu, row0, i);
                 const int t0 = __shfl_sync(0xffffffffu, tok0, i);
+                if (lane == 0 && i == 0 && base == j0) SV_STAMP(3);
                 if (lane == 0 && !dead) {
                     for (int uo = 0; uo < upb; ++uo) {
                         const int u = (base - j0 + i) * upb + uo;
@@ -329,6 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             tma_load_2d(dst + 8192, &tm_k, 64, y, fb, policy);
                             tma_load_2d(dst + 16384, &tm_v, 0, y, fb, policy);
                             tma_load_2d(dst + 24576, &tm_v, 64, y, fb, policy);
+                            if (u == 0) SV_STAMP(4);
                         } else {
                             mbar_arrive(fb);
                         }
@@ -339,11 +307,57 @@ __global__ void __launch_bounds__(kThreads, 1)
         return;
     }
 
-    // ------------------------------------------------------------------ consumer warps
+    // ------------------------------------------------------------------ math warpgroups
     reg_alloc<232>();
+    grid_dependency_wait();
+    grid_launch_dependents();   // the next kernel may be scheduled; it waits for this grid before reading
+    // Stage Q (and, in the last split, the draft tokens' K/V) while the producer chases the block list.
+    // Q rows r = i*G + g  ->  q[s][i][h*G + g][:], zero padded to ROWS_PAD, stored swizzled
+    for (int idx = tid; idx < ROWS_PAD * 16; idx += kMathThreads) {
+        const int r = idx >> 4, c = idx & 15;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (r < rows) {
+            const int i = r / p.G, g = r - i * p.G;
+            v = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
+        }
+        *reinterpret_cast<uint4 *>(smem + (q_base - smem0) + (c >> 3) * (ROWS_PAD * 128) + swz128(r, c & 7)) = v;
+    }
+    if (has_draft) {
+        for (int idx = tid; idx < 2 * kDraftRows * 16; idx += kMathThreads) {
+            const int which = idx / (kDraftRows * 16);   // 0: K, 1: V
+            const int r = (idx >> 4) % kDraftRows, c = idx & 15;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (r < p.T) {
+                const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
+                v = __ldg(reinterpret_cast<const uint4 *>(src) + c);
+            }
+            *reinterpret_cast<uint4 *>(smem + (draft_base - smem0) + which * (2 * kDraftRows * 128) +
+                                       (c >> 3) * (kDraftRows * 128) + swz128(r, c & 7)) = v;
+        }
+        if (tid < kDraftRows) {
+            uint32_t mask = 0;
+            if (tid < p.T) {
+                if (p.parent) {
+                    int a = tid;
+                    for (int step = 0; step < p.T && a >= 0; ++step) {
+                        mask |= 1u << a;
+                        const int nxt = p.parent[(size_t)s * p.T + a];
+                        a = nxt < a ? nxt : -1;   // parents must precede their children
+                    }
+                } else {
+                    mask = (tid == 31) ? 0xFFFFFFFFu : ((1u << (tid + 1)) - 1u);
+                }
+            }
+            anc[tid] = mask;
+        }
+    }
+    named_bar_sync(2, kMathThreads);
+    if (tid == 0) SV_STAMP(5);
     if (warp >= kConsumerWarps) return;   // math warps this shape does not use
-    const int wm = warp % WM, grp = warp / WM;
+
+    const int wm = warp % WM, kq = warp / WM;
     const int row_base = wm * MT * 16;
+    const int key0 = kq * KW;
     uint32_t qf[8][4];
     if constexpr (MT == 1) {
 #pragma unroll
@@ -369,35 +383,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     }
 
-    bool dead = false;
-    for (int u = grp; u < n_units; u += WT) {
-        const int stage = u % STAGES, it = u / STAGES;
-        if (!dead && (*abort_flag || !mbar_wait_bounded(full_bar + 8 * stage, it & 1))) {
-            dead = true;
-            *abort_flag = 1;
-            if (p.status && lane == 0) atomicOr(p.status, 2);
-        }
-        if (dead) continue;
-        const int nvalid = min(meta[stage], kUnit);
-        if (nvalid > 0) {
-            const uint32_t kb = stage_base + stage * kStageBytes, vb = kb + 16384;
-            if (nvalid < kUnit) {
-                // zero the value rows past the end of the sequence (0 * junk must stay 0)
-                for (int idx = lane; idx < (kUnit - nvalid) * 16; idx += 32) {
-                    const int r = nvalid + (idx >> 4), c = idx & 15;
-                    *reinterpret_cast<uint4 *>(smem + (vb - smem0) + (c >> 3) * 8192 + swz128(r, c & 7)) =
-                        make_uint4(0u, 0u, 0u, 0u);
-                }
-                fence_proxy_async();   // order these generic writes before the next TMA fill of the stage
-                __syncwarp();
-            }
-            process_unit<MT, kUnit, false>(kb, vb, q_base, ROWS_PAD * 128, row_base, qf, o, m, l, p.scale_log2, nvalid,
-                                           vis, lane);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
-    }
-    if (has_draft && grp == n_units % WT) {
+    // the draft tokens first: their tile is already in shared memory (warps kq == 0 take all 32 keys)
+    if (has_draft && kq == 0) {
         const uint32_t all = (p.T == 32) ? 0xFFFFFFFFu : ((1u << p.T) - 1u);
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -406,11 +393,50 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int row = row_base + mt * 16 + (lane >> 2) + 8 * r;
                 vis[mt][r] = row < rows ? anc[row / p.G] : all;
             }
-        process_unit<MT, kDraftRows, true>(draft_base, draft_base + 2 * kDraftRows * 128, q_base, ROWS_PAD * 128,
-                                           row_base, qf, o, m, l, p.scale_log2, p.T, vis, lane);
+        process_keys<MT, kDraftRows, kDraftRows * 128, true>(draft_base, draft_base + 2 * kDraftRows * 128, q_base,
+                                                             ROWS_PAD * 128, row_base, qf, o, m, l, p.scale_log2, 0,
+                                                             p.T, vis, lane);
     }
 
-    // ------------------------------------------------------------------ merge the warp groups
+    if (tid == 0) SV_STAMP(6);
+    const int L = p.seq_lens[s];
+    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+    const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
+    const int j0 = (int)((long long)split * n_sel / p.splits);
+    const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+    const int n_units = (j1 - j0) * upb;
+    bool dead = false;
+    for (int u = 0; u < n_units; ++u) {
+        const int stage = u % STAGES, it = u / STAGES;
+        if (!dead && (*abort_flag || !mbar_wait_bounded(full_bar + 8 * stage, it & 1))) {
+            dead = true;
+            *abort_flag = 1;
+            if (p.status && lane == 0) atomicOr(p.status, 2);
+        }
+        if (dead) continue;
+        if (tid == 0 && u == 0) SV_STAMP(7);
+        if (tid == 0 && u == n_units - 1) SV_STAMP(8);
+        const int nvalid = min(meta[stage], kUnit);
+        if (nvalid > key0) {
+            const uint32_t kb = stage_base + stage * kStageBytes, vb = kb + 16384;
+            if (nvalid < key0 + KW) {
+                // zero this warp's value rows past the end of the sequence (0 * junk must stay 0)
+                for (int idx = lane; idx < (key0 + KW - nvalid) * 16; idx += 32) {
+                    const int r = nvalid + (idx >> 4), c = idx & 15;
+                    *reinterpret_cast<uint4 *>(smem + (vb - smem0) + (c >> 3) * 8192 + swz128(r, c & 7)) =
+                        make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_proxy_async();   // order these generic writes before the next TMA fill of the stage
+                __syncwarp();
+            }
+            process_keys<MT, KW, kUnit * 128, false>(kb, vb, q_base, ROWS_PAD * 128, row_base, qf, o, m, l, p.scale_log2,
+                                                     key0, nvalid, vis, lane);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
+    }
+
+    // ------------------------------------------------------------------ merge the key splits of the CTA
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -418,22 +444,23 @@ __global__ void __launch_bounds__(kThreads, 1)
             l[mt][r] += __shfl_xor_sync(0xffffffffu, l[mt][r], 1);
             l[mt][r] += __shfl_xor_sync(0xffffffffu, l[mt][r], 2);
         }
+    if (tid == 0) SV_STAMP(9);
     named_bar_sync(1, kConsumerThreads);   // every stage has been consumed: the ring is free
-    float *part_o = reinterpret_cast<float *>(smem);                 // [WT][ROWS_PAD][128]
-    float *part_m = part_o + WT * ROWS_PAD * 128;                    // [WT][ROWS_PAD]
-    float *part_l = part_m + WT * ROWS_PAD;
+    float *part_o = reinterpret_cast<float *>(smem);                 // [KS][ROWS_PAD][128]
+    float *part_m = part_o + KS * ROWS_PAD * 128;                    // [KS][ROWS_PAD]
+    float *part_l = part_m + KS * ROWS_PAD;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const int row = row_base + mt * 16 + (lane >> 2) + 8 * r;
-            float *dst = part_o + ((size_t)grp * ROWS_PAD + row) * 128 + 2 * (lane & 3);
+            float *dst = part_o + ((size_t)kq * ROWS_PAD + row) * 128 + 2 * (lane & 3);
 #pragma unroll
             for (int nt = 0; nt < 16; ++nt)
                 *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(o[mt][nt][2 * r], o[mt][nt][2 * r + 1]);
             if ((lane & 3) == 0) {
-                part_m[grp * ROWS_PAD + row] = m[mt][r];
-                part_l[grp * ROWS_PAD + row] = l[mt][r];
+                part_m[kq * ROWS_PAD + row] = m[mt][r];
+                part_l[kq * ROWS_PAD + row] = l[mt][r];
             }
         }
     named_bar_sync(1, kConsumerThreads);
@@ -443,12 +470,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int row = idx >> 5, c4 = idx & 31;
         float M = -INFINITY;
 #pragma unroll
-        for (int g = 0; g < WT; ++g) M = fmaxf(M, part_m[g * ROWS_PAD + row]);
+        for (int g = 0; g < KS; ++g) M = fmaxf(M, part_m[g * ROWS_PAD + row]);
         const float M_use = (M == -INFINITY) ? 0.f : M;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float lsum = 0.f;
 #pragma unroll
-        for (int g = 0; g < WT; ++g) {
+        for (int g = 0; g < KS; ++g) {
             const float w = fast_exp2(part_m[g * ROWS_PAD + row] - M_use);
             const float4 v = *reinterpret_cast<const float4 *>(part_o + ((size_t)g * ROWS_PAD + row) * 128 + c4 * 4);
             acc.x += w * v.x, acc.y += w * v.y, acc.z += w * v.z, acc.w += w * v.w;
@@ -469,30 +496,50 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (c4 == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
         }
     }
+    if (tid == 0) SV_STAMP(10);
 }
 
 // Combine the per-split partials: o = sum_j 2^(m_j - m) o_j / sum_j 2^(m_j - m) l_j.
+// One thread per (row, 4 output dims).  The partials sit in L2; all loads of up to 16 splits are
+// issued before the first use so that the kernel costs one memory round trip, not one per split.
 __global__ void __launch_bounds__(256) merge_splits_kernel(const AttnParams p)
 {
+    constexpr int U = 16;
     const int h = blockIdx.y, s = blockIdx.z;
     const int rows = p.G * p.T;
     const int idx = blockIdx.x * 256 + threadIdx.x;
+    grid_dependency_wait();     // the partials come from the attention kernel just before
+    grid_launch_dependents();
     if (idx >= rows * 32) return;
     const int row = idx >> 5, c4 = idx & 31;
     const size_t sh = (size_t)s * p.Hkv + h;
     const float2 *ml = reinterpret_cast<const float2 *>(p.ws_ml) + sh * p.splits * rows + row;
     const float4 *po = reinterpret_cast<const float4 *>(p.ws_o) + (sh * p.splits * rows + row) * 32 + c4;
-    float M = -INFINITY;
-    for (int j = 0; j < p.splits; ++j) M = fmaxf(M, ml[(size_t)j * rows].x);
-    const float M_use = (M == -INFINITY) ? 0.f : M;
+    float M = -INFINITY, lsum = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float lsum = 0.f;
-    for (int j = 0; j < p.splits; ++j) {
-        const float2 mlj = ml[(size_t)j * rows];
-        const float w = fast_exp2(mlj.x - M_use);
-        const float4 v = po[(size_t)j * rows * 32];
-        acc.x += w * v.x, acc.y += w * v.y, acc.z += w * v.z, acc.w += w * v.w;
-        lsum += w * mlj.y;
+    for (int j0 = 0; j0 < p.splits; j0 += U) {
+        float2 mlv[U];
+        float4 ov[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool in = j0 + u < p.splits;
+            mlv[u] = in ? ml[(size_t)(j0 + u) * rows] : make_float2(-INFINITY, 0.f);
+            ov[u] = in ? po[(size_t)(j0 + u) * rows * 32] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float Mb = M;
+#pragma unroll
+        for (int u = 0; u < U; ++u) Mb = fmaxf(Mb, mlv[u].x);
+        const float M_use = (Mb == -INFINITY) ? 0.f : Mb;
+        const float c = fast_exp2(M - M_use);   // rescale what earlier batches accumulated
+        acc.x *= c, acc.y *= c, acc.z *= c, acc.w *= c;
+        lsum *= c;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const float w = fast_exp2(mlv[u].x - M_use);
+            acc.x += w * ov[u].x, acc.y += w * ov[u].y, acc.z += w * ov[u].z, acc.w += w * ov[u].w;
+            lsum += w * mlv[u].y;
+        }
+        M = Mb;
     }
     const int i = row / p.G, g = row - i * p.G;
     const size_t orow = ((size_t)s * p.T + i) * p.Hq + h * p.G + g;
@@ -582,6 +629,17 @@ int choose_splits(const sv_geom *g, int n_blocks)
     return (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
 }
 
+// The tcgen05 kernel is the product path.  Setting SV_ATTN_IMPL=mma in the environment (read once)
+// selects the older mma.sync kernel, kept for A/B comparisons of the two tensor-core paths.
+bool use_tensor_memory_path()
+{
+    static const bool tc = [] {
+        const char *v = getenv("SV_ATTN_IMPL");
+        return !(v && v[0] == 'm');
+    }();
+    return tc;
+}
+
 template <int WM, int MT, int WT>
 cudaError_t launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p, dim3 grid, cudaStream_t cs)
 {
@@ -593,8 +651,16 @@ cudaError_t launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, const Attn
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    verify_attn_kernel<WM, MT, WT><<<grid, kThreads, C::kSmemBytes, cs>>>(tk, tv, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = cs;
+    cudaLaunchAttribute attr[1];
+    svh::pdl_attribute(attr);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, verify_attn_kernel<WM, MT, WT>, tk, tv, p);
 }
 
 }  // namespace
@@ -667,19 +733,27 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     dim3 grid(splits, geom->n_kv_heads, geom->n_seq);
     cudaError_t e;
-    if (rows <= 16)
-        e = launch_attn<1, 1, 6>(tk, tv, p, grid, cs);   // 6 warps, one stage each, ring of 6
+    if (use_tensor_memory_path())
+        e = launch_attn_tc(tk, tv, p, grid, cs);          // tcgen05 + TMEM, rows padded to one M = 128 tile
+    else if (rows <= 16)
+        e = launch_attn<1, 1, 4>(tk, tv, p, grid, cs);   // 4 warps: 16 rows x 16 keys of each stage
     else if (rows <= 32)
-        e = launch_attn<2, 1, 4>(tk, tv, p, grid, cs);   // 4 groups of 2 warps, ring of 4
+        e = launch_attn<2, 1, 4>(tk, tv, p, grid, cs);   // 8 warps: 2 row tiles x 4 key quarters
     else if (rows <= 64)
-        e = launch_attn<4, 1, 2>(tk, tv, p, grid, cs);   // 2 groups of 4 warps, ring of 6
+        e = launch_attn<4, 1, 2>(tk, tv, p, grid, cs);   // 8 warps: 4 row tiles x 2 key halves
     else
-        e = launch_attn<4, 2, 2>(tk, tv, p, grid, cs);   // 2 groups of 4 warps x 32 rows, ring of 4
+        e = launch_attn<4, 2, 2>(tk, tv, p, grid, cs);   // 8 warps: 4 x 32 rows x 2 key halves
     if (e != cudaSuccess) return SV_ERR_CUDA;
-    if (splits > 1) {
-        dim3 mgrid((rows * 32 + 255) / 256, geom->n_kv_heads, geom->n_seq);
-        merge_splits_kernel<<<mgrid, 256, 0, cs>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return SV_ERR_CUDA;
+    if (splits > 1 && !getenv("SV_PROBE_SKIP_MERGE")) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((rows * 32 + 255) / 256, geom->n_kv_heads, geom->n_seq);
+        cfg.blockDim = dim3(256);
+        cfg.stream = cs;
+        cudaLaunchAttribute attr[1];
+        svh::pdl_attribute(attr);
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, merge_splits_kernel, p) != cudaSuccess) return SV_ERR_CUDA;
     }
     return SV_OK;
 }

@@ -1,0 +1,613 @@
+// Sparse verification attention on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// Same contract as the mma.sync kernel in verify_attn.cu: grid (split, KV head, sequence); a CTA owns
+// a contiguous slice of the ascending block list of its (sequence, KV head) and all G*T query rows of
+// that KV head, padded to one M = 128 tile.  Per 64-key unit (32 KB of K and V gathered by TMA):
+//
+//   S[128 x 64]  = Q[128 x 128] . K^T     8 x tcgen05.mma (M128 N64 K16), operands in shared memory
+//                                         (Q, K: K-major, 128-byte swizzle), accumulator in TMEM
+//   softmax      four threads per query row (tcgen05.ld 16x256b: the mma.sync accumulator fragment
+//                layout): mask, running max / sum in fp32 with quad shuffles, P rounded to bf16 into
+//                shared memory (K-major, 128-byte swizzle)
+//   Ou[128x128]  = P[128 x 64] . V        4 x tcgen05.mma (M128 N128 K16), V read MN-major from the
+//                                         tile exactly as TMA stored it, accumulator in TMEM
+//   O            = O * 2^(m_old - m_new) + Ou   in registers (32 dims of a row per thread)
+//
+// Warp roles (384 threads): warps 0-3 and 4-7 are two softmax warpgroups that take units alternately,
+// each with its own S / P / Ou buffers; warp 8 is the TMA producer, one thread of warp 9 issues every
+// S = Q K^T (and the warp owns the TMEM allocation), one thread of warp 10 issues every Ou = P V.  The third warpgroup gives its registers to the other
+// two (setmaxnreg).  Everything is chained with mbarriers; tcgen05.commit signals MMA completion.
+// All waits are bounded; a wait that gives up sets *status and the CTA drains and frees its TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "attn_common.cuh"
+#include "sv_ptx.cuh"
+
+#ifdef SV_TRACE
+// Development aid (never compiled into the library): cycle stamps of the first CTAs.
+__device__ long long g_sv_trace_tc[32 * 128];
+extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_tc()
+{
+    long long *p = nullptr;
+    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace_tc);
+    return p;
+}
+#define TC_STAMP(slot)                                                                     \
+    do {                                                                                   \
+        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);   \
+        if (cta_ < 32 && (slot) < 128) g_sv_trace_tc[cta_ * 128 + (slot)] = clock64();     \
+    } while (0)
+#else
+#define TC_STAMP(slot) \
+    do {               \
+    } while (0)
+#endif
+
+namespace svk {
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int kUnit = 64;                        // keys per unit
+constexpr int kTile = kUnit * 128;               // bytes of one [64 rows][64 bf16] half tile (8 KB)
+constexpr int kStageBytes = 4 * kTile;           // K lo/hi + V lo/hi
+constexpr int kStages = 4;
+constexpr int kQBytes = 2 * 128 * 128;           // Q: two halves [128 rows][64 bf16]
+constexpr int kPBytes = 128 * 128;               // P: [128 rows][64 bf16]
+constexpr int kOffQ = kStages * kStageBytes;
+constexpr int kOffP = kOffQ + kQBytes;
+constexpr int kOffDraft = kOffP + 2 * kPBytes;   // draft unit: same layout as a stage
+constexpr int kOffMisc = kOffDraft + kStageBytes;
+constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+static_assert(20 <= 32, "one lane of the producer warp per barrier");
+constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, Ou: 2 x 128 columns
+constexpr int kMergeStride = 132;                // floats per row of the cross-warpgroup merge buffer
+
+// barrier slots (8 bytes each) inside the misc area
+enum Bar {
+    kFull = 0,                  // [kStages] TMA landed
+    kEmpty = kFull + kStages,   // [kStages] PV of the unit finished reading the stage
+    kSReady = kEmpty + kStages, // [2] S of the warpgroup's unit is in TMEM
+    kSFree = kSReady + 2,       // [2] the warpgroup has read S
+    kPReady = kSFree + 2,       // [2] P is in shared memory
+    kOReady = kPReady + 2,      // [2] Ou is in TMEM
+    kOFree = kOReady + 2,       // [2] the warpgroup has read Ou
+    kStaged = kOFree + 2,       // Q (and the draft unit) are staged
+    kTmemDone = kStaged + 1,    // all warps are done with TMEM
+    kNumBars = kTmemDone + 1
+};
+
+// NH = 8-row groups per TMEM lane quadrant that hold real query rows: 1 (rows <= 32), 2 (<= 64), 4 (<= 128).
+template <int NH>
+__global__ void __launch_bounds__(kThreads, 1)
+    verify_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                          const AttnParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (smem0 - smem_u32(smem_raw));
+    uint8_t *misc = smem + kOffMisc;
+    const uint32_t bars = smem0 + kOffMisc;                               // kNumBars x 8 bytes
+    int *meta = reinterpret_cast<int *>(misc + 256);                      // [kStages] valid keys per stage
+    uint32_t *anc = reinterpret_cast<uint32_t *>(misc + 320);             // [32] visible-draft masks
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 448);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 456);
+    auto bar = [&](int slot) { return bars + 8u * slot; };
+
+    const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int upb = p.B / kUnit;
+    const bool has_draft = split == p.splits - 1;
+    const int rows = p.G * p.T;
+    constexpr int RPQ = 8 * NH;                              // query rows per TMEM lane quadrant
+    const int n_active = min(4, (rows + RPQ - 1) / RPQ);     // warps per softmax warpgroup that own real rows
+
+    if (tid == 0) TC_STAMP(0);
+    // The TMA producer warp initialises the barriers and runs ahead; everybody else meets it at a named
+    // barrier (the producer only arrives), with the TMEM allocation done by warp 9 on the way.
+    if (warp == 8) {
+        if (lane < kNumBars) {
+            uint32_t count = 1;
+            if (lane >= kSFree && lane < kSFree + 2) count = n_active;
+            if (lane >= kPReady && lane < kPReady + 2) count = n_active;
+            if (lane >= kOFree && lane < kOFree + 2) count = n_active;
+            if (lane == kStaged) count = 8;
+            if (lane == kTmemDone) count = 2 * n_active;
+            mbar_init(bar(lane), count);
+            mbar_fence_init();
+        }
+        if (lane == 0) *abort_flag = 0;
+        __syncwarp();
+        named_bar_arrive(3, kThreads);
+    } else {
+        if (warp == 9) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tc_fence_before_sync();
+        named_bar_sync(3, kThreads);
+        tc_fence_after_sync();
+    }
+    const uint32_t tmem_base = warp == 8 ? 0u : *tmem_slot;
+    if (tid == 0) TC_STAMP(1);
+
+    if (warp >= 8) {
+        reg_dealloc<40>();   // hand registers to the softmax warpgroups
+        if (warp == 8) {
+            // ---------------------------------------------------------- TMA producer
+            if (lane == 0) {
+                tma_prefetch_desc(&tm_k);
+                tma_prefetch_desc(&tm_v);
+            }
+            const uint64_t policy = policy_evict_first();
+            // pull this sequence's block-table row towards L2 while the previous kernel drains
+            for (int i = lane * 32; i < p.NBmax; i += 32 * 32) prefetch_l2(p.block_table + (size_t)s * p.NBmax + i);
+            grid_dependency_wait();   // the block list is written by the kernel just before
+            // First batch of block indices speculatively, assuming the list is full (cnt == max_sel): its
+            // load then overlaps the loads of the count and the length instead of following them.
+            const int j0_spec = (int)((long long)split * p.max_sel / p.splits);
+            int blk_spec = 0;
+            if (p.sel_idx && j0_spec + lane < p.max_sel)
+                blk_spec = p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j0_spec + lane];
+            const int L = p.seq_lens[s];
+            const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+            const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
+            const int j0 = (int)((long long)split * n_sel / p.splits);
+            const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+            bool dead = false;
+            for (int base = j0; base < j1; base += 32) {
+                const int j = base + lane;
+                int row0 = 0, tok0 = 0;
+                if (j < j1) {
+                    int blk = j;
+                    if (p.sel_idx)
+                        blk = (base == j0 && j0 == j0_spec) ? blk_spec : p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j];
+                    blk = max(0, min(blk, p.NBmax - 1));
+                    const int page = p.block_table[(size_t)s * p.NBmax + blk];
+                    row0 = (page * p.Hkv + h) * p.B;
+                    tok0 = blk * p.B;
+                }
+                const int n_here = min(32, j1 - base);
+                for (int i = 0; i < n_here; ++i) {
+                    const int r0 = __shfl_sync(0xffffffffu, row0, i);
+                    const int t0 = __shfl_sync(0xffffffffu, tok0, i);
+                    if (lane == 0 && !dead) {
+                        for (int uo = 0; uo < upb; ++uo) {
+                            const int u = (base - j0 + i) * upb + uo;
+                            const int stage = u % kStages, it = u / kStages;
+                            if (it > 0 && (*abort_flag || !mbar_wait_bounded(bar(kEmpty + stage), (it - 1) & 1))) {
+                                dead = true;
+                                *abort_flag = 1;
+                                if (p.status) atomicOr(p.status, 1);
+                                break;
+                            }
+                            const int nvalid = max(0, min(kUnit, L - (t0 + uo * kUnit)));
+                            meta[stage] = nvalid;
+                            const uint32_t fb = bar(kFull + stage);
+                            const uint32_t dst = smem0 + stage * kStageBytes;
+                            const int y = r0 + uo * kUnit;
+                            // an empty unit (block 128, tail of at most 64 tokens) is still loaded:
+                            // it keeps the unit sequence uniform and is fully masked downstream
+                            if (u < 24) TC_STAMP(8 + u);
+                            mbar_arrive_expect_tx(fb, kStageBytes);
+                            tma_load_2d(dst, &tm_k, 0, y, fb, policy);
+                            tma_load_2d(dst + kTile, &tm_k, 64, y, fb, policy);
+                            tma_load_2d(dst + 2 * kTile, &tm_v, 0, y, fb, policy);
+                            tma_load_2d(dst + 3 * kTile, &tm_v, 64, y, fb, policy);
+                        }
+                    }
+                }
+            }
+        } else if (warp == 9 || warp == 10) {
+            // ---------------------------------------------------------- MMA issuers (one thread each)
+            // warp 9 issues every S = Q K^T and owns the TMEM allocation; warp 10 issues every Ou = P V.
+            // Descriptors are built once; per instruction only the 14-bit address field moves.
+            if (lane == 0) {
+                const int L = p.seq_lens[s];
+                grid_dependency_wait();
+                const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+                const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
+                const int j0 = (int)((long long)split * n_sel / p.splits);
+                const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+                const int off = has_draft ? 1 : 0;
+                const int n_total = (j1 - j0) * upb + off;
+                bool dead = !mbar_wait_bounded(bar(kStaged), 0);
+                if (warp == 9) {
+                    constexpr uint32_t idesc_s = umma_idesc_bf16(128, kUnit, false);
+                    const uint64_t dq = umma_desc_sw128(smem0 + kOffQ, 16, 1024);
+                    const uint64_t dk = umma_desc_sw128(smem0, 16, 1024);
+                    const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk;
+                    const uint64_t d_hi = dq & 0xFFFFFFFF00000000ull;
+                    for (int u = 0; u < n_total && !dead; ++u) {
+                        const int g = u & 1, k = u >> 1;
+                        const bool ring = u >= off;
+                        const int stage = ring ? (u - off) % kStages : 0;
+                        const int it = ring ? (u - off) / kStages : 0;
+                        if (*abort_flag || (ring && !mbar_wait_bounded(bar(kFull + stage), it & 1)) ||
+                            (k > 0 && !mbar_wait_bounded(bar(kSFree + g), (k - 1) & 1))) {
+                            dead = true;
+                            *abort_flag = 1;
+                            if (p.status) atomicOr(p.status, 8);
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        const uint32_t k_lo = dk_lo + (uint32_t)((ring ? stage * kStageBytes : kOffDraft) >> 4);
+                        const uint32_t d = tmem_base + g * kUnit;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint32_t qo = (uint32_t)(((ks >> 2) * (kQBytes / 2) + (ks & 3) * 32) >> 4);
+                            const uint32_t ko = (uint32_t)(((ks >> 2) * kTile + (ks & 3) * 32) >> 4);
+                            tc_mma_bf16(d, d_hi | (dq_lo + qo), d_hi | (k_lo + ko), idesc_s, ks > 0);
+                        }
+                        tc_commit(bar(kSReady + g));
+                        if (u < 24) TC_STAMP(32 + u);
+                    }
+                    // free TMEM only after every softmax warp has finished reading it
+                    if (!mbar_wait_bounded(bar(kTmemDone), 0) && p.status) atomicOr(p.status, 16);
+                } else {
+                    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, true);
+                    const uint64_t dp = umma_desc_sw128(smem0 + kOffP, 16, 1024);
+                    const uint64_t dv = umma_desc_sw128(smem0 + 2 * kTile, kTile, 1024);
+                    const uint32_t dp_lo = (uint32_t)dp, dv_lo = (uint32_t)dv;
+                    const uint64_t dp_hi = dp & 0xFFFFFFFF00000000ull, dv_hi = dv & 0xFFFFFFFF00000000ull;
+                    for (int u = 0; u < n_total && !dead; ++u) {
+                        const int g = u & 1, k = u >> 1;
+                        const bool ring = u >= off;
+                        const int stage = ring ? (u - off) % kStages : 0;
+                        if (*abort_flag || !mbar_wait_bounded(bar(kPReady + g), k & 1) ||
+                            (k > 0 && !mbar_wait_bounded(bar(kOFree + g), (k - 1) & 1))) {
+                            dead = true;
+                            *abort_flag = 1;
+                            if (p.status) atomicOr(p.status, 32);
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        const uint32_t v_lo = dv_lo + (uint32_t)((ring ? stage * kStageBytes : kOffDraft) >> 4);
+                        const uint32_t p_lo = dp_lo + (uint32_t)((g * kPBytes) >> 4);
+                        const uint32_t d = tmem_base + 128 + g * 128;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            tc_mma_bf16(d, dp_hi | (p_lo + (uint32_t)((kk * 32) >> 4)), dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)),
+                                        idesc_pv, kk > 0);
+                        tc_commit(bar(kOReady + g));
+                        if (ring) tc_commit(bar(kEmpty + stage));
+                        if (u < 24) TC_STAMP(56 + u);
+                    }
+                }
+            }
+            if (warp == 9) {
+                __syncwarp();
+                tc_fence_after_sync();
+                tmem_dealloc(tmem_base, kTmemCols);
+            }
+        }
+        return;
+    }
+
+    // ------------------------------------------------------------------ softmax warpgroups
+    reg_alloc<232>();
+    // Stage Q and, in the last split, the draft tokens' K/V as one more unit; both in the swizzled layout
+    // the tensor cores read.  Query row r = i*G + g (q[s][i][h*G + g][:]) goes to tile row
+    // (r / RPQ)*32 + r % RPQ: RPQ rows per TMEM lane quadrant, so that all four warps of a warpgroup
+    // share the softmax work even when only a few of the 128 tile rows are real.
+    // The zero padding needs no input and is written while the previous kernel in the stream drains.
+    for (int idx = tid; idx < 128 * 16; idx += 256) {
+        const int tr = idx >> 4, c = idx & 15;
+        const int r = (tr >> 5) * RPQ + (tr & 31);
+        if (!((tr & 31) < RPQ && r < rows))
+            *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (has_draft) {
+        for (int idx = tid; idx < 2 * kUnit * 16; idx += 256) {
+            const int which = idx / (kUnit * 16);   // 0: K, 1: V
+            const int r = (idx >> 4) % kUnit, c = idx & 15;
+            if (r >= p.T)
+                *reinterpret_cast<uint4 *>(smem + kOffDraft + which * (2 * kTile) + (c >> 3) * kTile + swz128(r, c & 7)) =
+                    make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    grid_dependency_wait();
+    grid_launch_dependents();   // the next kernel may be scheduled; it waits for this grid before reading
+    {
+        // real rows: all loads of a thread are in flight together
+        const int n_q = rows * 16, n_d = has_draft ? 2 * p.T * 16 : 0;
+        uint4 v[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int idx = tid + x * 256;
+            if (idx < n_q) {
+                const int r = idx >> 4, c = idx & 15;
+                const int i = r / p.G, g = r - i * p.G;
+                v[x] = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
+            }
+        }
+        uint4 w[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int idx = tid + x * 256;
+            if (idx < n_d) {
+                const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
+                const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
+                w[x] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
+            }
+        }
+        if (has_draft && tid < 32) {
+            uint32_t mask = 0;
+            if (tid < p.T) {
+                if (p.parent) {
+                    int a = tid;
+                    for (int step = 0; step < p.T && a >= 0; ++step) {
+                        mask |= 1u << a;
+                        const int nxt = p.parent[(size_t)s * p.T + a];
+                        a = nxt < a ? nxt : -1;   // parents must precede their children
+                    }
+                } else {
+                    mask = (tid == 31) ? 0xFFFFFFFFu : ((1u << (tid + 1)) - 1u);
+                }
+            }
+            anc[tid] = mask;
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int idx = tid + x * 256;
+            if (idx < n_q) {
+                const int r = idx >> 4, c = idx & 15;
+                const int tr = (r / RPQ) * 32 + (r % RPQ);
+                *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = v[x];
+            }
+            if (idx < n_d) {
+                const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
+                *reinterpret_cast<uint4 *>(smem + kOffDraft + which * (2 * kTile) + (c >> 3) * kTile + swz128(r, c & 7)) = w[x];
+            }
+        }
+        // shapes with more than 64 query rows or more than 16 draft tokens: the remaining chunks
+        for (int idx = tid + 4 * 256; idx < n_q; idx += 256) {
+            const int r = idx >> 4, c = idx & 15;
+            const int i = r / p.G, g = r - i * p.G;
+            const int tr = (r / RPQ) * 32 + (r % RPQ);
+            *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) =
+                __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
+        }
+        for (int idx = tid + 4 * 256; idx < n_d; idx += 256) {
+            const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
+            const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
+            *reinterpret_cast<uint4 *>(smem + kOffDraft + which * (2 * kTile) + (c >> 3) * kTile + swz128(r, c & 7)) =
+                __ldg(reinterpret_cast<const uint4 *>(src) + c);
+        }
+    }
+    fence_proxy_async();   // the tensor cores read these tiles through the async proxy
+    named_bar_sync(2, 256);
+    if (lane == 0) mbar_arrive(bar(kStaged));
+    if (tid == 0) TC_STAMP(2);
+
+    const int wg = warp >> 2, quad = warp & 3;
+    if (quad >= n_active) return;                                 // this warp's TMEM lanes hold padding only
+    const int qd = lane & 3, lr = lane >> 2;
+    const uint32_t t_lane = (uint32_t)(quad * 32) << 16;
+    const uint32_t t_s = tmem_base + t_lane + wg * kUnit;
+    const uint32_t t_o = tmem_base + t_lane + 128 + wg * 128;
+    const uint32_t all_t = (p.T == 32) ? 0xFFFFFFFFu : ((1u << p.T) - 1u);
+    const int wg_threads = n_active * 32;
+    uint32_t vis[NH];
+    int trow[NH], lrow[NH];
+#pragma unroll
+    for (int i = 0; i < NH; ++i) {
+        lrow[i] = quad * RPQ + 8 * i + lr;
+        trow[i] = quad * 32 + 8 * i + lr;
+        vis[i] = (has_draft && lrow[i] < rows) ? anc[lrow[i] / p.G] : all_t;
+    }
+
+    const int L = p.seq_lens[s];
+    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+    const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
+    const int j0 = (int)((long long)split * n_sel / p.splits);
+    const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+    const int off = has_draft ? 1 : 0;
+    const int n_total = (j1 - j0) * upb + off;
+
+    // per slot: 32 output dims 8*jj + 2*qd + e  (index 2*jj + e), running max and partial row sum
+    float o[NH][32], m[NH], l[NH], corr_prev[NH];
+#pragma unroll
+    for (int i = 0; i < NH; ++i) {
+#pragma unroll
+        for (int d = 0; d < 32; ++d) o[i][d] = 0.f;
+        m[i] = -INFINITY;
+        l[i] = 0.f;
+        corr_prev[i] = 1.f;
+    }
+    bool dead = false;
+
+    // O = O * corr + Ou for the warpgroup's k-th unit, then hand the Ou buffer back
+    auto accumulate = [&](int k) {
+        if (!dead && __any_sync(0xffffffffu, *abort_flag || !mbar_wait_bounded(bar(kOReady + wg), k & 1))) {
+            dead = true;   // warp-uniform: the tcgen05.ld below must be executed by the whole warp or not at all
+            *abort_flag = 1;
+            if (p.status && lane == 0) atomicOr(p.status, 4);
+        }
+        if (dead) return;
+        if (tid == 0 && k < 12) TC_STAMP(104 + k);
+        tc_fence_after_sync();
+#pragma unroll
+        for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t r[32];
+                tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + c * 64, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int i = lo * 2 + hh;
+                            o[i][(c * 8 + j) * 2 + e] = fmaf(o[i][(c * 8 + j) * 2 + e], corr_prev[i], __uint_as_float(r[4 * j + 2 * hh + e]));
+                        }
+            }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kOFree + wg));
+    };
+
+    int k = 0;
+    for (int u = wg; u < n_total; u += 2, ++k) {
+        if (!dead && __any_sync(0xffffffffu, *abort_flag || !mbar_wait_bounded(bar(kSReady + wg), k & 1))) {
+            dead = true;
+            *abort_flag = 1;
+            if (p.status && lane == 0) atomicOr(p.status, 2);
+        }
+        if (dead) break;
+        if (tid == 0 && k < 12) TC_STAMP(80 + k);
+        tc_fence_after_sync();
+        uint32_t sr[NH == 4 ? 2 : 1][32];
+        tmem_ld_16x256b_x8(t_s, sr[0]);
+        if constexpr (NH == 4) tmem_ld_16x256b_x8(t_s + (16u << 16), sr[1]);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kSFree + wg));   // the next S of this warpgroup may be issued
+
+        if (k > 0) accumulate(k - 1);                   // Ou of the previous unit is normally ready by now
+
+        const bool is_draft = u < off;
+        const int stage = is_draft ? 0 : (u - off) % kStages;
+        const int nvalid = is_draft ? p.T : min(meta[stage], kUnit);
+        uint8_t *pbuf = smem + kOffP + wg * kPBytes;
+#pragma unroll
+        for (int i = 0; i < NH; ++i) {
+            float sc[16];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) sc[2 * j + e] = __uint_as_float(sr[i >> 1][4 * j + 2 * (i & 1) + e]);
+            if (is_draft || nvalid < kUnit) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int col = 8 * j + 2 * qd + e;
+                        bool ok = col < nvalid;
+                        if (is_draft) ok = ok && col < 32 && ((vis[i] >> (col & 31)) & 1u);
+                        if (!ok) sc[2 * j + e] = -INFINITY;
+                    }
+            }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) mx = fmaxf(mx, sc[c]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m[i], mx * p.scale_log2);
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            corr_prev[i] = fast_exp2(m[i] - m_use);
+            m[i] = m_new;
+            float lsum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float p0 = fast_exp2(fmaf(sc[2 * j], p.scale_log2, -m_use));
+                const float p1 = fast_exp2(fmaf(sc[2 * j + 1], p.scale_log2, -m_use));
+                lsum += p0 + p1;
+                *reinterpret_cast<uint32_t *>(pbuf + swz128(trow[i], j) + 4 * qd) = pack_bf16(p0, p1);
+            }
+            l[i] = l[i] * corr_prev[i] + lsum;
+        }
+        if (!is_draft && nvalid < kUnit) {
+            // zero the value rows past the end of the sequence (0 * junk must stay 0)
+            const int t = quad * 32 + lane;
+            for (int idx = t; idx < (kUnit - nvalid) * 16; idx += wg_threads) {
+                const int r = nvalid + (idx >> 4), c = idx & 15;
+                *reinterpret_cast<uint4 *>(smem + stage * kStageBytes + 2 * kTile + (c >> 3) * kTile + swz128(r, c & 7)) =
+                    make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kPReady + wg));
+        if (tid == 0 && k < 12) TC_STAMP(92 + k);
+    }
+    if (k > 0) accumulate(k - 1);
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(kTmemDone));
+
+    // ------------------------------------------------------------------ merge the two warpgroups, write out
+    const int n_sm = 2 * wg_threads;
+    named_bar_sync(1, n_sm);   // both warpgroups are past their last unit: the ring is free
+    float *mx_buf = reinterpret_cast<float *>(smem);             // [NH*34][128] floats, index k*128 + t
+    const int t = quad * 32 + lane;
+    if (wg == 1) {
+#pragma unroll
+        for (int i = 0; i < NH; ++i) {
+#pragma unroll
+            for (int d = 0; d < 32; ++d) mx_buf[(i * 34 + d) * 128 + t] = o[i][d];
+            mx_buf[(i * 34 + 32) * 128 + t] = m[i];
+            mx_buf[(i * 34 + 33) * 128 + t] = l[i];
+        }
+    }
+    named_bar_sync(1, n_sm);
+    if (wg == 1) return;
+#pragma unroll
+    for (int i = 0; i < NH; ++i) {
+        const float m1 = mx_buf[(i * 34 + 32) * 128 + t], l1 = mx_buf[(i * 34 + 33) * 128 + t];
+        const float M = fmaxf(m[i], m1);
+        const float M_use = (M == -INFINITY) ? 0.f : M;
+        const float w0 = fast_exp2(m[i] - M_use), w1 = fast_exp2(m1 - M_use);
+        float lsum = w0 * l[i] + w1 * l1;
+        lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+        lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+#pragma unroll
+        for (int d = 0; d < 32; ++d) o[i][d] = w0 * o[i][d] + w1 * mx_buf[(i * 34 + d) * 128 + t];
+        const int row = lrow[i];
+        if (row >= rows) continue;
+        if (p.splits == 1) {
+            const int ii = row / p.G, g = row - ii * p.G;
+            const size_t orow = ((size_t)s * p.T + ii) * p.Hq + h * p.G + g;
+            const float inv = 1.f / lsum;
+            uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + qd;
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) dst[4 * jj] = pack_bf16(o[i][2 * jj] * inv, o[i][2 * jj + 1] * inv);
+            if (p.lse && qd == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
+        } else {
+            const size_t prow = (((size_t)s * p.Hkv + h) * p.splits + split) * rows + row;
+            float2 *dst = reinterpret_cast<float2 *>(p.ws_o + prow * 128) + qd;
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) dst[4 * jj] = make_float2(o[i][2 * jj], o[i][2 * jj + 1]);
+            if (qd == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
+        }
+    }
+    if (tid == 0) TC_STAMP(120);
+}
+
+}  // namespace
+
+template <int NH>
+static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
+                             cudaStream_t stream)
+{
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(verify_attn_tc_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH>, tm_k, tm_v, p);
+}
+
+cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
+                           cudaStream_t stream)
+{
+    const int rows = p.G * p.T;
+    if (rows <= 32) return launch_tc<1>(tm_k, tm_v, p, grid, stream);
+    if (rows <= 64) return launch_tc<2>(tm_k, tm_v, p, grid, stream);
+    return launch_tc<4>(tm_k, tm_v, p, grid, stream);
+}
+
+}  // namespace svk

@@ -35,12 +35,34 @@ class SparseVerifier:
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.kv: List[Optional[sv.sv_kv]] = [None] * n_layers
         self._pools = [None] * n_layers   # keep the tensors alive
-        self._side = None
-        self._events = None
+        self._stack_kv = None
 
     def set_layer_kv(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
         self._pools[layer] = (k_pool, v_pool)
         self.kv[layer] = sv.make_kv(k_pool, v_pool, self.block_table, self.seq_lens)
+
+    def set_kv_stack(self, k_all: torch.Tensor, v_all: torch.Tensor) -> None:
+        """All layers' pools in one allocation, bf16 [layers][n_pages][Hkv][B][D].  Besides the per-layer
+        descriptors this builds a stacked view in which (layer, sequence) is the batch dimension, so that
+        the tail-block refresh of every layer is a single sv_block_reps launch."""
+        n_layers, n_pages = int(k_all.shape[0]), int(k_all.shape[1])
+        assert n_layers == self.n_layers and k_all.is_contiguous() and v_all.is_contiguous()
+        for l in range(n_layers):
+            self.set_layer_kv(l, k_all[l], v_all[l])
+        g = self.geom
+        offs = (torch.arange(n_layers, device=k_all.device, dtype=torch.int32) * n_pages).view(n_layers, 1, 1)
+        self._stack_table = (self.block_table.unsqueeze(0) + offs).reshape(n_layers * g.n_seq, g.max_blocks).contiguous()
+        self._stack_lens = self.seq_lens.repeat(n_layers).contiguous()
+        self._stack_geom = sv.make_geom(g.n_seq * n_layers, g.n_q_heads, g.n_kv_heads, g.head_dim, g.block_size,
+                                        g.max_blocks, g.n_draft)
+        self._stack_pools = (k_all, v_all)
+        self._stack_kv = sv.make_kv(k_all.view(n_layers * n_pages, *k_all.shape[2:]),
+                                    v_all.view(n_layers * n_pages, *v_all.shape[2:]), self._stack_table,
+                                    self._stack_lens)
+
+    def refresh_tail_all(self) -> None:
+        """Recompute the representative of every sequence's last block in all layers (one launch)."""
+        sv.sv_block_reps(self._stack_geom, self._stack_kv, self.reps.view(-1, *self.reps.shape[2:]), sv.SV_TAIL_BLOCK)
 
     def build_reps(self, layer: int, block_begin: int = 0, block_end: int = -1) -> None:
         """(Re)compute block representatives of a layer; a decoding loop only refreshes the tail block."""
@@ -68,27 +90,18 @@ class SparseVerifier:
     def verify_step(self, q, draft_k, draft_v, out, refresh_tail: bool = False) -> None:
         """One verification step of the whole stack.  q/out: [layers][S][T][Hq][D]; draft_k/v: [layers][S][T][Hkv][D].
 
-        refresh_tail: first recompute the representative of every sequence's last block in the anchor
-        layers (the block that grew when the previous step's accepted tokens were appended).  These
-        small launches do not depend on the layer chain, so they go to a side stream and each anchor
-        layer waits only for its own."""
-        cur = torch.cuda.current_stream()
+        refresh_tail: first recompute the representative of every sequence's last block (the block that
+        grew when the previous step's accepted tokens were appended) -- one launch for all layers when the
+        pools were given with set_kv_stack, else one per anchor layer."""
         if refresh_tail:
-            if self._side is None:
-                self._side = torch.cuda.Stream()
-                self._events = [torch.cuda.Event() for _ in range(self.n_layers)]
-            self._side.wait_stream(cur)
-            with torch.cuda.stream(self._side):
+            if self._stack_kv is not None:
+                self.refresh_tail_all()
+            else:
                 for l in range(self.n_layers):
                     if self.anchors[l]:
                         sv.sv_block_reps(self.geom, self.kv[l], self.reps[l], sv.SV_TAIL_BLOCK)
-                        self._events[l].record(self._side)
         for l in range(self.n_layers):
-            if refresh_tail and self.anchors[l]:
-                cur.wait_event(self._events[l])
             self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l])
-        if refresh_tail:
-            cur.wait_stream(self._side)
 
     def dense_step(self, q, draft_k, draft_v, out) -> None:
         for l in range(self.n_layers):
@@ -100,4 +113,5 @@ class SparseVerifier:
         attn = self.n_layers * (2 if splits > 1 else 1)
         if dense:
             return attn
-        return sum(self.anchors) * (2 if refresh_tail else 1) + attn
+        refresh = 0 if not refresh_tail else (1 if self._stack_kv is not None else sum(self.anchors))
+        return refresh + sum(self.anchors) + attn

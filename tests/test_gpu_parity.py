@@ -354,3 +354,33 @@ def test_full_size_cfg3_sampled(sv):
 def test_sweep_points(sv, point):
     c = si.make_layer(si.make_geometry(si.sweep_workload(*point)), sharp=True)
     _sampled_check(sv, c, 48, f"sweep {point}")
+
+
+def test_stacked_tail_refresh_equals_per_layer(sv):
+    """set_kv_stack: one sv_block_reps launch refreshes the tail block of every layer."""
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(900, 2000), budget_blocks=10, n_layers=3)
+    geom = si.make_geometry(w)
+    layers = [si.make_layer(geom, layer=l) for l in range(3)]
+    eng = sv.SparseVerifier(n_seq=3, n_q_heads=32, n_kv_heads=8, head_dim=128, block_size=64,
+                            max_blocks=geom["max_blocks"], n_draft=5, n_layers=3,
+                            block_table=torch.from_numpy(geom["block_table"]).cuda(),
+                            seq_lens=torch.from_numpy(geom["seq_lens"]).cuda(),
+                            budget_blocks=torch.from_numpy(geom["budget"]).cuda(), max_sel=geom["max_sel"])
+    k_all = torch.stack([bf16_dev(c["k_pool"]) for c in layers])
+    v_all = torch.stack([bf16_dev(c["v_pool"]) for c in layers])
+    eng.set_kv_stack(k_all, v_all)
+    for l in range(3):
+        eng.build_reps(l)
+    full = eng.reps.clone()
+    eng.reps.fill_(5.0)
+    eng.refresh_tail_all()
+    torch.cuda.synchronize()
+    for l in range(3):
+        for s in range(3):
+            t = int(geom["n_blocks"][s]) - 1
+            assert torch.equal(eng.reps[l, s, :, t], full[l, s, :, t])
+            assert (eng.reps[l, s, :, :t] == 5.0).all()
+        ref = oracle.block_reps(layers[l]["k_pool"], geom["block_table"], geom["seq_lens"])
+        for s in range(3):
+            nb = int(geom["n_blocks"][s])
+            np.testing.assert_allclose(full[l, s, :, :nb].cpu().numpy(), ref[s, :, :nb], rtol=1e-5, atol=1e-6)
