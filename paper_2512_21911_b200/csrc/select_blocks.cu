@@ -17,6 +17,26 @@
 
 namespace cg = cooperative_groups;
 
+#ifdef SV_TRACE
+// Development aid (never compiled into the library): cycle stamps of cluster 0.
+__device__ long long g_sv_trace_sel[8 * 32];
+extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_sel()
+{
+    long long *p = nullptr;
+    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace_sel);
+    return p;
+}
+#define SEL_STAMP(slot)                                                                              \
+    do {                                                                                             \
+        if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 8)                \
+            g_sv_trace_sel[blockIdx.x * 32 + (slot)] = clock64();                                    \
+    } while (0)
+#else
+#define SEL_STAMP(slot) \
+    do {                \
+    } while (0)
+#endif
+
 namespace {
 
 constexpr int kThreads = 512;
@@ -40,6 +60,40 @@ struct SelectParams {
     int T, Hq, Hkv, B, NBmax, n_sink, n_local, max_sel, chunk;
 };
 
+__device__ __forceinline__ uint32_t cluster_map_shared(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_shared_cluster_v4(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t parity, uint32_t limit = (1u << 19))
+{
+    for (uint32_t i = 0; i < limit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+// Cluster of CL CTAs per (sequence, KV head).  Every CTA scores a slice of the blocks and writes the
+// keys straight into CTA 0's shared memory (distributed shared memory), then signals an mbarrier there
+// and exits; CTA 0 selects.  The only cluster-wide barrier is split (arrive early, wait late) so that
+// its latency hides behind the loads.
 __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
 {
     cg::cluster_group cluster = cg::this_cluster();
@@ -48,167 +102,201 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     const int h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    extern __shared__ uint32_t smem_keys[];
-    uint32_t *keys_local = smem_keys;              // [chunk]   this CTA's slice
-    uint32_t *keys_all = smem_keys + p.chunk;      // [CL*chunk] gathered by CTA 0
+    extern __shared__ __align__(16) uint32_t keys_all[];         // [CL*chunk] keys of all blocks (used in CTA 0)
     __shared__ float qbar[128];
-    __shared__ uint32_t hist[256];
-    __shared__ uint32_t sh_bin, sh_remaining;
+    __shared__ uint32_t hist[4][256];
     __shared__ uint32_t warp_sel[kWarps], warp_eq[kWarps];
+    __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: one arrival per CTA of the cluster
 
-    const int L = p.seq_lens[s];
-    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
-    const int forced = min(nb, p.n_sink + p.n_local);
-    int N = min(max(p.budget[s], forced), p.max_sel);
-    const bool keep_all = N >= nb;
-    if (keep_all) N = nb;
-
-    // While the kernel that precedes this one in the stream drains, pull this warp's first batch of
-    // representative rows towards L2 (a prefetch consumes no data, so it is safe even if that kernel
-    // is still writing them); all real loads come after the dependency wait.
-    const bool need_scores = !keep_all || p.out_scores;
-    const int b0 = rank * p.chunk;
-    const int b1 = min(b0 + p.chunk, nb);
-    const float4 *rbase = reinterpret_cast<const float4 *>(p.reps + ((size_t)s * p.Hkv + h) * p.NBmax * 128);
-    float4 r[kRowsPerIter];
-    int b = b0 + warp * kRowsPerIter;
-    auto load_rows = [&](int bb) {
-#pragma unroll
-        for (int i = 0; i < kRowsPerIter; ++i)
-            r[i] = (bb + i < b1) ? __ldg(rbase + (size_t)(bb + i) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
-    };
-    if (need_scores) {
-#pragma unroll
-        for (int i = 0; i < kRowsPerIter; ++i)
-            if (b + i < b1) svk::prefetch_l2(rbase + (size_t)(b + i) * 32 + lane);
+    SEL_STAMP(0);
+    // While the kernel that precedes this one in the stream drains: pull this warp's first batch of
+    // representative rows and the query row towards L2 (a prefetch consumes no data, so it is safe even if
+    // that kernel is still writing them), set up the barrier, zero the histograms.
+    if (tid == 0) {
+        svk::mbar_init(svk::smem_u32(&keys_ready), CL);
+        svk::mbar_fence_init();
     }
+    for (int i = tid; i < 4 * 256; i += kThreads) (&hist[0][0])[i] = 0;
+    SEL_STAMP(10);
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // before any global request is in flight
+    SEL_STAMP(11);
+    const int b0 = rank * p.chunk;
+    const float4 *rbase = reinterpret_cast<const float4 *>(p.reps + ((size_t)s * p.Hkv + h) * p.NBmax * 128);
+    int b = b0 + warp * kRowsPerIter;
+#pragma unroll
+    for (int i = 0; i < kRowsPerIter; ++i)
+        if (b + i < min(b0 + p.chunk, p.NBmax)) svk::prefetch_l2(rbase + (size_t)(b + i) * 32 + lane);
+    const int G = p.Hq / p.Hkv;
+    const __nv_bfloat16 *q0 = p.q + ((size_t)s * p.T * p.Hq + (size_t)h * G) * 128;
+    if (tid < G * 2) svk::prefetch_l2(q0 + tid * 64);
+    SEL_STAMP(1);
     svk::grid_dependency_wait();
     svk::grid_launch_dependents();
-    if (need_scores && b < b1) load_rows(b);
+    SEL_STAMP(2);
+
+    // every load below is issued before the first use
+    const int L = p.seq_lens[s];
+    const int budget = p.budget[s];
+    float4 r[kRowsPerIter];
+    auto load_rows = [&](int bb, int hi) {
+#pragma unroll
+        for (int i = 0; i < kRowsPerIter; ++i)
+            r[i] = (bb + i < hi) ? __ldg(rbase + (size_t)(bb + i) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    load_rows(b, min(b0 + p.chunk, p.NBmax));
+    float qsum = 0.f;
+    if (tid < 128)
+        for (int g = 0; g < G; ++g) qsum += __bfloat162float(q0[(size_t)g * 128 + tid]);
+
+    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+    const int forced = min(nb, p.n_sink + p.n_local);
+    int N = min(max(budget, forced), p.max_sel);
+    const bool keep_all = N >= nb;
+    if (keep_all) N = nb;
+    const bool need_scores = !keep_all || p.out_scores;
+    const int b1 = min(b0 + p.chunk, nb);
 
     // retrieval query: mean of the first draft token's query over the GQA group
-    const int G = p.Hq / p.Hkv;
-    if (tid < 128) {
-        const __nv_bfloat16 *q0 = p.q + ((size_t)s * p.T * p.Hq + (size_t)h * G) * 128 + tid;
-        float sum = 0.f;
-        for (int g = 0; g < G; ++g) sum += __bfloat162float(q0[(size_t)g * 128]);
-        qbar[tid] = sum / (float)G;
-    }
+    if (tid < 128) qbar[tid] = qsum / (float)G;
     __syncthreads();
+    SEL_STAMP(3);
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // CTA 0's barrier is initialised
+    SEL_STAMP(12);
 
+    const uint32_t keys0 = cluster_map_shared(svk::smem_u32(keys_all), 0);
     if (need_scores) {
         const float4 qv = reinterpret_cast<const float4 *>(qbar)[lane];
         for (; b < b1; b += kWarps * kRowsPerIter) {
+            uint32_t kk[kRowsPerIter];
 #pragma unroll
             for (int i = 0; i < kRowsPerIter; ++i) {
                 float d = r[i].x * qv.x + r[i].y * qv.y + r[i].z * qv.z + r[i].w * qv.w;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-                if (lane == 0 && b + i < b1) {
-                    const int bb = b + i;
-                    const bool is_forced = bb < p.n_sink || bb >= nb - p.n_local;
-                    keys_local[bb - b0] = is_forced ? 0xFFFFFFFFu : order_key(d);
-                    if (p.out_scores) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = d;
-                }
+                const int bb = b + i;
+                const bool is_forced = bb < p.n_sink || bb >= nb - p.n_local;
+                kk[i] = is_forced ? 0xFFFFFFFFu : order_key(d);
+                if (p.out_scores && lane == 0 && bb < b1) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = d;
             }
-            if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter);
+            // rows b .. b+3 are 4 consecutive keys: one 16-byte store into CTA 0 (entries past nb are never read)
+            if (lane == 0 && !keep_all) st_shared_cluster_v4(keys0 + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]));
+            if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter, b1);
         }
     }
-    cluster.sync();
-    if (rank == 0 && !keep_all) {
-        for (int b = tid; b < nb; b += kThreads) {
-            const uint32_t *remote = cluster.map_shared_rank(keys_local, b / p.chunk);
-            keys_all[b] = remote[b % p.chunk];
-        }
-    }
-    cluster.sync();   // no CTA may exit while CTA 0 still reads its shared memory
+    SEL_STAMP(13);
+    __syncthreads();   // the release (cluster scope) of the arrive below covers the stores this barrier ordered before it
+    SEL_STAMP(4);
+    if (tid == 0) mbar_arrive_cluster(cluster_map_shared(svk::smem_u32(&keys_ready), 0));
     if (rank != 0) return;
 
     int32_t *out = p.out_idx + ((size_t)s * p.Hkv + h) * p.max_sel;
     if (keep_all) {
-        for (int b = tid; b < nb; b += kThreads) out[b] = b;
+        for (int bb = tid; bb < nb; bb += kThreads) out[bb] = bb;
         if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = nb;
+        // the other CTAs still signal the barrier in this CTA's shared memory: wait for them before exiting
+        mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0);
         return;
     }
+    if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) return;   // gave up: leave the output untouched
+    SEL_STAMP(5);
 
-    // exact radix select of the N-th largest key
+    // exact radix select of the N-th largest key: up to 4 passes of 8 bits, one histogram per pass.  Every
+    // warp scans the histogram itself (one block barrier per pass), and the passes stop as soon as the
+    // boundary bin is taken whole (then every key with the prefix found so far is kept).
     uint32_t prefix = 0, mask = 0, remaining = (uint32_t)N;
 #pragma unroll 1
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        if (tid < 256) hist[tid] = 0;
-        __syncthreads();
-        for (int b = tid; b < nb; b += kThreads) {
-            const uint32_t k = keys_all[b];
-            if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        // one shared-memory atomic per distinct digit per warp (scores share their leading bits, so
+        // un-aggregated atomics would pile onto a single bin)
+        for (int c0 = 0; c0 < nb; c0 += kThreads) {
+            const int bb = c0 + tid;
+            const uint32_t k = bb < nb ? keys_all[bb] : 0u;
+            const bool cand = bb < nb && (k & mask) == prefix;
+            const uint32_t digit = cand ? ((k >> shift) & 255u) : 256u;
+            const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+            if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[pass][digit], (uint32_t)__popc(peers));
         }
         __syncthreads();
-        if (warp == 0) {
-            // lane j owns bins 255-8j .. 248-8j (descending)
-            uint32_t c[8], tot = 0;
+        // lane j owns bins 255-8j .. 248-8j (descending)
+        uint32_t c[8], tot = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            c[i] = hist[pass][255 - 8 * lane - i];
+            tot += c[i];
+        }
+        uint32_t incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const uint32_t excl = incl - tot;
+        uint32_t found = 0;   // (bin << 16) | (bin count << 0 ... ) packed below
+        uint32_t bin = 0, rem_in_bin = 0, bin_count = 0;
+        if (excl < remaining && remaining <= incl) {   // exactly one lane
+            uint32_t above = excl;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                c[i] = hist[255 - 8 * lane - i];
-                tot += c[i];
-            }
-            uint32_t incl = tot;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            const uint32_t excl = incl - tot;
-            if (excl < remaining && remaining <= incl) {   // exactly one lane
-                uint32_t above = excl;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (above < remaining && remaining <= above + c[i]) {
-                        sh_bin = 255 - 8 * lane - i;
-                        sh_remaining = remaining - above;
-                    }
-                    above += c[i];
+                if (above < remaining && remaining <= above + c[i]) {
+                    bin = 255 - 8 * lane - i;
+                    rem_in_bin = remaining - above;
+                    bin_count = c[i];
+                    found = 1;
                 }
+                above += c[i];
             }
         }
-        __syncthreads();
-        prefix |= sh_bin << shift;
+        const uint32_t src = __ffs(__ballot_sync(0xffffffffu, found != 0)) - 1;
+        bin = __shfl_sync(0xffffffffu, bin, src);
+        rem_in_bin = __shfl_sync(0xffffffffu, rem_in_bin, src);
+        bin_count = __shfl_sync(0xffffffffu, bin_count, src);
+        prefix |= bin << shift;
         mask |= 0xFFu << shift;
-        remaining = sh_remaining;
-        __syncthreads();
+        remaining = rem_in_bin;
+        SEL_STAMP(14 + pass);
+        if (remaining == bin_count) break;   // the whole boundary bin is kept: lower digits cannot matter
     }
-    const uint32_t thr = prefix;          // N-th largest key
-    const uint32_t take_eq = remaining;   // how many keys equal to thr are kept (smallest indices first)
+    // keys whose masked part exceeds the prefix are kept; of those equal to it, the first `remaining` in
+    // index order (all of them after an early stop)
+    SEL_STAMP(7);
+    const uint32_t thr = prefix;          // N-th largest key (its bits under the mask)
+    const uint32_t take_eq = remaining;   // how many keys equal to thr under the mask are kept (smallest indices first)
 
     // ascending compaction
     uint32_t base_sel = 0, base_eq = 0;
     for (int c0 = 0; c0 < nb; c0 += kThreads) {
-        const int b = c0 + tid;
-        const uint32_t k = b < nb ? keys_all[b] : 0u;
-        const bool gt = b < nb && k > thr;
-        const bool eq = b < nb && k == thr;
+        const int bb = c0 + tid;
+        const uint32_t k = bb < nb ? (keys_all[bb] & mask) : 0u;
+        const bool gt = bb < nb && k > thr;
+        const bool eq = bb < nb && k == thr;
         const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
-        if (lane == 0) warp_eq[warp] = __popc(eq_ballot);
-        __syncthreads();
-        uint32_t eq_before = base_eq, eq_total = 0;
-        for (int w = 0; w < kWarps; ++w) {
-            if (w < warp) eq_before += warp_eq[w];
-            eq_total += warp_eq[w];
+        const uint32_t gt_ballot = __ballot_sync(0xffffffffu, gt);
+        if (lane == 0) {
+            warp_eq[warp] = __popc(eq_ballot);
+            warp_sel[warp] = __popc(gt_ballot);
         }
-        const uint32_t eq_rank = eq_before + __popc(eq_ballot & ((1u << lane) - 1u));
+        __syncthreads();
+        uint32_t eq_before = base_eq, eq_total = 0, gt_before = 0, gt_total = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const uint32_t e = warp_eq[w], g = warp_sel[w];
+            if (w < warp) eq_before += e, gt_before += g;
+            eq_total += e, gt_total += g;
+        }
+        // kept ties are the first take_eq in index order
+        const uint32_t lt = (1u << lane) - 1u;
+        const uint32_t eq_rank = eq_before + __popc(eq_ballot & lt);
         const bool sel = gt || (eq && eq_rank < take_eq);
-        const uint32_t sel_ballot = __ballot_sync(0xffffffffu, sel);
-        if (lane == 0) warp_sel[warp] = __popc(sel_ballot);
-        __syncthreads();
-        uint32_t sel_before = base_sel, sel_total = 0;
-        for (int w = 0; w < kWarps; ++w) {
-            if (w < warp) sel_before += warp_sel[w];
-            sel_total += warp_sel[w];
-        }
-        if (sel) out[sel_before + __popc(sel_ballot & ((1u << lane) - 1u))] = b;
-        base_sel += sel_total;
+        // position = kept entries before this one = greater keys before + kept ties before
+        const uint32_t eq_kept_before = min(eq_rank, take_eq) - min(base_eq, take_eq);   // kept ties before, this chunk
+        if (sel) out[base_sel + gt_before + __popc(gt_ballot & lt) + eq_kept_before] = bb;
+        base_sel += gt_total + min(base_eq + eq_total, take_eq) - min(base_eq, take_eq);
         base_eq += eq_total;
         __syncthreads();
     }
     if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
+    SEL_STAMP(8);
 }
 
 __global__ void copy_selection_kernel(const int32_t *__restrict__ prev_idx, const int32_t *__restrict__ prev_cnt,
@@ -265,7 +353,7 @@ extern "C" sv_status sv_select_blocks(const sv_geom *geom, const void *q, const 
     p.T = geom->n_draft, p.Hq = geom->n_q_heads, p.Hkv = geom->n_kv_heads, p.B = geom->block_size;
     p.NBmax = geom->max_blocks, p.n_sink = n_sink, p.n_local = n_local, p.max_sel = max_sel, p.chunk = chunk;
 
-    const size_t smem = (size_t)(CL + 1) * chunk * sizeof(uint32_t);
+    const size_t smem = (size_t)CL * chunk * sizeof(uint32_t);
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SV_ERR_CUDA;

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "sv.h"
 
@@ -44,7 +45,7 @@ inline sv_status check_kv(const sv_geom *g, const sv_kv *kv, bool need_v)
 inline void pdl_attribute(cudaLaunchAttribute *attr)
 {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;
 }
 
 inline sv_status launch_status()

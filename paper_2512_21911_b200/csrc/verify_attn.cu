@@ -25,7 +25,6 @@
 
 #include <cstdlib>
 #include <mutex>
-#include <unordered_map>
 
 #include "attn_common.cuh"
 #include "sv_host.h"
@@ -571,25 +570,25 @@ EncodeTiledFn encode_fn()
 }
 
 // Tensor map over a pool viewed as a 2-D bf16 matrix [n_pages*Hkv*B rows][128 cols]; box = 64 rows x 64 cols
-// (128 bytes wide, 128-byte swizzle).  Encoding costs microseconds of host time, so maps are cached per pool.
+// (128 bytes wide, 128-byte swizzle).  Encoding costs microseconds of host time, so maps are kept in a
+// small fixed table keyed by (pool, rows) (no heap use; a full table is overwritten round-robin).
 bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
 {
-    struct Key {
-        const void *p;
+    struct Entry {
+        const void *pool;
         int64_t rows;
-        bool operator==(const Key &o) const { return p == o.p && rows == o.rows; }
+        CUtensorMap map;
     };
-    struct Hash {
-        size_t operator()(const Key &k) const { return std::hash<const void *>()(k.p) ^ (size_t)k.rows * 0x9E3779B97F4A7C15ull; }
-    };
+    constexpr int kEntries = 256;
+    static Entry table[kEntries];
+    static int used = 0, next = 0;
     static std::mutex mu;
-    static std::unordered_map<Key, CUtensorMap, Hash> cache;
     std::lock_guard<std::mutex> lock(mu);
-    auto it = cache.find(Key{pool, n_rows});
-    if (it != cache.end()) {
-        *out = it->second;
-        return true;
-    }
+    for (int i = 0; i < used; ++i)
+        if (table[i].pool == pool && table[i].rows == n_rows) {
+            *out = table[i].map;
+            return true;
+        }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {128, (cuuint64_t)n_rows};
@@ -601,8 +600,10 @@ bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
-    if (cache.size() > 4096) cache.clear();
-    cache.emplace(Key{pool, n_rows}, tm);
+    const int slot = used < kEntries ? used++ : (next++ % kEntries);
+    table[slot].pool = pool;
+    table[slot].rows = n_rows;
+    table[slot].map = tm;
     *out = tm;
     return true;
 }
