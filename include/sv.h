@@ -50,7 +50,8 @@ typedef enum {
     SV_ERR_BUDGET = 4,      /* n_sink + n_local exceeds max_sel */
     SV_ERR_WORKSPACE = 5,   /* workspace_bytes is smaller than sv_workspace_bytes() */
     SV_ERR_UNSUPPORTED = 6, /* head_dim != 128, block_size not 64/128, more than 128 query rows per KV head ... */
-    SV_ERR_CUDA = 7         /* a CUDA call or kernel launch failed */
+    SV_ERR_CUDA = 7,        /* a CUDA call or kernel launch failed */
+    SV_ERR_SCRATCH_LIMIT = 8 /* sv_verify_attn_noalloc: the problem needs more scratch than the built-in buffer holds */
 } sv_status;
 
 /* Static, human-readable text for a status code. */
@@ -168,6 +169,35 @@ SV_API sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv 
                          const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
                          const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
                          void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
+
+/*
+ * sv_verify_attn for callers that cannot provide or allocate a workspace.  (The paper has no
+ * counterpart: this is a packaging variant of sv_verify_attn, not another operation.)
+ *
+ * Some callers have no way to obtain device scratch at the point where they need the attention: a
+ * serving process that handed every byte of HBM to its KV-cache pool at start-up, so that a late
+ * cudaMalloc fails; a plug-in that runs inside somebody else's allocator and may not call cudaMalloc /
+ * cudaFree (both may synchronise the whole device); a latency-critical decode loop that must not risk
+ * an allocation stall.  For them the split-KV partials live in a buffer that is part of the library
+ * image: a file-scope device array of SV_NOALLOC_SCRATCH_BYTES bytes.  Every GPU that loads the library
+ * holds that array from the first CUDA call of the process until exit.
+ *
+ * Same arguments and results as sv_verify_attn, minus workspace / workspace_bytes.  The call allocates
+ * nothing on the device or through any allocating library routine.  Differences:
+ *   - sizes: if sv_workspace_bytes(geom, max_sel) exceeds SV_NOALLOC_SCRATCH_BYTES the call launches
+ *     nothing and returns SV_ERR_SCRATCH_LIMIT (use sv_verify_attn with your own workspace instead);
+ *   - set-up: the first call on each device looks up the device address of the built-in array (with
+ *     that device current) and keeps it; make that first call outside any stream capture;
+ *   - sharing: all calls on a device use the same array, and it keeps whatever the last call left in
+ *     it.  Nothing in it has to start at zero (every partial is written before it is read), but two
+ *     calls that overlap on the GPU (different streams, or a second process thread) race on it and
+ *     corrupt each other's results: serialise them, or use sv_verify_attn with separate workspaces.
+ */
+#define SV_NOALLOC_SCRATCH_BYTES (4u * 1024u * 1024u)
+SV_API sv_status sv_verify_attn_noalloc(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                                        const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                                        const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out,
+                                        float *lse, int32_t *status_word, void *stream);
 
 /* Number of KV splits (CTAs per (sequence, KV head)) sv_verify_attn uses for this geometry. */
 SV_API int32_t sv_verify_attn_splits(const sv_geom *geom, int32_t max_sel);

@@ -18,10 +18,11 @@ LIB_PATH = os.path.join(_HERE, "libsv.so")
 SV_OK = 0
 SV_TAIL_BLOCK = -1   # sv_block_reps(block_begin=SV_TAIL_BLOCK): refresh only each sequence's last block
 STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIGN", 4: "SV_ERR_BUDGET",
-                5: "SV_ERR_WORKSPACE", 6: "SV_ERR_UNSUPPORTED", 7: "SV_ERR_CUDA"}
+                5: "SV_ERR_WORKSPACE", 6: "SV_ERR_UNSUPPORTED", 7: "SV_ERR_CUDA", 8: "SV_ERR_SCRATCH_LIMIT"}
+SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
 EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
-           "sv_verify_attn", "sv_verify_attn_splits")
+           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc")
 
 
 class SvError(RuntimeError):
@@ -63,6 +64,8 @@ def _load() -> ctypes.CDLL:
     lib.sv_select_blocks.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
     lib.sv_verify_attn.restype = ctypes.c_int
     lib.sv_verify_attn.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
+    lib.sv_verify_attn_noalloc.restype = ctypes.c_int
+    lib.sv_verify_attn_noalloc.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     return lib
 
 
@@ -146,3 +149,22 @@ def sv_verify_attn(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_id
                                _ptr(sel_cnt, torch.int32, "sel_cnt"), max_sel, float(softmax_scale),
                                _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"), ws_ptr, ws_bytes,
                                _ptr(status_word, torch.int32, "status_word"), _stream(stream)), "sv_verify_attn")
+
+
+def sv_verify_attn_noalloc(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=None,
+                           softmax_scale: float = 0.0, status_word=None, stream=None) -> None:
+    """sv_verify_attn without a caller workspace: the split-KV partials go to the scratch array built into
+    the library (SV_NOALLOC_SCRATCH_BYTES).  For callers that cannot allocate device memory where they
+    need the attention -- a server whose HBM is fully reserved by its KV-cache pool, code that runs under
+    another component's allocator.  Nothing is allocated here, by torch or otherwise: only the caller's
+    input and output tensors are passed through.  Problems whose partials do not fit raise
+    SvError(SV_ERR_SCRATCH_LIMIT).  All calls on a device share that array, so calls that may overlap on
+    the GPU must be serialised by the caller; make the first call on a device outside any stream capture."""
+    max_sel = int(sel_idx.shape[-1]) if sel_idx is not None else int(geom.max_blocks)
+    _check(_lib.sv_verify_attn_noalloc(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), ctypes.byref(kv),
+                                       _ptr(draft_k, torch.bfloat16, "draft_k"),
+                                       _ptr(draft_v, torch.bfloat16, "draft_v"), _ptr(parent, torch.int32, "parent"),
+                                       _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                       max_sel, float(softmax_scale), _ptr(out, torch.bfloat16, "out"),
+                                       _ptr(lse, torch.float32, "lse"), _ptr(status_word, torch.int32, "status_word"),
+                                       _stream(stream)), "sv_verify_attn_noalloc")

@@ -14,6 +14,7 @@ extern "C" const char *sv_strerror(sv_status st)
         case SV_ERR_WORKSPACE: return "workspace too small";
         case SV_ERR_UNSUPPORTED: return "unsupported geometry";
         case SV_ERR_CUDA: return "CUDA call or kernel launch failed";
+        case SV_ERR_SCRATCH_LIMIT: return "the problem needs more scratch than the built-in buffer of sv_verify_attn_noalloc holds";
     }
     return "unknown status";
 }

@@ -758,3 +758,52 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
     }
     return SV_OK;
 }
+
+// ---------------------------------------------------------------------- sv_verify_attn_noalloc
+//
+// Built-in scratch for callers that cannot allocate (see sv.h).  The array below is device memory that
+// belongs to the library image.  In host code its name is only a handle for the runtime, not an address
+// a kernel could use, so the device address is looked up once per device with cudaGetSymbolAddress
+// (with that device current) and handed to the ordinary entry point as its workspace.
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SV_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+
+// Device address of g_noalloc_scratch on the current device, or nullptr if the look-up fails.
+void *noalloc_scratch_address()
+{
+    constexpr int kMaxDevices = 64;
+    static void *addr[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess) {
+            cudaGetLastError();   // leave no sticky error behind
+            return nullptr;
+        }
+        addr[dev] = p;
+    }
+    return addr[dev];
+}
+
+}  // namespace
+
+extern "C" sv_status sv_verify_attn_noalloc(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                                            const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                                            const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out,
+                                            float *lse, int32_t *status_word, void *stream)
+{
+    const sv_status st = svh::check_geom(geom);
+    if (st != SV_OK) return st;
+    const int32_t eff_sel = sel_idx ? max_sel : geom->max_blocks;
+    if (eff_sel < 1) return SV_ERR_SHAPE;
+    if (sv_workspace_bytes(geom, eff_sel) > (size_t)SV_NOALLOC_SCRATCH_BYTES) return SV_ERR_SCRATCH_LIMIT;
+    void *scratch = noalloc_scratch_address();
+    if (!scratch) return SV_ERR_CUDA;
+    return sv_verify_attn(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
+                          scratch, (size_t)SV_NOALLOC_SCRATCH_BYTES, status_word, stream);
+}
