@@ -372,6 +372,88 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """--sweep: single-layer sparse vs dense verification over context x budget fraction x draft length
+    (32 q / 8 kv heads, head_dim 128, block 64, batch 1).  Timing only (parity of these shapes is covered by
+    the tests): K/V are seeded device-side N(0, 1/128) tensors, the block list comes from sv_select_blocks.
+    Every point rotates over enough independent KV replicas that at least 256 MiB is gathered between two
+    uses of the same replica, so nothing is found in L2.  One JSON line per point on stdout."""
+    import torch
+
+    import paper_2512_21911_b200 as sv
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peaks()
+    stream = torch.cuda.Stream(device=dev)
+    Hq, Hkv, D, B = 32, 8, 128, 64
+    for L in (8192, 32768, 131072):
+        NB = L // B
+        n_rep = max(2, min(16, (4 << 30) // (2 * NB * Hkv * B * D * 2)))
+        gen = torch.Generator(device=dev).manual_seed(1004 + L)
+        pools = [(torch.randn((NB, Hkv, B, D), generator=gen, device=dev, dtype=torch.float32).mul_(128 ** -0.5).to(torch.bfloat16),
+                  torch.randn((NB, Hkv, B, D), generator=gen, device=dev, dtype=torch.float32).mul_(128 ** -0.5).to(torch.bfloat16))
+                 for _ in range(n_rep)]
+        bt = torch.randperm(NB, generator=gen, device=dev).to(torch.int32).view(1, NB)
+        sl = torch.tensor([L], dtype=torch.int32, device=dev)
+        for T in (1, 4, 8, 16):
+            geom = sv.make_geom(1, Hq, Hkv, D, B, NB, T)
+            q = torch.randn((1, T, Hq, D), generator=gen, device=dev).mul_(128 ** -0.5).to(torch.bfloat16)
+            dk = torch.randn((1, T, Hkv, D), generator=gen, device=dev).mul_(128 ** -0.5).to(torch.bfloat16)
+            dv = torch.randn((1, T, Hkv, D), generator=gen, device=dev).mul_(128 ** -0.5).to(torch.bfloat16)
+            out = torch.zeros_like(q)
+            kvs = [sv.make_kv(k, v, bt, sl) for k, v in pools]
+            reps = [torch.zeros((1, Hkv, NB, D), device=dev) for _ in pools]
+            for kv, r in zip(kvs, reps):
+                sv.sv_block_reps(geom, kv, r)
+            for frac in (1 / 32, 1 / 16, 1 / 8, 1 / 4, 1.0):
+                dense = frac == 1.0
+                N = NB if dense else max(2, int(round(NB * frac)))
+                idx = torch.zeros((1, Hkv, N), dtype=torch.int32, device=dev)
+                cnt = torch.zeros((1, Hkv), dtype=torch.int32, device=dev)
+                bud = torch.tensor([N], dtype=torch.int32, device=dev)
+                ws = torch.zeros(max(16, sv.sv_workspace_bytes(geom, N)), dtype=torch.uint8, device=dev)
+                if not dense:
+                    sv.sv_select_blocks(geom, q, reps[0], sl, bud, 1, 1, idx, cnt)
+
+                def attn_all():
+                    for kv in kvs:
+                        sv.sv_verify_attn(geom, q, kv, dk, dv, None, None if dense else idx, None if dense else cnt, out,
+                                          workspace=ws)
+
+                def both_all():
+                    for kv, r in zip(kvs, reps):
+                        sv.sv_select_blocks(geom, q, r, sl, bud, 1, 1, idx, cnt)
+                        sv.sv_verify_attn(geom, q, kv, dk, dv, None, idx, cnt, out, workspace=ws)
+
+                def timed(fn, iters=20):
+                    with torch.cuda.stream(stream):
+                        fn(); fn()
+                        stream.synchronize()
+                        g = torch.cuda.CUDAGraph()
+                        with torch.cuda.graph(g, stream=stream):
+                            fn()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        for _ in range(3):
+                            g.replay()
+                        e0.record(stream)
+                        for _ in range(iters):
+                            g.replay()
+                        e1.record(stream)
+                        stream.synchronize()
+                    return e0.elapsed_time(e1) * 1e3 / iters / len(kvs)
+
+                us_attn = timed(attn_all)
+                us_both = None if dense else timed(both_all)
+                kv_bytes = Hkv * N * B * 2 * D * 2
+                print(json.dumps({"context": L, "budget_frac": "dense" if dense else round(frac, 5), "n_draft": T,
+                                  "kept_blocks": N, "gathered_kv_mib": kv_bytes / 2 ** 20, "replicas": len(kvs),
+                                  "attn_us": round(us_attn, 2), "select_plus_attn_us": None if dense else round(us_both, 2),
+                                  "kv_gbs": round(kv_bytes / us_attn / 1e3, 1),
+                                  "frac_of_measured_peak": round(kv_bytes / us_attn / 1e3 / peak, 3),
+                                  "pct_of_8tbs": round(kv_bytes / us_attn / 1e3 / 80.0, 1)}), flush=True)
+        del pools
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -382,8 +464,12 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: run a shorter stack (default: all 32)")
     ap.add_argument("--only-step", action="store_true",
                     help="profiling aid: time only the main step graph (no reuse / dense / attention-only / e2e passes)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark line: sparse vs dense latency over context x budget x draft length")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
