@@ -117,6 +117,14 @@ def workload_config(w, geom):
             "l2": "inputs larger than L2: every layer has its own 128 MiB K/V pool; a step gathers 512 MiB out of 4 GiB"}
 
 
+def aggregate_over_ranks(ms_local, world, all_reduce_max):
+    """Whole-job numbers from per-rank step times: N GPUs run N independent replicas of the workload
+    (no collective on the data path), the job's step time is the slowest rank's, and the job verifies
+    N times as many layers per step.  Returns (ms_per_step, layers_multiplier)."""
+    ms = all_reduce_max(ms_local) if world > 1 else ms_local
+    return ms, world
+
+
 # ----------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -317,7 +325,8 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e = (allmax(x) for x in (ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e))
+    ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e = (aggregate_over_ranks(x, world, allmax)[0]
+                                                    for x in (ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e))
 
     # algorithmic bytes of one sv_verify_attn launch (K+V of the kept tokens and draft tokens, Q in, O out)
     S, T, Hq, Hkv, D, B, N = w.n_seq, w.n_draft, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, w.budget_blocks

@@ -384,3 +384,18 @@ def test_stacked_tail_refresh_equals_per_layer(sv):
         for s in range(3):
             nb = int(geom["n_blocks"][s])
             np.testing.assert_allclose(full[l, s, :, :nb].cpu().numpy(), ref[s, :, :nb], rtol=1e-5, atol=1e-6)
+
+
+def test_mma_sync_attention_path_stays_green():
+    """The older bf16 mma.sync attention kernel is kept selectable (SV_ATTN_IMPL=mma, read once per
+    process) for A/B runs against the tcgen05 kernel; run the small parity cases through it in a child."""
+    import os
+    import subprocess
+    import sys
+    if os.environ.get("SV_ATTN_IMPL", "").startswith("m"):
+        pytest.skip("already running on the mma.sync path")
+    env = dict(os.environ, SV_ATTN_IMPL="mma")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-q", "-x", "-m", "gpu", "-k",
+                        "pipeline_parity_small or more_splits or empty_prefix"], env=env, capture_output=True, text=True,
+                       cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
