@@ -129,6 +129,11 @@ SMALL = {
     "cfg3_small": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(5000, 9000), budget_blocks=11, planted=3),
     "rows4": si.shrink(si.WORKLOADS["cfg1"], seq_len=(2048, 2048), budget_blocks=8, n_draft=1, n_layers=1),
     "t32": si.shrink(si.WORKLOADS["cfg0"], seq_len=(1000, 1000), budget_blocks=5, n_draft=32, tree=True, planted=2),
+    # multi-head attention (G = 1), a wide GQA group (G = 16, 128 rows), block 128 whose tail holds <= 64 tokens
+    "mha": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=4, seq_len=(1200, 1200), budget_blocks=6, planted=2),
+    "g16": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1500, 1500), budget_blocks=6, n_draft=8, planted=2),
+    "b128_short_tail": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(128 * 9 + 30, 128 * 9 + 30), n_q_heads=16, n_kv_heads=4,
+                                 budget_blocks=5, n_draft=6, planted=2),
 }
 
 
