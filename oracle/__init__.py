@@ -197,3 +197,20 @@ def budget_blocks(L, L0, rho, B, n_sink=0, n_local=0) -> int:
     lib.svo_budget_blocks.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_double, ctypes.c_int,
                                       ctypes.c_int, ctypes.c_int]
     return int(lib.svo_budget_blocks(int(L), int(L0), float(rho), int(B), int(n_sink), int(n_local)))
+
+
+def kv_append(k_pool, v_pool, block_table, seq_lens, draft_k, draft_v, accept_idx, n_accept, reps=None):
+    """Commit accepted draft tokens to the paged cache (in place) and refresh the representatives of the
+    blocks that grew.  accept_idx int32 [S][A], n_accept int32 [S].  Returns the new lengths (int32 [S])."""
+    _, Hkv, B, D = k_pool.shape
+    S, NBmax = block_table.shape
+    T = draft_k.shape[1]
+    A = accept_idx.shape[1]
+    out = np.zeros(S, dtype=np.int32)
+    rc = _load().svo_kv_append(S, T, Hkv, D, B, NBmax, _p(k_pool, np.uint16), _p(v_pool, np.uint16),
+                               _p(block_table, np.int32), _p(seq_lens, np.int32), _p(draft_k, np.uint16),
+                               _p(draft_v, np.uint16), _p(np.ascontiguousarray(accept_idx), np.int32),
+                               _p(np.ascontiguousarray(n_accept), np.int32), A, _p(out, np.int32), _p(reps, np.float64))
+    if rc:
+        raise ValueError(f"kv_append: bad argument ({rc})")
+    return out

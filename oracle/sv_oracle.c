@@ -24,6 +24,9 @@
  *       library scaled-dot-product attention with an explicit mask; prefix
  *       truncation; softmax weights sum to one; log-sum-exp split merge.
  *   svo_budget_blocks : closed form of Eq. 6 and the sparsity column of Table 2.
+ *   svo_kv_append : the appended cache read back with numpy indexing equals old tokens followed by the
+ *       accepted rows; one call equals token-by-token calls; attention afterwards equals attention on a
+ *       cache built with the longer prefix.
  *   Approximation quality of sparse vs dense attention: parity unpinned (the
  *       paper bounds nothing; reported as information only).
  */
@@ -374,4 +377,52 @@ int svo_budget_blocks(int64_t L, int64_t L0, double rho, int B, int n_sink, int 
     if (n < forced) n = forced;
     if (n > nb) n = nb;
     return n;
+}
+
+/*
+ * Commit of accepted draft tokens (Section 2.1: the accepted prefix of the draft is kept, the rest
+ * discarded; Section 3.1: blocks are cut from the *current* KV cache).  For every sequence the K/V rows of
+ * the accepted draft tokens accept_idx[s][0 .. n_accept[s]) are appended, in that order, at positions
+ * L_s, L_s + 1, ... of the paged cache (the pages must already be in block_table), the length grows by
+ * n_accept[s], and the representatives of the blocks that received tokens are recomputed as in
+ * svo_block_reps.  Pools are modified in place; new lengths go to seq_lens_out.
+ */
+int svo_kv_append(int S, int T, int Hkv, int D, int B, int NBmax, uint16_t *k_pool, uint16_t *v_pool,
+                  const int32_t *block_table, const int32_t *seq_lens, const uint16_t *draft_k,
+                  const uint16_t *draft_v, const int32_t *accept_idx, const int32_t *n_accept, int max_accept,
+                  int32_t *seq_lens_out, double *reps)
+{
+    for (int s = 0; s < S; ++s) {
+        int64_t L = seq_lens[s];
+        int n = n_accept[s];
+        if (n < 0 || n > max_accept || (L + n + B - 1) / B > NBmax) return 1;
+        for (int a = 0; a < n; ++a) {
+            int j = accept_idx[(int64_t)s * max_accept + a];
+            if (j < 0 || j >= T) return 2;
+            int64_t t = L + a;
+            int64_t page = block_table[(int64_t)s * NBmax + t / B];
+            for (int h = 0; h < Hkv; ++h)
+                for (int d = 0; d < D; ++d) {
+                    int64_t dst = ((page * Hkv + h) * B + (t % B)) * D + d;
+                    int64_t src = (((int64_t)s * T + j) * Hkv + h) * D + d;
+                    k_pool[dst] = draft_k[src];
+                    v_pool[dst] = draft_v[src];
+                }
+        }
+        int64_t Ln = L + n;
+        seq_lens_out[s] = (int32_t)Ln;
+        if (n == 0 || !reps) continue;
+        for (int64_t b = L / B; b <= (Ln - 1) / B; ++b) {
+            int64_t t0 = b * B;
+            int64_t cnt = (Ln - t0 < B) ? (Ln - t0) : B;
+            for (int h = 0; h < Hkv; ++h)
+                for (int d = 0; d < D; ++d) {
+                    double sum = 0.0;
+                    for (int64_t t = t0; t < t0 + cnt; ++t)
+                        sum += kv_at(k_pool, block_table, s, h, t, d, Hkv, D, B, NBmax);
+                    reps[(((int64_t)s * Hkv + h) * NBmax + b) * D + d] = sum / (double)cnt;
+                }
+        }
+    }
+    return 0;
 }

@@ -431,3 +431,85 @@ def test_budget_reproduces_table2_sparsity_column():
             if n == name:
                 kept = oracle.budget_blocks(L, L0, 0.1, 1)
                 assert abs((1 - kept / L) - sa) < 0.035, (name, L0, 1 - kept / L, sa)
+
+
+# --------------------------------------------------------------------------- commit of accepted tokens
+
+def _append_case(seed=41):
+    c = _tiny_case(S=2, Hq=4, Hkv=2, D=8, B=4, T=5, lens=(9, 6), seed=seed)
+    # room for growth: table of 5 blocks per sequence, fresh pages for the blocks that will be entered
+    S, NB = 2, 5
+    n_pages = S * NB + 1
+    g = np.random.default_rng(seed)
+    perm = g.permutation(n_pages)
+    bt = perm[:S * NB].reshape(S, NB).astype(np.int32)
+    k_pool = _bits(g.standard_normal((n_pages, 2, 4, 8)))
+    v_pool = _bits(g.standard_normal((n_pages, 2, 4, 8)))
+    c.update(block_table=bt, k_pool=k_pool, v_pool=v_pool, n_blocks=(c["seq_lens"] + 3) // 4)
+    return c
+
+
+def test_kv_append_places_rows_and_updates_lengths_and_reps():
+    c = _append_case()
+    accept = np.array([[0, 2, 3, 0, 0], [0, 1, 0, 0, 0]], np.int32)     # sequence 0 keeps drafts 0,2,3; sequence 1 keeps 0,1
+    n_acc = np.array([3, 2], np.int32)
+    old_k = [_gather_tokens(c["k_pool"], c["block_table"], s, h, int(c["seq_lens"][s]), 4) for s in range(2) for h in range(2)]
+    old_v = [_gather_tokens(c["v_pool"], c["block_table"], s, h, int(c["seq_lens"][s]), 4) for s in range(2) for h in range(2)]
+    reps = oracle.block_reps(c["k_pool"], c["block_table"], c["seq_lens"])
+    untouched = reps.copy()
+    new_len = oracle.kv_append(c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"], c["draft_v"],
+                               accept, n_acc, reps)
+    assert new_len.tolist() == [12, 8]
+    i = 0
+    for s in range(2):
+        for h in range(2):
+            want_k = np.concatenate([old_k[i], si.bf16_bits_to_f64(c["draft_k"][s, accept[s, :n_acc[s]], h])])
+            want_v = np.concatenate([old_v[i], si.bf16_bits_to_f64(c["draft_v"][s, accept[s, :n_acc[s]], h])])
+            np.testing.assert_array_equal(_gather_tokens(c["k_pool"], c["block_table"], s, h, int(new_len[s]), 4), want_k)
+            np.testing.assert_array_equal(_gather_tokens(c["v_pool"], c["block_table"], s, h, int(new_len[s]), 4), want_v)
+            for b in range((int(new_len[s]) + 3) // 4):        # every block's representative is the mean of its tokens
+                np.testing.assert_allclose(reps[s, h, b], want_k[4 * b:4 * b + 4].mean(axis=0), rtol=0, atol=1e-14)
+            i += 1
+    # blocks that received nothing keep their representative bit for bit
+    np.testing.assert_array_equal(reps[0, :, :2], untouched[0, :, :2])
+    np.testing.assert_array_equal(reps[1, :, :1], untouched[1, :, :1])
+
+
+def test_kv_append_at_once_equals_token_by_token_and_zero_accept_is_a_no_op():
+    a = _append_case(43)
+    b = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in a.items()}
+    accept = np.array([[1, 4, 2, 0, 0], [3, 0, 0, 0, 0]], np.int32)
+    n_acc = np.array([3, 0], np.int32)
+    ra = oracle.block_reps(a["k_pool"], a["block_table"], a["seq_lens"])
+    rb = ra.copy()
+    la = oracle.kv_append(a["k_pool"], a["v_pool"], a["block_table"], a["seq_lens"], a["draft_k"], a["draft_v"], accept, n_acc, ra)
+    lens = b["seq_lens"].copy()
+    for step in range(3):
+        lens = oracle.kv_append(b["k_pool"], b["v_pool"], b["block_table"], lens, b["draft_k"], b["draft_v"],
+                                accept[:, step:step + 1].copy(), np.array([1, 0], np.int32), rb)
+    assert la.tolist() == lens.tolist() == [12, 6]
+    np.testing.assert_array_equal(a["k_pool"], b["k_pool"])
+    np.testing.assert_array_equal(a["v_pool"], b["v_pool"])
+    np.testing.assert_allclose(ra, rb, rtol=0, atol=1e-14)
+    with pytest.raises(ValueError):
+        oracle.kv_append(a["k_pool"], a["v_pool"], a["block_table"], la, a["draft_k"], a["draft_v"],
+                         np.array([[7], [0]], np.int32), np.array([1, 0], np.int32), ra)     # draft index out of range
+
+
+def test_attention_after_append_sees_the_committed_tokens():
+    """After committing draft tokens 0..2 of a chain, the next step's dense attention over the cache equals
+    attention over a prefix that already contained them."""
+    c = _append_case(47)
+    accept = np.tile(np.arange(5, dtype=np.int32), (2, 1))
+    n_acc = np.array([3, 3], np.int32)
+    new_len = oracle.kv_append(c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"], c["draft_v"],
+                               accept, n_acc, None)
+    # verification of draft token 3 before the commit: it saw the old prefix and drafts 0..3 (chain);
+    # after the commit the same query with a single draft token (the old draft 3) sees prefix' + itself
+    q1 = c["q"][:, 3:4].copy()
+    dk1, dv1 = c["draft_k"][:, 3:4].copy(), c["draft_v"][:, 3:4].copy()
+    after, _ = oracle.dense_verify_attn(q1, c["k_pool"], c["v_pool"], c["block_table"], new_len, dk1, dv1, None)
+    c0 = _append_case(47)
+    before, _ = oracle.dense_verify_attn(c0["q"], c0["k_pool"], c0["v_pool"], c0["block_table"], c0["seq_lens"],
+                                         c0["draft_k"], c0["draft_v"], None)
+    np.testing.assert_allclose(after[:, 0], before[:, 3], rtol=0, atol=1e-12)
