@@ -13,6 +13,8 @@
  *                     last few; or reuse the previous layer's set  (Eq. 5, Eq. 9)
  *   sv_verify_attn    attention of all draft tokens over the kept blocks
  *                     and the draft tokens' own K/V                       (Fig. 1)
+ *   sv_kv_append      commit of the accepted draft tokens to the cache, with
+ *                     the representatives of the grown blocks refreshed (Section 2.1)
  *
  * Conventions for every entry point
  *   - "dev" pointers are device memory owned by the caller; the library never
@@ -111,6 +113,26 @@ SV_API size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel);
 #define SV_TAIL_BLOCK (-1)
 SV_API sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
                         float *reps, void *stream);
+
+/*
+ * Commit of the accepted draft tokens (Section 2.1: the accepted prefix of the draft is kept; Section 3.1:
+ * blocks are cut from the current KV cache).  For every sequence s the K/V rows of the draft tokens
+ * accept_idx[s][0 .. n_accept[s]) are appended, in that order, at positions L_s, L_s + 1, ... of the paged
+ * cache, seq_lens_out[s] = L_s + n_accept[s], and the representatives of the (at most two) blocks that
+ * received tokens are recomputed exactly as sv_block_reps would.  The pages of blocks that are entered
+ * must already be listed in block_table; tokens that would fall behind the last page of the table are
+ * dropped (n_accept is clamped).  Replaces "append + sv_block_reps(SV_TAIL_BLOCK)" in a decoding loop.
+ *   k_pool/v_pool   dev bf16 [n_pages][Hkv][B][D], modified in place
+ *   seq_lens        dev int32 [S] lengths before the commit; seq_lens_out dev int32 [S], a different buffer
+ *   draft_k/draft_v dev bf16 [S][T][Hkv][D] of the step just verified
+ *   accept_idx      dev int32 [S][max_accept] draft-token indices (0..T-1) in acceptance order
+ *   n_accept        dev int32 [S], 0..max_accept; max_accept <= T
+ *   reps            dev fp32 [S][Hkv][NBmax][D] or NULL (no representative update)
+ */
+SV_API sv_status sv_kv_append(const sv_geom *geom, void *k_pool, void *v_pool, int32_t n_pages,
+                              const int32_t *block_table, const int32_t *seq_lens, const void *draft_k,
+                              const void *draft_v, const int32_t *accept_idx, const int32_t *n_accept,
+                              int32_t max_accept, int32_t *seq_lens_out, float *reps, void *stream);
 
 /*
  * Block selection (Section 3.1; Section 2.2: only the first draft token

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIG
 SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
 EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
-           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc")
+           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append")
 
 
 class SvError(RuntimeError):
@@ -64,6 +64,8 @@ def _load() -> ctypes.CDLL:
     lib.sv_select_blocks.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
     lib.sv_verify_attn.restype = ctypes.c_int
     lib.sv_verify_attn.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
+    lib.sv_kv_append.restype = ctypes.c_int
+    lib.sv_kv_append.argtypes = [gp, vp, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
     lib.sv_verify_attn_noalloc.restype = ctypes.c_int
     lib.sv_verify_attn_noalloc.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     return lib
@@ -168,3 +170,16 @@ def sv_verify_attn_noalloc(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent
                                        max_sel, float(softmax_scale), _ptr(out, torch.bfloat16, "out"),
                                        _ptr(lse, torch.float32, "lse"), _ptr(status_word, torch.int32, "status_word"),
                                        _stream(stream)), "sv_verify_attn_noalloc")
+
+
+def sv_kv_append(geom: sv_geom, k_pool, v_pool, block_table, seq_lens, draft_k, draft_v, accept_idx, n_accept,
+                 seq_lens_out, reps=None, stream=None) -> None:
+    """Commit accepted draft tokens to the paged cache (pools modified in place), write the new lengths to
+    seq_lens_out (a different tensor than seq_lens) and refresh the representatives of the grown blocks."""
+    _check(_lib.sv_kv_append(ctypes.byref(geom), _ptr(k_pool, torch.bfloat16, "k_pool"), _ptr(v_pool, torch.bfloat16, "v_pool"),
+                             int(k_pool.shape[0]), _ptr(block_table, torch.int32, "block_table"),
+                             _ptr(seq_lens, torch.int32, "seq_lens"), _ptr(draft_k, torch.bfloat16, "draft_k"),
+                             _ptr(draft_v, torch.bfloat16, "draft_v"), _ptr(accept_idx, torch.int32, "accept_idx"),
+                             _ptr(n_accept, torch.int32, "n_accept"), int(accept_idx.shape[-1]),
+                             _ptr(seq_lens_out, torch.int32, "seq_lens_out"), _ptr(reps, torch.float32, "reps"),
+                             _stream(stream)), "sv_kv_append")

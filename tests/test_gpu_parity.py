@@ -404,3 +404,64 @@ def test_mma_sync_attention_path_stays_green():
                         "pipeline_parity_small or more_splits or empty_prefix"], env=env, capture_output=True, text=True,
                        cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+@pytest.mark.parametrize("block", [64, 128])
+def test_kv_append_parity(sv, block):
+    """Commit of accepted draft tokens: pools and lengths bit-exact against the oracle, representatives of the
+    grown blocks equal to the oracle's (fp32 vs fp64) and bit-identical to a full sv_block_reps rebuild."""
+    base = SMALL["cfg2_small"] if block == 64 else SMALL["cfg3_small"]
+    w = si.shrink(base, n_draft=8)
+    geom = si.make_geometry(w)
+    c = si.make_layer(geom)
+    S, Hkv, T = w.n_seq, w.n_kv_heads, w.n_draft
+    g = np.random.default_rng(5)
+    # one more table column with fresh pages, so that sequences may enter a new block
+    extra = np.arange(c["n_pages"], c["n_pages"] + S, dtype=np.int32)
+    bt = np.concatenate([c["block_table"], np.zeros((S, 1), np.int32)], axis=1)
+    for s in range(S):
+        bt[s, c["n_blocks"][s]] = extra[s]
+    junk = si.f32_to_bf16_bits(g.standard_normal((S, Hkv, block, 128)).astype(np.float32))
+    k_pool = np.concatenate([c["k_pool"], junk]); v_pool = np.concatenate([c["v_pool"], junk[::-1].copy()])
+    lens = c["seq_lens"].copy()
+    lens[0] = (lens[0] // block) * block + block - 3          # 3 slots left: an 8-token commit crosses into the new block
+    lens[1] = (lens[1] // block) * block                      # exactly at a block boundary
+    n_acc = g.integers(0, T + 1, size=S).astype(np.int32)
+    n_acc[0], n_acc[1] = 8, 5
+    if S > 2:
+        n_acc[2] = 0
+    acc = np.stack([np.sort(g.choice(T, size=T, replace=False)) for _ in range(S)]).astype(np.int32)
+    NB = bt.shape[1]
+    geom_c = sv.make_geom(S, w.n_q_heads, Hkv, 128, block, NB, T)
+    kp, vp = bf16_dev(k_pool), bf16_dev(v_pool)
+    btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
+    dk, dv = bf16_dev(c["draft_k"]), bf16_dev(c["draft_v"])
+    kv = sv.make_kv(kp, vp, btd, sld)
+    reps = torch.zeros((S, Hkv, NB, 128), device="cuda")
+    sv.sv_block_reps(geom_c, kv, reps)
+    before = reps.clone()
+    new_len = torch.zeros_like(sld)
+    sv.sv_kv_append(geom_c, kp, vp, btd, sld, dk, dv, torch.from_numpy(acc).cuda(), torch.from_numpy(n_acc).cuda(), new_len, reps)
+    torch.cuda.synchronize()
+    # oracle on the same inputs
+    ko, vo = k_pool.copy(), v_pool.copy()
+    reps_o = oracle.block_reps(ko, bt, lens)
+    len_o = oracle.kv_append(ko, vo, bt, lens, c["draft_k"], c["draft_v"], acc, n_acc, reps_o)
+    np.testing.assert_array_equal(new_len.cpu().numpy(), len_o)
+    np.testing.assert_array_equal(kp.cpu().view(torch.int16).numpy().view(np.uint16), ko)
+    np.testing.assert_array_equal(vp.cpu().view(torch.int16).numpy().view(np.uint16), vo)
+    r = reps.cpu().numpy()
+    for s in range(S):
+        nbn = (int(len_o[s]) + block - 1) // block
+        np.testing.assert_allclose(r[s, :, :nbn], reps_o[s, :, :nbn], rtol=1e-5, atol=1e-6)
+        first = int(lens[s]) // block
+        assert torch.equal(reps[s, :, :first], before[s, :, :first])          # blocks that did not grow are untouched
+    rebuilt = torch.zeros_like(reps)
+    kv2 = sv.make_kv(kp, vp, btd, new_len)
+    sv.sv_block_reps(geom_c, kv2, rebuilt)
+    torch.cuda.synchronize()
+    for s in range(S):
+        nbn = (int(len_o[s]) + block - 1) // block
+        assert torch.equal(reps[s, :, :nbn], rebuilt[s, :, :nbn])
+    with pytest.raises(sv.SvError):
+        sv.sv_kv_append(geom_c, kp, vp, btd, sld, dk, dv, torch.from_numpy(acc).cuda(), torch.from_numpy(n_acc).cuda(), sld, reps)
