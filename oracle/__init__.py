@@ -214,3 +214,27 @@ def kv_append(k_pool, v_pool, block_table, seq_lens, draft_k, draft_v, accept_id
     if rc:
         raise ValueError(f"kv_append: bad argument ({rc})")
     return out
+
+
+def jaccard_adjacent(idx_all, cnt_all):
+    """Eq. 7 between adjacent layers.  idx_all int32 [layers][S][Hkv][max_sel], cnt_all int32 [layers][S][Hkv].
+    Returns (inter int32 [layers][S], union int32 [layers][S], J fp64 [layers]); J[0] = 0 by definition."""
+    n_layers, S, Hkv, max_sel = idx_all.shape
+    inter = np.zeros((n_layers, S), np.int32)
+    uni = np.zeros((n_layers, S), np.int32)
+    J = np.zeros(n_layers, np.float64)
+    rc = _load().svo_jaccard_adjacent(n_layers, S, Hkv, max_sel, _p(np.ascontiguousarray(idx_all), np.int32),
+                                      _p(np.ascontiguousarray(cnt_all), np.int32), _p(inter, np.int32), _p(uni, np.int32),
+                                      _p(J, np.float64))
+    assert rc == 0, rc
+    return inter, uni, J
+
+
+def pick_anchors(J, K):
+    """Eq. 8: the K layers least similar to their predecessor.  Returns a bool array [layers]."""
+    J = np.ascontiguousarray(J, dtype=np.float64)
+    anchors = np.zeros(J.shape[0], np.uint8)
+    rc = _load().svo_pick_anchors(J.shape[0], _p(J, np.float64), int(K), _p(anchors, np.uint8))
+    if rc:
+        raise ValueError("K must be between 1 and the number of layers")
+    return anchors.astype(bool)

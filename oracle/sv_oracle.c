@@ -27,6 +27,8 @@
  *   svo_kv_append : the appended cache read back with numpy indexing equals old tokens followed by the
  *       accepted rows; one call equals token-by-token calls; attention afterwards equals attention on a
  *       cache built with the longer prefix.
+ *   svo_jaccard_adjacent / svo_pick_anchors : Python set arithmetic on random subsets; identical layers give
+ *       J = 1, disjoint ones 0; numpy argsort for the top-K.
  *   Approximation quality of sparse vs dense attention: parity unpinned (the
  *       paper bounds nothing; reported as information only).
  */
@@ -423,6 +425,59 @@ int svo_kv_append(int S, int T, int Hkv, int D, int B, int NBmax, uint16_t *k_po
                     reps[(((int64_t)s * Hkv + h) * NBmax + b) * D + d] = sum / (double)cnt;
                 }
         }
+    }
+    return 0;
+}
+
+/*
+ * Anchor-layer calibration (Section 3.3, Eq. 7-8).  Input: the block sets kept by every layer for a batch
+ * of calibration samples (idx[l][s][h][0..cnt[l][s][h])).  The mask M_l of a sample spans all its
+ * candidate blocks (every KV head); adjacent layers are compared by the Jaccard similarity
+ * J(M_l, M_{l-1}) = |M_l n M_{l-1}| / |M_l u M_{l-1}| (Eq. 7), averaged over the samples, with
+ * J(M_1, M_0) = 0 for the first layer by definition.  inter/uni[l][s] are the set sizes, J[l] the mean.
+ */
+int svo_jaccard_adjacent(int n_layers, int S, int Hkv, int max_sel, const int32_t *idx, const int32_t *cnt,
+                         int32_t *inter, int32_t *uni, double *J)
+{
+    for (int l = 0; l < n_layers; ++l) {
+        double sum = 0.0;
+        for (int s = 0; s < S; ++s) {
+            int in = 0, un = 0;
+            if (l > 0) {
+                for (int h = 0; h < Hkv; ++h) {
+                    const int32_t *a = idx + ((((int64_t)l * S + s) * Hkv + h) * max_sel);
+                    const int32_t *b = idx + ((((int64_t)(l - 1) * S + s) * Hkv + h) * max_sel);
+                    int na = cnt[((int64_t)l * S + s) * Hkv + h], nb = cnt[((int64_t)(l - 1) * S + s) * Hkv + h];
+                    int common = 0;
+                    for (int i = 0; i < na; ++i)
+                        for (int j = 0; j < nb; ++j)
+                            if (a[i] == b[j]) ++common;
+                    in += common;
+                    un += na + nb - common;
+                }
+                sum += un > 0 ? (double)in / (double)un : 1.0;   /* two empty masks are identical */
+            }
+            inter[(int64_t)l * S + s] = in;
+            uni[(int64_t)l * S + s] = un;
+        }
+        J[l] = l > 0 ? sum / (double)S : 0.0;
+    }
+    return 0;
+}
+
+/*
+ * Eq. 8: the K layers with the lowest similarity to their predecessor (largest 1 - J) become anchors;
+ * equal similarities: the earlier layer first.  anchors[l] = 1 / 0.
+ */
+int svo_pick_anchors(int n_layers, const double *J, int K, uint8_t *anchors)
+{
+    if (K < 1 || K > n_layers) return 1;
+    for (int l = 0; l < n_layers; ++l) anchors[l] = 0;
+    for (int k = 0; k < K; ++k) {
+        int best = -1;
+        for (int l = 0; l < n_layers; ++l)
+            if (!anchors[l] && (best < 0 || 1.0 - J[l] > 1.0 - J[best])) best = l;
+        anchors[best] = 1;
     }
     return 0;
 }

@@ -513,3 +513,58 @@ def test_attention_after_append_sees_the_committed_tokens():
     before, _ = oracle.dense_verify_attn(c0["q"], c0["k_pool"], c0["v_pool"], c0["block_table"], c0["seq_lens"],
                                          c0["draft_k"], c0["draft_v"], None)
     np.testing.assert_allclose(after[:, 0], before[:, 3], rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- anchor calibration (Eq. 7-8)
+
+def _random_selection_stack(n_layers=6, S=3, Hkv=2, nb=40, n_keep=9, seed=3, p_keep=0.7):
+    """Selection lists with inter-layer correlation: a layer keeps each block of the previous layer with
+    probability p_keep (layer 3 is redrawn from scratch)."""
+    g = np.random.default_rng(seed)
+    idx = np.full((n_layers, S, Hkv, n_keep + 3), -1, np.int32)
+    cnt = np.zeros((n_layers, S, Hkv), np.int32)
+    for s in range(S):
+        for h in range(Hkv):
+            cur = set(g.choice(nb, n_keep, replace=False).tolist())
+            for l in range(n_layers):
+                if l == 3:
+                    cur = set(g.choice(nb, n_keep, replace=False).tolist())
+                elif l > 0:
+                    keep = {b for b in cur if g.random() < p_keep}
+                    rest = [b for b in range(nb) if b not in cur]
+                    cur = keep | set(g.choice(rest, max(0, n_keep + int(g.integers(0, 3)) - len(keep)), replace=False).tolist())
+                lst = sorted(cur)
+                idx[l, s, h, :len(lst)] = lst
+                cnt[l, s, h] = len(lst)
+    return idx, cnt
+
+
+def test_jaccard_matches_python_sets_and_first_layer_is_zero():
+    idx, cnt = _random_selection_stack()
+    inter, uni, J = oracle.jaccard_adjacent(idx, cnt)
+    L, S, H, _ = idx.shape
+    assert J[0] == 0.0 and (inter[0] == 0).all() and (uni[0] == 0).all()
+    for l in range(1, L):
+        js = []
+        for s in range(S):
+            a = {(h, b) for h in range(H) for b in idx[l, s, h, :cnt[l, s, h]].tolist()}
+            b_ = {(h, b) for h in range(H) for b in idx[l - 1, s, h, :cnt[l - 1, s, h]].tolist()}
+            assert inter[l, s] == len(a & b_) and uni[l, s] == len(a | b_)
+            js.append(len(a & b_) / len(a | b_))
+        assert abs(J[l] - np.mean(js)) < 1e-15
+    assert J[3] == J[1:].min()                    # the redrawn layer is the least similar to its predecessor
+    same = np.stack([idx[0]] * 3), np.stack([cnt[0]] * 3)
+    assert oracle.jaccard_adjacent(*same)[2].tolist() == [0.0, 1.0, 1.0]
+
+
+def test_pick_anchors_is_topk_of_dissimilarity():
+    idx, cnt = _random_selection_stack(n_layers=9, seed=8)
+    J = oracle.jaccard_adjacent(idx, cnt)[2]
+    for K in (1, 3, 9):
+        a = oracle.pick_anchors(J, K)
+        want = np.argsort(-(1.0 - J), kind="stable")[:K]
+        assert sorted(np.flatnonzero(a).tolist()) == sorted(want.tolist())
+        assert a[0]                                # J = 0 makes the first layer the most dissimilar one
+    assert oracle.pick_anchors(np.array([0.0, 0.5, 0.5, 0.5]), 2).tolist() == [True, True, False, False]
+    with pytest.raises(ValueError):
+        oracle.pick_anchors(J, 0)
