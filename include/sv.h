@@ -221,6 +221,23 @@ SV_API sv_status sv_verify_attn_noalloc(const sv_geom *geom, const void *q, cons
                                         const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out,
                                         float *lse, int32_t *status_word, void *stream);
 
+/*
+ * Anchor-layer calibration (Section 3.3).  sv_anchor_jaccard compares, for every calibration sample (the
+ * sequences of the batch) and every layer l >= 1, the block mask kept by layer l with that of layer l-1
+ * over all KV heads (Eq. 7): inter[l][s] = |M_l n M_{l-1}|, uni[l][s] = |M_l u M_{l-1}|; row l = 0 is zero.
+ *   sel_idx_all dev int32 [n_layers][S][Hkv][max_sel], sel_cnt_all dev int32 [n_layers][S][Hkv]: the lists
+ *   written by sv_select_blocks with every layer retrieving; inter / uni dev int32 [n_layers][S].
+ * sv_pick_anchors (host arithmetic on host arrays; several batches may be concatenated along the sample
+ * axis): J[l] = mean over samples of inter / uni, J[0] = 0 by definition, and the n_anchors layers with
+ * the largest 1 - J become anchors (Eq. 8; equal values: the earlier layer).  anchors: host uint8
+ * [n_layers]; jaccard: host double [n_layers] or NULL (then n_layers <= 256).
+ */
+SV_API sv_status sv_anchor_jaccard(const sv_geom *geom, int32_t n_layers, const int32_t *sel_idx_all,
+                                   const int32_t *sel_cnt_all, int32_t max_sel, int32_t *inter, int32_t *uni,
+                                   void *stream);
+SV_API sv_status sv_pick_anchors(const int32_t *inter, const int32_t *uni, int32_t n_layers, int32_t n_samples,
+                                 int32_t n_anchors, uint8_t *anchors, double *jaccard);
+
 /* Number of KV splits (CTAs per (sequence, KV head)) sv_verify_attn uses for this geometry. */
 SV_API int32_t sv_verify_attn_splits(const sv_geom *geom, int32_t max_sel);
 

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIG
 SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
 EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
-           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append")
+           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors")
 
 
 class SvError(RuntimeError):
@@ -64,6 +64,10 @@ def _load() -> ctypes.CDLL:
     lib.sv_select_blocks.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
     lib.sv_verify_attn.restype = ctypes.c_int
     lib.sv_verify_attn.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
+    lib.sv_anchor_jaccard.restype = ctypes.c_int
+    lib.sv_anchor_jaccard.argtypes = [gp, i32, vp, vp, i32, vp, vp, vp]
+    lib.sv_pick_anchors.restype = ctypes.c_int
+    lib.sv_pick_anchors.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     lib.sv_kv_append.restype = ctypes.c_int
     lib.sv_kv_append.argtypes = [gp, vp, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
     lib.sv_verify_attn_noalloc.restype = ctypes.c_int
@@ -183,3 +187,25 @@ def sv_kv_append(geom: sv_geom, k_pool, v_pool, block_table, seq_lens, draft_k, 
                              _ptr(n_accept, torch.int32, "n_accept"), int(accept_idx.shape[-1]),
                              _ptr(seq_lens_out, torch.int32, "seq_lens_out"), _ptr(reps, torch.float32, "reps"),
                              _stream(stream)), "sv_kv_append")
+
+
+def sv_anchor_jaccard(geom: sv_geom, sel_idx_all, sel_cnt_all, inter, uni, stream=None) -> None:
+    """Eq. 7 set sizes between adjacent layers.  sel_idx_all int32 [layers][S][Hkv][max_sel], sel_cnt_all int32
+    [layers][S][Hkv]; inter / uni int32 [layers][S] (outputs)."""
+    _check(_lib.sv_anchor_jaccard(ctypes.byref(geom), int(sel_idx_all.shape[0]), _ptr(sel_idx_all, torch.int32, "sel_idx_all"),
+                                  _ptr(sel_cnt_all, torch.int32, "sel_cnt_all"), int(sel_idx_all.shape[-1]),
+                                  _ptr(inter, torch.int32, "inter"), _ptr(uni, torch.int32, "uni"), _stream(stream)),
+           "sv_anchor_jaccard")
+
+
+def sv_pick_anchors(inter, uni, n_anchors: int):
+    """Eq. 8 on host arrays (numpy int32 [layers][samples]).  Returns (anchors bool [layers], J float64 [layers])."""
+    import numpy as np
+    inter = np.ascontiguousarray(inter, dtype=np.int32)
+    uni = np.ascontiguousarray(uni, dtype=np.int32)
+    n_layers, n_samples = inter.shape
+    anchors = np.zeros(n_layers, dtype=np.uint8)
+    J = np.zeros(n_layers, dtype=np.float64)
+    _check(_lib.sv_pick_anchors(inter.ctypes.data, uni.ctypes.data, n_layers, n_samples, int(n_anchors), anchors.ctypes.data,
+                                J.ctypes.data), "sv_pick_anchors")
+    return anchors.astype(bool), J

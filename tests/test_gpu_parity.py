@@ -465,3 +465,44 @@ def test_kv_append_parity(sv, block):
         assert torch.equal(reps[s, :, :nbn], rebuilt[s, :, :nbn])
     with pytest.raises(sv.SvError):
         sv.sv_kv_append(geom_c, kp, vp, btd, sld, dk, dv, torch.from_numpy(acc).cuda(), torch.from_numpy(n_acc).cuda(), sld, reps)
+
+
+def test_anchor_calibration_parity(sv):
+    """Eq. 7-8 on a stack whose layers retrieve from inputs with planted inter-layer correlation: set sizes
+    bit-exact against the oracle, same anchors."""
+    n_layers = 6
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=4, seq_len=(1500, 4000), budget_blocks=12, n_layers=n_layers)
+    geom = si.make_geometry(w)
+    layers = [si.make_layer(geom, layer=l) for l in range(n_layers)]
+    # correlate the layers: layers 1, 2, 4, 5 reuse the keys of their predecessor with a little noise in Q only
+    for l in (1, 2, 4, 5):
+        layers[l]["k_pool"] = layers[l - 1]["k_pool"]
+        layers[l]["q"] = layers[l - 1]["q"].copy()
+        layers[l]["q"][:, 0, ::5] = layers[l]["q"][:, 0, 1::5][:, :layers[l]["q"][:, 0, ::5].shape[1]]
+    S, Hkv, max_sel = w.n_seq, w.n_kv_heads, geom["max_sel"]
+    idx_all = torch.zeros((n_layers, S, Hkv, max_sel), dtype=torch.int32, device="cuda")
+    cnt_all = torch.zeros((n_layers, S, Hkv), dtype=torch.int32, device="cuda")
+    ref = []
+    for l, c in enumerate(layers):
+        d = Dev(sv, c)
+        sv.sv_block_reps(d.geom, d.kv, d.reps)
+        sv.sv_select_blocks(d.geom, d.q, d.reps, d.seq_lens, d.budget, 1, 1, idx_all[l], cnt_all[l])
+        ref.append(oracle_select(c, 1, 1, max_sel))
+    torch.cuda.synchronize()
+    # the perturbed queries were not gap-repaired: compare the calibration on the GPU's own lists
+    idx_h, cnt_h = idx_all.cpu().numpy(), cnt_all.cpu().numpy()
+    for l in (0, 3):
+        np.testing.assert_array_equal(cnt_h[l], ref[l][1])
+        np.testing.assert_array_equal(idx_h[l], ref[l][0])
+    inter = torch.full((n_layers, S), -1, dtype=torch.int32, device="cuda")
+    uni = torch.full((n_layers, S), -1, dtype=torch.int32, device="cuda")
+    gm = sv.make_geom(S, w.n_q_heads, Hkv, 128, 64, geom["max_blocks"], w.n_draft)
+    sv.sv_anchor_jaccard(gm, idx_all, cnt_all, inter, uni)
+    torch.cuda.synchronize()
+    inter_o, uni_o, J_o = oracle.jaccard_adjacent(idx_h, cnt_h)
+    np.testing.assert_array_equal(inter.cpu().numpy(), inter_o)
+    np.testing.assert_array_equal(uni.cpu().numpy(), uni_o)
+    anchors, J = sv.sv_pick_anchors(inter.cpu().numpy(), uni.cpu().numpy(), 2)
+    np.testing.assert_allclose(J, J_o, rtol=0, atol=1e-15)
+    np.testing.assert_array_equal(anchors, oracle.pick_anchors(J_o, 2))
+    assert anchors.tolist() == [True, False, False, True, False, False]     # the two layers with fresh keys

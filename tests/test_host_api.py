@@ -84,3 +84,19 @@ def test_workspace_size_formula(svb):
     assert 1 <= splits <= 64
     assert svb.sv_workspace_bytes(g, 64) == 1 * 8 * splits * 32 * 130 * 4 + 256
     assert svb.sv_workspace_bytes(svb.make_geom(1, 8, 3, 128, 64, 64, 4), 16) == 0
+
+
+def test_pick_anchors_matches_oracle_on_host(svb):
+    import numpy as np
+    g = np.random.default_rng(2)
+    uni = g.integers(5, 40, size=(12, 7)).astype(np.int32)
+    inter = (uni * g.random((12, 7))).astype(np.int32)
+    inter[0] = 0
+    uni[0] = 0
+    for K in (1, 5, 12):
+        a, J = svb.sv_pick_anchors(inter, uni, K)
+        Jo = np.concatenate([[0.0], (inter[1:] / uni[1:]).mean(axis=1)])
+        np.testing.assert_allclose(J, Jo, rtol=0, atol=1e-15)
+        np.testing.assert_array_equal(a, oracle.pick_anchors(Jo, K))
+    with pytest.raises(svb.SvError):
+        svb.sv_pick_anchors(inter, uni, 13)
