@@ -498,15 +498,18 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (tid == 0) SV_STAMP(10);
 }
 
+// Small CTAs: the reads of one launch (all partials, ~2 MB for the 32K-context case) spread over every SM.
+constexpr int kMergeThreads = 64;
+
 // Combine the per-split partials: o = sum_j 2^(m_j - m) o_j / sum_j 2^(m_j - m) l_j.
 // One thread per (row, 4 output dims).  The partials sit in L2; all loads of up to 16 splits are
 // issued before the first use so that the kernel costs one memory round trip, not one per split.
-__global__ void __launch_bounds__(256) merge_splits_kernel(const AttnParams p)
+__global__ void __launch_bounds__(kMergeThreads) merge_splits_kernel(const AttnParams p)
 {
     constexpr int U = 16;
     const int h = blockIdx.y, s = blockIdx.z;
     const int rows = p.G * p.T;
-    const int idx = blockIdx.x * 256 + threadIdx.x;
+    const int idx = blockIdx.x * kMergeThreads + threadIdx.x;
     grid_dependency_wait();     // the partials come from the attention kernel just before
     grid_launch_dependents();
     if (idx >= rows * 32) return;
@@ -747,8 +750,8 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
     if (e != cudaSuccess) return SV_ERR_CUDA;
     if (splits > 1 && !getenv("SV_PROBE_SKIP_MERGE")) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((rows * 32 + 255) / 256, geom->n_kv_heads, geom->n_seq);
-        cfg.blockDim = dim3(256);
+        cfg.gridDim = dim3((rows * 32 + kMergeThreads - 1) / kMergeThreads, geom->n_kv_heads, geom->n_seq);
+        cfg.blockDim = dim3(kMergeThreads);
         cfg.stream = cs;
         cudaLaunchAttribute attr[1];
         svh::pdl_attribute(attr);
