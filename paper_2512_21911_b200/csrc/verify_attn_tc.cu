@@ -9,14 +9,17 @@
 //   softmax      four threads per query row (tcgen05.ld 16x256b: the mma.sync accumulator fragment
 //                layout): mask, running max / sum in fp32 with quad shuffles, P rounded to bf16 into
 //                shared memory (K-major, 128-byte swizzle)
-//   Ou[128x128]  = P[128 x 64] . V        4 x tcgen05.mma (M128 N128 K16), V read MN-major from the
-//                                         tile exactly as TMA stored it, accumulator in TMEM
-//   O            = O * 2^(m_old - m_new) + Ou   in registers (32 dims of a row per thread)
+//   O[128x128]  += P[128 x 64] . V        4 x tcgen05.mma (M128 N128 K16), V read MN-major from the
+//                                         tile exactly as TMA stored it; O stays in TMEM for the whole
+//                                         kernel.  The exponentials use a reference maximum that is only
+//                                         moved -- with a rescale of O in TMEM -- when the true maximum
+//                                         has grown by more than 2^8 (the final O / l does not depend on
+//                                         the reference), so most units never touch O.
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 are two softmax warpgroups that take units alternately,
-// each with its own S / P / Ou buffers; warp 8 is the TMA producer, one thread of warp 9 issues every
-// S = Q K^T (and the warp owns the TMEM allocation), one thread of warp 10 issues every Ou = P V.  The third warpgroup gives its registers to the other
-// two (setmaxnreg).  Everything is chained with mbarriers; tcgen05.commit signals MMA completion.
+// each with its own S / P / O buffers; warp 8 is the TMA producer, one thread of warp 9 issues every
+// S = Q K^T (and the warp owns the TMEM allocation), one thread of warp 10 issues every O += P V.  The
+// third warpgroup gives its registers to the other two (setmaxnreg).  Everything is chained with mbarriers; tcgen05.commit signals MMA completion.
 // All waits are bounded; a wait that gives up sets *status and the CTA drains and frees its TMEM.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -63,7 +66,7 @@ constexpr int kOffMisc = kOffDraft + kStageBytes;
 constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 static_assert(20 <= 32, "one lane of the producer warp per barrier");
-constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, Ou: 2 x 128 columns
+constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns
 constexpr int kMergeStride = 132;                // floats per row of the cross-warpgroup merge buffer
 
 // barrier slots (8 bytes each) inside the misc area
@@ -73,9 +76,8 @@ enum Bar {
     kSReady = kEmpty + kStages, // [2] S of the warpgroup's unit is in TMEM
     kSFree = kSReady + 2,       // [2] the warpgroup has read S
     kPReady = kSFree + 2,       // [2] P is in shared memory
-    kOReady = kPReady + 2,      // [2] Ou is in TMEM
-    kOFree = kOReady + 2,       // [2] the warpgroup has read Ou
-    kStaged = kOFree + 2,       // Q (and the draft unit) are staged
+    kOReady = kPReady + 2,      // [2] the warpgroup's latest PV has been added to O in TMEM
+    kStaged = kOReady + 2,      // Q (and the draft unit) are staged
     kTmemDone = kStaged + 1,    // all warps are done with TMEM
     kNumBars = kTmemDone + 1
 };
@@ -113,7 +115,6 @@ __global__ void __launch_bounds__(kThreads, 1)
             uint32_t count = 1;
             if (lane >= kSFree && lane < kSFree + 2) count = n_active;
             if (lane >= kPReady && lane < kPReady + 2) count = n_active;
-            if (lane >= kOFree && lane < kOFree + 2) count = n_active;
             if (lane == kStaged) count = 8;
             if (lane == kTmemDone) count = 2 * n_active;
             mbar_init(bar(lane), count);
@@ -254,8 +255,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const int g = u & 1, k = u >> 1;
                         const bool ring = u >= off;
                         const int stage = ring ? (u - off) % kStages : 0;
-                        if (*abort_flag || !mbar_wait_bounded(bar(kPReady + g), k & 1) ||
-                            (k > 0 && !mbar_wait_bounded(bar(kOFree + g), (k - 1) & 1))) {
+                        if (*abort_flag || !mbar_wait_bounded(bar(kPReady + g), k & 1)) {
                             dead = true;
                             *abort_flag = 1;
                             if (p.status) atomicOr(p.status, 32);
@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             tc_mma_bf16(d, dp_hi | (p_lo + (uint32_t)((kk * 32) >> 4)), dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)),
-                                        idesc_pv, kk > 0);
+                                        idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);   // the warpgroup's first unit starts O
                         tc_commit(bar(kOReady + g));
                         if (ring) tc_commit(bar(kEmpty + stage));
                         if (u < 24) TC_STAMP(56 + u);
@@ -405,49 +405,24 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int off = has_draft ? 1 : 0;
     const int n_total = (j1 - j0) * upb + off;
 
-    // per slot: 32 output dims 8*jj + 2*qd + e  (index 2*jj + e), running max and partial row sum
-    float o[NH][32], m[NH], l[NH], corr_prev[NH];
+    // per slot (row): reference maximum of the exponentials (log2 units) and partial row sum
+    float m[NH], l[NH];
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
-#pragma unroll
-        for (int d = 0; d < 32; ++d) o[i][d] = 0.f;
         m[i] = -INFINITY;
         l[i] = 0.f;
-        corr_prev[i] = 1.f;
     }
     bool dead = false;
+    constexpr float kLazy = 8.f;   // the reference maximum may trail the true one by up to 2^8
 
-    // O = O * corr + Ou for the warpgroup's k-th unit, then hand the Ou buffer back
-    auto accumulate = [&](int k) {
+    // wait until the warpgroup's k-th PV has been added to O (warp-uniform outcome)
+    auto wait_pv = [&](int k) {
         if (!dead && __any_sync(0xffffffffu, *abort_flag || !mbar_wait_bounded(bar(kOReady + wg), k & 1))) {
-            dead = true;   // warp-uniform: the tcgen05.ld below must be executed by the whole warp or not at all
+            dead = true;
             *abort_flag = 1;
             if (p.status && lane == 0) atomicOr(p.status, 4);
         }
-        if (dead) return;
-        if (tid == 0 && k < 12) TC_STAMP(104 + k);
-        tc_fence_after_sync();
-#pragma unroll
-        for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo) {
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t r[32];
-                tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + c * 64, r);
-                tmem_ld_wait();
-#pragma unroll
-                for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int i = lo * 2 + hh;
-                            o[i][(c * 8 + j) * 2 + e] = fmaf(o[i][(c * 8 + j) * 2 + e], corr_prev[i], __uint_as_float(r[4 * j + 2 * hh + e]));
-                        }
-            }
-        }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(kOFree + wg));
+        if (!dead) tc_fence_after_sync();
     };
 
     int k = 0;
@@ -468,19 +443,18 @@ __global__ void __launch_bounds__(kThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kSFree + wg));   // the next S of this warpgroup may be issued
 
-        if (k > 0) accumulate(k - 1);                   // Ou of the previous unit is normally ready by now
-
         const bool is_draft = u < off;
         const int stage = is_draft ? 0 : (u - off) % kStages;
         const int nvalid = is_draft ? p.T : min(meta[stage], kUnit);
         uint8_t *pbuf = smem + kOffP + wg * kPBytes;
+        float sc[NH][16], factor[NH];
+        bool move = false;
 #pragma unroll
         for (int i = 0; i < NH; ++i) {
-            float sc[16];
 #pragma unroll
             for (int j = 0; j < 8; ++j)
 #pragma unroll
-                for (int e = 0; e < 2; ++e) sc[2 * j + e] = __uint_as_float(sr[i >> 1][4 * j + 2 * (i & 1) + e]);
+                for (int e = 0; e < 2; ++e) sc[i][2 * j + e] = __uint_as_float(sr[i >> 1][4 * j + 2 * (i & 1) + e]);
             if (is_draft || nvalid < kUnit) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
@@ -489,27 +463,65 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const int col = 8 * j + 2 * qd + e;
                         bool ok = col < nvalid;
                         if (is_draft) ok = ok && col < 32 && ((vis[i] >> (col & 31)) & 1u);
-                        if (!ok) sc[2 * j + e] = -INFINITY;
+                        if (!ok) sc[i][2 * j + e] = -INFINITY;
                     }
             }
             float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) mx = fmaxf(mx, sc[c]);
+            for (int c = 0; c < 16; ++c) mx = fmaxf(mx, sc[i][c]);
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float m_new = fmaxf(m[i], mx * p.scale_log2);
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-            corr_prev[i] = fast_exp2(m[i] - m_use);
-            m[i] = m_new;
+            const float um = mx * p.scale_log2;
+            // move the reference only when this unit's maximum exceeds it by more than 2^kLazy (or there is none yet)
+            factor[i] = 1.f;
+            if (um > m[i] + kLazy || (m[i] == -INFINITY && um > -INFINITY)) {
+                factor[i] = fast_exp2(m[i] - um);   // 0 when there was no reference
+                m[i] = um;
+                l[i] *= factor[i];
+                move = true;
+            }
+        }
+        // Every completion of the warpgroup's PV barrier is observed, in order (a parity wait cannot tell phase
+        // n from phase n - 2); by now the previous PV has normally landed, so this does not stall.
+        if (k > 0) {
+            wait_pv(k - 1);
+            if (dead) break;
+        }
+        if (k > 0 && __any_sync(0xffffffffu, move)) {
+            // rare: rescale this warp's rows of O in TMEM (the previous PV has landed, the next one is not issued
+            // before this warp reports P ready)
+#pragma unroll
+            for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t r[32];
+                    const uint32_t addr = t_o + ((uint32_t)(lo * 16) << 16) + c * 64;
+                    tmem_ld_16x256b_x8(addr, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+#pragma unroll
+                            for (int e = 0; e < 2; ++e)
+                                r[4 * j + 2 * hh + e] = __float_as_uint(__uint_as_float(r[4 * j + 2 * hh + e]) * factor[lo * 2 + hh]);
+                    tmem_st_16x256b_x8(addr, r);
+                }
+            tmem_st_wait();
+            tc_fence_before_sync();
+        }
+#pragma unroll
+        for (int i = 0; i < NH; ++i) {
+            const float m_use = (m[i] == -INFINITY) ? 0.f : m[i];
             float lsum = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float p0 = fast_exp2(fmaf(sc[2 * j], p.scale_log2, -m_use));
-                const float p1 = fast_exp2(fmaf(sc[2 * j + 1], p.scale_log2, -m_use));
+                const float p0 = fast_exp2(fmaf(sc[i][2 * j], p.scale_log2, -m_use));
+                const float p1 = fast_exp2(fmaf(sc[i][2 * j + 1], p.scale_log2, -m_use));
                 lsum += p0 + p1;
                 *reinterpret_cast<uint32_t *>(pbuf + swz128(trow[i], j) + 4 * qd) = pack_bf16(p0, p1);
             }
-            l[i] = l[i] * corr_prev[i] + lsum;
+            l[i] += lsum;
         }
         if (!is_draft && nvalid < kUnit) {
             // zero the value rows past the end of the sequence (0 * junk must stay 0)
@@ -525,7 +537,33 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (lane == 0) mbar_arrive(bar(kPReady + wg));
         if (tid == 0 && k < 12) TC_STAMP(92 + k);
     }
-    if (k > 0) accumulate(k - 1);
+    // fetch this warp's rows of O: 32 output dims 8*jj + 2*qd + e (index 2*jj + e) per slot
+    float o[NH][32];
+#pragma unroll
+    for (int i = 0; i < NH; ++i)
+#pragma unroll
+        for (int d = 0; d < 32; ++d) o[i][d] = 0.f;
+    if (k > 0) {
+        wait_pv(k - 1);
+        if (!dead) {
+            if (tid == 0) TC_STAMP(104);
+#pragma unroll
+            for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + c * 64, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) o[lo * 2 + hh][(c * 8 + j) * 2 + e] = __uint_as_float(r[4 * j + 2 * hh + e]);
+                }
+        }
+    }
+    if (tid == 0) TC_STAMP(105);
     tc_fence_before_sync();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar(kTmemDone));
@@ -533,6 +571,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------------ merge the two warpgroups, write out
     const int n_sm = 2 * wg_threads;
     named_bar_sync(1, n_sm);   // both warpgroups are past their last unit: the ring is free
+    if (tid == 0) TC_STAMP(106);
     float *mx_buf = reinterpret_cast<float *>(smem);             // [NH*34][128] floats, index k*128 + t
     const int t = quad * 32 + lane;
     if (wg == 1) {
@@ -545,6 +584,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     }
     named_bar_sync(1, n_sm);
+    if (tid == 0) TC_STAMP(107);
     if (wg == 1) return;
 #pragma unroll
     for (int i = 0; i < NH; ++i) {

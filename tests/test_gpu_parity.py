@@ -506,3 +506,32 @@ def test_anchor_calibration_parity(sv):
     np.testing.assert_allclose(J, J_o, rtol=0, atol=1e-15)
     np.testing.assert_array_equal(anchors, oracle.pick_anchors(J_o, 2))
     assert anchors.tolist() == [True, False, False, True, False, False]     # the two layers with fresh keys
+
+
+@pytest.mark.parametrize("name", ["cfg1_small", "rows64", "cfg3_small"])
+def test_attention_with_growing_logits_rescales_accumulator(sv, name):
+    """Keys that get larger along the sequence make the running maximum jump by far more than 2^8 between
+    units, which forces the in-TMEM rescale of the output accumulator; an arbitrary fixed block list is used
+    on both sides (no selection involved)."""
+    c = si.make_layer(si.make_geometry(SMALL[name]), sharp=True)
+    w = c["workload"]
+    kp = si.bf16_bits_to_f32(c["k_pool"])
+    for s in range(w.n_seq):
+        nb = int(c["n_blocks"][s])
+        for b in range(nb):
+            kp[c["block_table"][s, b]] *= np.float32(2.0 ** (4 * b // max(1, nb - 1)))     # x1 ... x16 along the sequence
+    c = dict(c, k_pool=si.f32_to_bf16_bits(kp))
+    idx = np.full((w.n_seq, w.n_kv_heads, c["max_sel"]), -1, np.int32)
+    cnt = np.zeros((w.n_seq, w.n_kv_heads), np.int32)
+    for s in range(w.n_seq):
+        nb = int(c["n_blocks"][s])
+        for h in range(w.n_kv_heads):
+            pick = np.arange(h % 2, nb, max(1, nb // c["max_sel"]) + 1)[:c["max_sel"]]
+            pick = np.union1d(pick, [nb - 1])[:c["max_sel"]]
+            idx[s, h, :len(pick)] = pick
+            cnt[s, h] = len(pick)
+    d = Dev(sv, c)
+    o, lse = gpu_attn(sv, d, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda())
+    o_ref, lse_ref = oracle_attn(c, idx, cnt)
+    assert np.abs(lse_ref).max() > 20          # the logits really are large
+    check_attn(o, lse, o_ref, lse_ref, f"growing logits {name}")
