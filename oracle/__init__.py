@@ -238,3 +238,75 @@ def pick_anchors(J, K):
     if rc:
         raise ValueError("K must be between 1 and the number of layers")
     return anchors.astype(bool)
+
+
+# ------------------------------------------------------------------ retrieval variants the paper discusses
+
+
+def group_query_row(q, Hkv, row):
+    """Retrieval query of draft token ``row`` (Section 2.2): group mean of that token's query heads."""
+    S, T, Hq, D = q.shape
+    qbar = np.zeros((S, Hkv, D), dtype=np.float64)
+    rc = _load().svo_group_query_row(S, T, Hq, Hkv, D, _p(q, np.uint16), int(row), _p(qbar, np.float64))
+    if rc:
+        raise ValueError("row outside the draft tokens")
+    return qbar
+
+
+def select_global(sc, seq_lens, budget, B, n_sink, n_local, max_sel):
+    """Budget shared by the KV heads (Eq. 6 read over all heads): the budget*Hkv best (head, block) pairs.
+    Returns (idx [S][Hkv][max_sel], cnt [S][Hkv])."""
+    S, Hkv, NBmax = sc.shape
+    idx = np.full((S, Hkv, max_sel), -1, dtype=np.int32)
+    cnt = np.zeros((S, Hkv), dtype=np.int32)
+    rc = _load().svo_select_global(S, Hkv, B, NBmax, _p(np.ascontiguousarray(sc), np.float64),
+                                   _p(seq_lens, np.int32), _p(budget, np.int32), n_sink, n_local, max_sel,
+                                   _p(idx, np.int32), _p(cnt, np.int32))
+    if rc == 2:
+        raise ValueError("forced sink/local blocks exceed the budget")
+    if rc == 3:
+        raise ValueError("a head's set does not fit max_sel")
+    assert rc == 0, rc
+    return idx, cnt
+
+
+def select_tokens(q, k_pool, block_table, seq_lens, budget, n_sink, n_local, max_sel):
+    """Every draft token retrieves with its own query.  Returns (idx [T][S][Hkv][max_sel], cnt [T][S][Hkv])."""
+    S, T, _, _ = q.shape
+    _, Hkv, B, _ = k_pool.shape
+    reps = block_reps(k_pool, block_table, seq_lens)
+    idx_all = np.full((T, S, Hkv, max_sel), -1, dtype=np.int32)
+    cnt_all = np.zeros((T, S, Hkv), dtype=np.int32)
+    for i in range(T):
+        sc = scores(group_query_row(q, Hkv, i), reps, seq_lens, B)
+        idx_all[i], cnt_all[i] = select(sc, seq_lens, budget, B, n_sink, n_local, max_sel)
+    return idx_all, cnt_all
+
+
+def pair_overlap(idx_all, cnt_all):
+    """|Sel_i n Sel_j| for every pair of draft tokens: int32 [S][Hkv][T][T]."""
+    T, S, Hkv, max_sel = idx_all.shape
+    inter = np.zeros((S, Hkv, T, T), np.int32)
+    rc = _load().svo_pair_overlap(T, S, Hkv, max_sel, _p(np.ascontiguousarray(idx_all), np.int32),
+                                  _p(np.ascontiguousarray(cnt_all), np.int32), _p(inter, np.int32))
+    assert rc == 0, rc
+    return inter
+
+
+def overlap_by_distance(inter, cnt_all, position):
+    """The statistic of the block-overlap figure (Section 2.2): for token pairs i != j at positional distance
+    |position[i] - position[j]|, the intersection of their retrieved blocks divided by the number of blocks a
+    token retrieves, averaged over pairs, heads and sequences.  Returns {distance: mean ratio}."""
+    S, Hkv, T, _ = inter.shape
+    acc = {}
+    for i in range(T):
+        for j in range(T):
+            if i == j:
+                continue
+            d = abs(int(position[i]) - int(position[j]))
+            for s in range(S):
+                for h in range(Hkv):
+                    n = max(int(cnt_all[i, s, h]), int(cnt_all[j, s, h]))
+                    r = float(inter[s, h, i, j]) / n if n else 1.0
+                    acc.setdefault(d, []).append(r)
+    return {d: float(np.mean(v)) for d, v in sorted(acc.items())}

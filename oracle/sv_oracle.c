@@ -29,6 +29,9 @@
  *       cache built with the longer prefix.
  *   svo_jaccard_adjacent / svo_pick_anchors : Python set arithmetic on random subsets; identical layers give
  *       J = 1, disjoint ones 0; numpy argsort for the top-K.
+ *   svo_group_query_row / svo_select_global / svo_pair_overlap (retrieval variants the paper discusses):
+ *       row 0 equals svo_group_query; brute-force enumeration over all (head, block) subsets on tiny inputs,
+ *       one KV head equals svo_select, numpy lexsort; Python set intersections.
  *   Approximation quality of sparse vs dense attention: parity unpinned (the
  *       paper bounds nothing; reported as information only).
  */
@@ -479,5 +482,108 @@ int svo_pick_anchors(int n_layers, const double *J, int K, uint8_t *anchors)
             if (!anchors[l] && (best < 0 || 1.0 - J[l] > 1.0 - J[best])) best = l;
         anchors[best] = 1;
     }
+    return 0;
+}
+
+/*
+ * Retrieval variants the paper discusses but does not adopt.
+ *
+ * (1) Retrieval query of draft token `row` (Section 2.2 measures how much the blocks retrieved by different
+ *     draft tokens "based on their respective query values" overlap): the group mean of that token's query
+ *     heads.  row = 0 is svo_group_query.
+ */
+int svo_group_query_row(int S, int T, int Hq, int Hkv, int D, const uint16_t *q, int row, double *qbar)
+{
+    if (Hq % Hkv || row < 0 || row >= T) return 1;
+    int G = Hq / Hkv;
+    for (int s = 0; s < S; ++s)
+        for (int h = 0; h < Hkv; ++h)
+            for (int d = 0; d < D; ++d) {
+                double sum = 0.0;
+                for (int g = 0; g < G; ++g)
+                    sum += bf16_to_f64(q[(((int64_t)s * T + row) * Hq + h * G + g) * D + d]);
+                qbar[((int64_t)s * Hkv + h) * D + d] = sum / (double)G;
+            }
+    return 0;
+}
+
+/*
+ * (2) Budget shared by the KV heads (Eq. 6 counts N_budget = ... x H / B blocks over all heads): the
+ *     budget[s] * Hkv best (head, block) pairs of a sequence are kept, whichever head they belong to.
+ *     The first n_sink and last n_local blocks of every head are kept first and count against the total.
+ *     Equal scores: the smaller head, then the smaller block index wins.  budget[s] >= number of blocks
+ *     keeps everything.  idx[s][h][0..cnt[s][h]) ascending.  Returns 2 when the forced blocks exceed the
+ *     total, 3 when a head's set does not fit max_sel.
+ */
+int svo_select_global(int S, int Hkv, int B, int NBmax, const double *scores, const int32_t *seq_lens,
+                      const int32_t *budget, int n_sink, int n_local, int max_sel, int32_t *idx, int32_t *cnt)
+{
+    for (int s = 0; s < S; ++s) {
+        int nb = (int)(((int64_t)seq_lens[s] + B - 1) / B);
+        int64_t total = (int64_t)budget[s] * Hkv;
+        char *keep = (char *)calloc((size_t)(nb > 0 ? (int64_t)nb * Hkv : 1), 1);
+        int64_t kept = 0;
+        if (budget[s] >= nb) {
+            for (int64_t e = 0; e < (int64_t)nb * Hkv; ++e) keep[e] = 1;
+        } else {
+            for (int h = 0; h < Hkv; ++h)
+                for (int b = 0; b < nb; ++b)
+                    if (b < n_sink || b >= nb - n_local) {
+                        keep[(int64_t)h * nb + b] = 1;
+                        ++kept;
+                    }
+            if (kept > total) {
+                free(keep);
+                return 2;
+            }
+            while (kept < total) {
+                int bh = -1, bb = -1;
+                for (int h = 0; h < Hkv; ++h)
+                    for (int b = 0; b < nb; ++b) {
+                        if (keep[(int64_t)h * nb + b]) continue;
+                        double v = scores[((int64_t)s * Hkv + h) * NBmax + b];
+                        if (bh < 0 || v > scores[((int64_t)s * Hkv + bh) * NBmax + bb]) bh = h, bb = b;
+                    }
+                keep[(int64_t)bh * nb + bb] = 1;
+                ++kept;
+            }
+        }
+        for (int h = 0; h < Hkv; ++h) {
+            int n = 0;
+            for (int b = 0; b < nb; ++b)
+                if (keep[(int64_t)h * nb + b]) {
+                    if (n >= max_sel) {
+                        free(keep);
+                        return 3;
+                    }
+                    idx[((int64_t)s * Hkv + h) * max_sel + n++] = b;
+                }
+            cnt[(int64_t)s * Hkv + h] = n;
+        }
+        free(keep);
+    }
+    return 0;
+}
+
+/*
+ * (3) Overlap of the blocks retrieved by two draft tokens (Section 2.2, the block-overlap figure): the size
+ *     of the intersection of their sets, per (sequence, KV head).  idx[i][s][h][0..cnt[i][s][h]) is the set
+ *     of draft token i.  inter[s][h][i][j] = |Sel_i n Sel_j| (the diagonal is the set size).
+ */
+int svo_pair_overlap(int T, int S, int Hkv, int max_sel, const int32_t *idx, const int32_t *cnt, int32_t *inter)
+{
+    for (int s = 0; s < S; ++s)
+        for (int h = 0; h < Hkv; ++h)
+            for (int i = 0; i < T; ++i)
+                for (int j = 0; j < T; ++j) {
+                    const int32_t *a = idx + (((int64_t)i * S + s) * Hkv + h) * max_sel;
+                    const int32_t *b = idx + (((int64_t)j * S + s) * Hkv + h) * max_sel;
+                    int na = cnt[((int64_t)i * S + s) * Hkv + h], nb = cnt[((int64_t)j * S + s) * Hkv + h];
+                    int common = 0;
+                    for (int x = 0; x < na; ++x)
+                        for (int y = 0; y < nb; ++y)
+                            if (a[x] == b[y]) ++common;
+                    inter[((((int64_t)s * Hkv + h) * T) + i) * T + j] = common;
+                }
     return 0;
 }

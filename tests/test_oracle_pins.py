@@ -568,3 +568,117 @@ def test_pick_anchors_is_topk_of_dissimilarity():
     assert oracle.pick_anchors(np.array([0.0, 0.5, 0.5, 0.5]), 2).tolist() == [True, True, False, False]
     with pytest.raises(ValueError):
         oracle.pick_anchors(J, 0)
+
+
+# ---------------------------------------------------------------------------- retrieval variants (Sections 2.2, 3.2)
+
+
+def test_group_query_row_zero_is_the_first_token_and_rows_follow_a_roll():
+    c = _tiny_case(T=4)
+    np.testing.assert_array_equal(oracle.group_query_row(c["q"], 2, 0), oracle.group_query(c["q"], 2))
+    for i in range(1, 4):
+        rolled = np.ascontiguousarray(np.roll(c["q"], -i, axis=1))
+        np.testing.assert_array_equal(oracle.group_query_row(c["q"], 2, i), oracle.group_query(rolled, 2))
+    # literal group mean of the widened values
+    want = si.bf16_bits_to_f64(c["q"])[:, 2].reshape(2, 2, 2, 8).mean(axis=2)
+    np.testing.assert_allclose(oracle.group_query_row(c["q"], 2, 2), want, rtol=0, atol=1e-15)
+    with pytest.raises(ValueError):
+        oracle.group_query_row(c["q"], 2, 4)
+
+
+def _brute_force_select_global(sc, nb, total, n_sink, n_local):
+    """Best-sum subset of (head, block) pairs of size `total` that contains the forced pairs."""
+    Hkv = sc.shape[0]
+    pairs = [(h, b) for h in range(Hkv) for b in range(nb)]
+    if total >= len(pairs):
+        return set(pairs)
+    forced = [(h, b) for (h, b) in pairs if b < n_sink or b >= nb - n_local]
+    rest = [x for x in pairs if x not in forced]
+    best, best_sum = None, -math.inf
+    for comb in itertools.combinations(rest, total - len(forced)):
+        tot = sum(sc[h, b] for (h, b) in comb)
+        if tot > best_sum:
+            best, best_sum = comb, tot
+    return set(forced) | set(best)
+
+
+@pytest.mark.parametrize("n_sink,n_local", [(0, 0), (1, 1)])
+def test_select_global_equals_brute_force_over_head_block_pairs(n_sink, n_local):
+    g = np.random.default_rng(23)
+    B, Hkv = 4, 2
+    for trial in range(10):
+        nb = int(g.integers(n_sink + n_local + 2, 8))
+        N = int(g.integers(n_sink + n_local, nb))          # per-head average; total = N * Hkv
+        L = nb * B - int(g.integers(0, B))
+        sc = np.full((1, Hkv, 8), -np.inf)
+        sc[0, :, :nb] = g.standard_normal((Hkv, nb))
+        idx, cnt = oracle.select_global(sc, np.array([L], np.int32), np.array([N], np.int32), B, n_sink, n_local, 8)
+        got = {(h, int(b)) for h in range(Hkv) for b in idx[0, h, :cnt[0, h]]}
+        assert got == _brute_force_select_global(sc[0], nb, N * Hkv, n_sink, n_local)
+        assert int(cnt.sum()) == N * Hkv
+        for h in range(Hkv):
+            assert np.all(np.diff(idx[0, h, :cnt[0, h]]) > 0)
+
+
+def test_select_global_special_cases():
+    g = np.random.default_rng(29)
+    B, nb = 4, 10
+    L = np.array([nb * B - 1], np.int32)
+    # one KV head: the shared budget is the per-head budget
+    sc1 = g.standard_normal((1, 1, nb))
+    for N in (3, 6, 10, 12):
+        a = oracle.select_global(sc1, L, np.array([N], np.int32), B, 1, 1, nb)
+        b = oracle.select(sc1, L, np.array([N], np.int32), B, 1, 1, nb)
+        np.testing.assert_array_equal(a[0], b[0])
+        np.testing.assert_array_equal(a[1], b[1])
+    # numpy statement: forced pairs, then the best of the rest by (score desc, head asc, block asc)
+    Hkv, N = 3, 4
+    sc = g.standard_normal((1, Hkv, nb))
+    sc[0, 1, 4] = sc[0, 0, 7]                                  # a tie across heads: the smaller head wins
+    idx, cnt = oracle.select_global(sc, L, np.array([N], np.int32), B, 1, 1, nb)
+    forced = {(h, b) for h in range(Hkv) for b in (0, nb - 1)}
+    rest = [(h, b) for h in range(Hkv) for b in range(1, nb - 1)]
+    order = np.lexsort(([b for _, b in rest], [h for h, _ in rest], [-sc[0, h, b] for h, b in rest]))
+    want = forced | {rest[i] for i in order[:N * Hkv - len(forced)]}
+    got = {(h, int(b)) for h in range(Hkv) for b in idx[0, h, :cnt[0, h]]}
+    assert got == want
+    # a head with uniformly higher scores takes the whole free budget
+    sc2 = g.standard_normal((1, 2, nb))
+    sc2[0, 1] += 100.0
+    idx, cnt = oracle.select_global(sc2, L, np.array([5], np.int32), B, 1, 1, nb)
+    assert cnt[0].tolist() == [2, 8]
+    with pytest.raises(ValueError):
+        oracle.select_global(sc2, L, np.array([1], np.int32), B, 1, 1, nb)       # forced pairs exceed the total
+    with pytest.raises(ValueError):
+        oracle.select_global(sc2, L, np.array([5], np.int32), B, 1, 1, 5)        # head 1 needs 8 slots
+
+
+def test_per_token_retrieval_and_pair_overlap_match_python_sets():
+    geom = si.make_geometry(si.WORKLOADS["cfg0"])
+    c = si.make_layer(geom)
+    T = c["q"].shape[1]
+    idx_all, cnt_all = oracle.select_tokens(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
+    first = oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
+    np.testing.assert_array_equal(idx_all[0], first[0])        # token 0 is the adopted strategy
+    np.testing.assert_array_equal(cnt_all[0], first[1])
+    inter = oracle.pair_overlap(idx_all, cnt_all)
+    S, Hkv = cnt_all.shape[1:]
+    for s in range(S):
+        for h in range(Hkv):
+            sets = [set(idx_all[i, s, h, :cnt_all[i, s, h]].tolist()) for i in range(T)]
+            for i in range(T):
+                for j in range(T):
+                    assert inter[s, h, i, j] == len(sets[i] & sets[j])
+    np.testing.assert_array_equal(inter, inter.transpose(0, 1, 3, 2))
+    # identical queries retrieve identical blocks: overlap ratio 1 at every distance
+    c2 = dict(c)
+    q_same = c["q"].copy()
+    q_same[:, 1:] = q_same[:, :1]
+    ia, ca = oracle.select_tokens(q_same, c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], 1, 1, 16)
+    ratios = oracle.overlap_by_distance(oracle.pair_overlap(ia, ca), ca, np.arange(T))
+    assert set(ratios) == set(range(1, T)) and all(abs(v - 1.0) < 1e-15 for v in ratios.values())
+    # hand-made sets: {0,1,2,3} vs {2,3,4,5} share half of their blocks
+    idx2 = np.array([[[[0, 1, 2, 3]]], [[[2, 3, 4, 5]]]], np.int32)
+    cnt2 = np.full((2, 1, 1), 4, np.int32)
+    r = oracle.overlap_by_distance(oracle.pair_overlap(idx2, cnt2), cnt2, [0, 1])
+    assert r == {1: 0.5}
