@@ -238,6 +238,38 @@ SV_API sv_status sv_anchor_jaccard(const sv_geom *geom, int32_t n_layers, const 
 SV_API sv_status sv_pick_anchors(const int32_t *inter, const int32_t *uni, int32_t n_layers, int32_t n_samples,
                                  int32_t n_anchors, uint8_t *anchors, double *jaccard);
 
+/*
+ * Retrieval variants the paper discusses but does not adopt; for comparison with sv_select_blocks.
+ *
+ * sv_select_blocks_tokens: every draft token retrieves with its own query (Section 2.2 analyses how much the
+ * blocks retrieved by different draft tokens "based on their respective query values" overlap).  Token i of
+ * every sequence runs the selection of sv_select_blocks with the group mean of its own query heads.
+ *   out_idx dev int32 [n_draft][S][Hkv][max_sel], out_cnt dev int32 [n_draft][S][Hkv]; the other arguments as
+ *   in sv_select_blocks.  n_draft launches on `stream`.
+ * sv_token_overlap: inter[s][h][i][j] = |Sel_i n Sel_j| for every pair of draft tokens (dev int32
+ *   [S][Hkv][n_draft][n_draft]; the diagonal is the set size).  The overlap ratio of the paper's block-overlap
+ *   figure is inter divided by the number of blocks a token retrieves, averaged per positional distance on
+ *   the host.  n_draft * ceil(max_blocks / 32) * 4 bytes of shared memory must fit in 48 KB
+ *   (SV_ERR_UNSUPPORTED otherwise).
+ * sv_select_blocks_global: Eq. 6 counts N_budget over all H KV heads; here the budget_blocks[s] * Hkv best
+ *   (head, block) pairs of a sequence are kept whichever head they belong to.  The first n_sink and last n_local
+ *   blocks of every head are kept first and count against the total; equal scores: the smaller head, then
+ *   the smaller block index.  budget_blocks[s] >= the number of blocks keeps everything.  A head may end up
+ *   with every block, so max_sel >= max_blocks is required (SV_ERR_SHAPE); Hkv * max_blocks <= 49152
+ *   (SV_ERR_UNSUPPORTED).  scores: dev float [S][Hkv][max_blocks], required; it receives the Eq. 5 scores.
+ *   Two launches on `stream`.  The lists feed sv_verify_attn unchanged (out_cnt differs per head).
+ */
+SV_API sv_status sv_select_blocks_tokens(const sv_geom *geom, const void *q, const float *reps,
+                                         const int32_t *seq_lens, const int32_t *budget_blocks, int32_t n_sink,
+                                         int32_t n_local, int32_t *out_idx, int32_t *out_cnt, int32_t max_sel,
+                                         void *stream);
+SV_API sv_status sv_token_overlap(const sv_geom *geom, const int32_t *sel_idx_all, const int32_t *sel_cnt_all,
+                                  int32_t max_sel, int32_t *inter, void *stream);
+SV_API sv_status sv_select_blocks_global(const sv_geom *geom, const void *q, const float *reps,
+                                         const int32_t *seq_lens, const int32_t *budget_blocks, int32_t n_sink,
+                                         int32_t n_local, int32_t *out_idx, int32_t *out_cnt, int32_t max_sel,
+                                         float *scores, void *stream);
+
 /* Number of KV splits (CTAs per (sequence, KV head)) sv_verify_attn uses for this geometry. */
 SV_API int32_t sv_verify_attn_splits(const sv_geom *geom, int32_t max_sel);
 

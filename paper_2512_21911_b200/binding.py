@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIG
 SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
 EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
-           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors")
+           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
+           "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global")
 
 
 class SvError(RuntimeError):
@@ -70,6 +71,12 @@ def _load() -> ctypes.CDLL:
     lib.sv_pick_anchors.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     lib.sv_kv_append.restype = ctypes.c_int
     lib.sv_kv_append.argtypes = [gp, vp, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+    lib.sv_select_blocks_tokens.restype = ctypes.c_int
+    lib.sv_select_blocks_tokens.argtypes = [gp, vp, vp, vp, vp, i32, i32, vp, vp, i32, vp]
+    lib.sv_token_overlap.restype = ctypes.c_int
+    lib.sv_token_overlap.argtypes = [gp, vp, vp, i32, vp, vp]
+    lib.sv_select_blocks_global.restype = ctypes.c_int
+    lib.sv_select_blocks_global.argtypes = [gp, vp, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]
     lib.sv_verify_attn_noalloc.restype = ctypes.c_int
     lib.sv_verify_attn_noalloc.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     return lib
@@ -196,6 +203,35 @@ def sv_anchor_jaccard(geom: sv_geom, sel_idx_all, sel_cnt_all, inter, uni, strea
                                   _ptr(sel_cnt_all, torch.int32, "sel_cnt_all"), int(sel_idx_all.shape[-1]),
                                   _ptr(inter, torch.int32, "inter"), _ptr(uni, torch.int32, "uni"), _stream(stream)),
            "sv_anchor_jaccard")
+
+
+def sv_select_blocks_tokens(geom: sv_geom, q, reps, seq_lens, budget_blocks, n_sink: int, n_local: int, out_idx,
+                            out_cnt, stream=None) -> None:
+    """Every draft token retrieves with its own query.  out_idx int32 [T][S][Hkv][max_sel], out_cnt int32 [T][S][Hkv]."""
+    _check(_lib.sv_select_blocks_tokens(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), _ptr(reps, torch.float32, "reps"),
+                                        _ptr(seq_lens, torch.int32, "seq_lens"),
+                                        _ptr(budget_blocks, torch.int32, "budget_blocks"), n_sink, n_local,
+                                        _ptr(out_idx, torch.int32, "out_idx"), _ptr(out_cnt, torch.int32, "out_cnt"),
+                                        int(out_idx.shape[-1]), _stream(stream)), "sv_select_blocks_tokens")
+
+
+def sv_token_overlap(geom: sv_geom, sel_idx_all, sel_cnt_all, inter, stream=None) -> None:
+    """|Sel_i n Sel_j| for every pair of draft tokens: inter int32 [S][Hkv][T][T] (output)."""
+    _check(_lib.sv_token_overlap(ctypes.byref(geom), _ptr(sel_idx_all, torch.int32, "sel_idx_all"),
+                                 _ptr(sel_cnt_all, torch.int32, "sel_cnt_all"), int(sel_idx_all.shape[-1]),
+                                 _ptr(inter, torch.int32, "inter"), _stream(stream)), "sv_token_overlap")
+
+
+def sv_select_blocks_global(geom: sv_geom, q, reps, seq_lens, budget_blocks, n_sink: int, n_local: int, out_idx,
+                            out_cnt, scores, stream=None) -> None:
+    """Budget shared by the KV heads: the budget * Hkv best (head, block) pairs of every sequence.
+    out_idx int32 [S][Hkv][max_sel >= max_blocks], out_cnt int32 [S][Hkv], scores float32 [S][Hkv][max_blocks]."""
+    _check(_lib.sv_select_blocks_global(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), _ptr(reps, torch.float32, "reps"),
+                                        _ptr(seq_lens, torch.int32, "seq_lens"),
+                                        _ptr(budget_blocks, torch.int32, "budget_blocks"), n_sink, n_local,
+                                        _ptr(out_idx, torch.int32, "out_idx"), _ptr(out_cnt, torch.int32, "out_cnt"),
+                                        int(out_idx.shape[-1]), _ptr(scores, torch.float32, "scores"), _stream(stream)),
+           "sv_select_blocks_global")
 
 
 def sv_pick_anchors(inter, uni, n_anchors: int):

@@ -72,6 +72,18 @@ def test_argument_validation_without_device(svb):
                                 0x6000, 16, None, None) == 4
     assert lib.sv_select_blocks(ctypes.byref(g), None, None, None, None, 1, 1, 1, None, None, 0x5000, 0x6000, 16,
                                 None, None) == 1
+    # retrieval variants: missing outputs, a list too narrow for one head to hold every block, too many pairs
+    assert lib.sv_select_blocks_tokens(ctypes.byref(g), 0x1000, 0x2000, 0x3000, 0x4000, 1, 1, None, None, 16, None) == 1
+    assert lib.sv_token_overlap(ctypes.byref(g), 0x1000, 0x2000, 16, None, None) == 1
+    assert lib.sv_select_blocks_global(ctypes.byref(g), 0x1000, 0x2000, 0x3000, 0x4000, 1, 1, 0x5000, 0x6000, 64,
+                                       None, None) == 1
+    assert lib.sv_select_blocks_global(ctypes.byref(g), 0x1000, 0x2000, 0x3000, 0x4000, 1, 1, 0x5000, 0x6000, 63,
+                                       0x7000, None) == 2
+    wide = svb.make_geom(1, 32, 8, 128, 64, 8192, 4)
+    assert lib.sv_select_blocks_global(ctypes.byref(wide), 0x1000, 0x2000, 0x3000, 0x4000, 1, 1, 0x5000, 0x6000, 8192,
+                                       0x7000, None) == 6
+    assert lib.sv_token_overlap(ctypes.byref(svb.make_geom(1, 32, 8, 128, 64, 32768, 32)), 0x1000, 0x2000, 16, 0x3000,
+                                None) == 6
     # attention: missing output
     kv = svb.sv_kv(0x1000, 0x2000, 0x3000, 0x4000, 4)
     assert lib.sv_verify_attn(ctypes.byref(g), 0x1000, ctypes.byref(kv), 0x1000, 0x1000, None, None, None, 0, 0.0,
