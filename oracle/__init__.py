@@ -310,3 +310,29 @@ def overlap_by_distance(inter, cnt_all, position):
                     r = float(inter[s, h, i, j]) / n if n else 1.0
                     acc.setdefault(d, []).append(r)
     return {d: float(np.mean(v)) for d, v in sorted(acc.items())}
+
+
+# ------------------------------------------------------------------ acceptance (Eq. 2-3)
+
+
+def accept(p_target, p_draft, tokens, parent, u_accept, u_next, want_dist=False):
+    """Acceptance walk of Section 2.1.  p_target, p_draft float32 [S][T][V]; tokens int32 [S][T]; parent int32
+    [S][T] or None (chain); u_accept float32 [S][T], u_next float32 [S] uniform numbers in [0, 1).
+    Returns dict(path int32 [S][T] (-1 padded), n_path int32 [S], next_token int32 [S], alpha float64 [S][T],
+    final_dist float64 [S][V] or None)."""
+    S, T, V = p_target.shape
+    path = np.full((S, T), -1, np.int32)
+    n_path = np.zeros(S, np.int32)
+    nxt = np.zeros(S, np.int32)
+    alpha = np.zeros((S, T), np.float64)
+    dist = np.zeros((S, V), np.float64) if want_dist else None
+    rc = _load().svo_accept(S, T, V, _p(np.ascontiguousarray(p_target), np.float32),
+                            _p(np.ascontiguousarray(p_draft), np.float32), _p(np.ascontiguousarray(tokens), np.int32),
+                            _p(None if parent is None else np.ascontiguousarray(parent), np.int32),
+                            _p(np.ascontiguousarray(u_accept), np.float32), _p(np.ascontiguousarray(u_next), np.float32),
+                            _p(path, np.int32), _p(n_path, np.int32), _p(nxt, np.int32), _p(alpha, np.float64),
+                            _p(dist, np.float64))
+    if rc == 2:
+        raise ValueError("token id outside the vocabulary")
+    assert rc == 0, rc
+    return dict(path=path, n_path=n_path, next_token=nxt, alpha=alpha, final_dist=dist)

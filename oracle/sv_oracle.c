@@ -32,6 +32,9 @@
  *   svo_group_query_row / svo_select_global / svo_pair_overlap (retrieval variants the paper discusses):
  *       row 0 equals svo_group_query; brute-force enumeration over all (head, block) subsets on tiny inputs,
  *       one KV head equals svo_select, numpy lexsort; Python set intersections.
+ *   svo_accept (Eq. 2-3): identical models accept everything and sample from the target (numpy searchsorted);
+ *       a one-hot target reduces to greedy prefix matching; the emitted token is distributed as the target,
+ *       summed exactly over the draft token(s) for one draft token and for two siblings.
  *   Approximation quality of sparse vs dense attention: parity unpinned (the
  *       paper bounds nothing; reported as information only).
  */
@@ -585,5 +588,99 @@ int svo_pair_overlap(int T, int S, int Hkv, int max_sel, const int32_t *idx, con
                             if (a[x] == b[y]) ++common;
                     inter[((((int64_t)s * Hkv + h) * T) + i) * T + j] = common;
                 }
+    return 0;
+}
+
+/*
+ * Acceptance of the draft tokens after verification (Section 2.1, Eq. 2-3).
+ *
+ * Rows of a step: row 0 is the token accepted in the previous step (the root), rows 1..T-1 the draft tokens;
+ * parent[s][i] < i is the row a draft token continues (NULL: the chain parent[i] = i - 1).  p_target[s][i][:]
+ * is the target model's distribution of the token that follows row i, p_draft[s][i][:] the draft model's
+ * distribution the children of row i were drawn from (fp32 probabilities, widened exactly).
+ *
+ * Walk from the root.  At row `cur` with current target distribution p (initially p_target[cur]) and draft
+ * distribution q = p_draft[cur], the children of cur are tried in row order: child c with token x is accepted
+ * with probability alpha = min(1, p(x) / q(x)) (Eq. 2), i.e. when u_accept[s][c] < alpha; the walk moves to c.
+ * A rejected child replaces p by norm(max(0, p - q)) (Eq. 3) before the next sibling is tried (a chain has no
+ * sibling: that case is Eq. 2-3 verbatim; for several siblings drawn independently from q this is the
+ * multi-round rule that keeps the output distributed as the target).  When no child is accepted (or cur is a
+ * leaf) the next token is drawn from the current p -- the adjusted distribution after a rejection, the
+ * target's own distribution after a fully accepted path -- by inversion of its cumulative sum in vocabulary
+ * order with u_next[s]: the smallest x with sum_{y<=x} p(y) >= u_next * sum_y p(y).  Everything after the
+ * first rejection on the path is discarded.
+ *
+ * A residual that is zero everywhere (p == q) leaves p unchanged.  q(x) = 0 gives alpha = 1.
+ *
+ * Outputs: path[s][0..n_path[s]) = rows whose tokens are kept (root first, then the accepted drafts in
+ * order); next_token[s]; alpha[s][c] for every child that was tried (NaN otherwise); final_dist[s][:]
+ * (optional) the normalised distribution next_token was drawn from.
+ */
+int svo_accept(int S, int T, int V, const float *p_target, const float *p_draft, const int32_t *tokens,
+               const int32_t *parent, const float *u_accept, const float *u_next, int32_t *path, int32_t *n_path,
+               int32_t *next_token, double *alpha, double *final_dist)
+{
+    double *p = (double *)malloc(sizeof(double) * (size_t)V);
+    if (!p) return 1;
+    for (int s = 0; s < S; ++s) {
+        const int32_t *tok = tokens + (int64_t)s * T;
+        for (int i = 0; i < T; ++i) alpha[(int64_t)s * T + i] = NAN;
+        int cur = 0, n = 0;
+        path[(int64_t)s * T + n++] = 0;
+        for (;;) {
+            const float *pt = p_target + ((int64_t)s * T + cur) * V;
+            const float *q = p_draft + ((int64_t)s * T + cur) * V;
+            for (int x = 0; x < V; ++x) p[x] = (double)pt[x];
+            int moved = 0;
+            for (int c = cur + 1; c < T; ++c) {
+                int par = parent ? parent[(int64_t)s * T + c] : c - 1;
+                if (par != cur) continue;
+                int x = tok[c];
+                if (x < 0 || x >= V) {
+                    free(p);
+                    return 2;
+                }
+                double qx = (double)q[x];
+                double a = (qx <= 0.0 || p[x] >= qx) ? 1.0 : p[x] / qx;
+                alpha[(int64_t)s * T + c] = a;
+                if ((double)u_accept[(int64_t)s * T + c] < a) {
+                    path[(int64_t)s * T + n++] = c;
+                    cur = c;
+                    moved = 1;
+                    break;
+                }
+                /* rejected: p <- norm(max(0, p - q)) (Eq. 3) */
+                double z = 0.0;
+                for (int y = 0; y < V; ++y) {
+                    double d = p[y] - (double)q[y];
+                    z += d > 0.0 ? d : 0.0;
+                }
+                if (z > 0.0)
+                    for (int y = 0; y < V; ++y) {
+                        double d = p[y] - (double)q[y];
+                        p[y] = d > 0.0 ? d / z : 0.0;
+                    }
+            }
+            if (moved) continue;
+            double tot = 0.0;
+            for (int y = 0; y < V; ++y) tot += p[y];
+            double target = (double)u_next[s] * tot, run = 0.0;
+            int pick = V - 1;
+            for (int y = 0; y < V; ++y) {
+                run += p[y];
+                if (run >= target && p[y] > 0.0) {
+                    pick = y;
+                    break;
+                }
+            }
+            next_token[s] = pick;
+            if (final_dist)
+                for (int y = 0; y < V; ++y) final_dist[(int64_t)s * V + y] = tot > 0.0 ? p[y] / tot : 0.0;
+            break;
+        }
+        n_path[s] = n;
+        for (int i = n; i < T; ++i) path[(int64_t)s * T + i] = -1;
+    }
+    free(p);
     return 0;
 }

@@ -682,3 +682,129 @@ def test_per_token_retrieval_and_pair_overlap_match_python_sets():
     cnt2 = np.full((2, 1, 1), 4, np.int32)
     r = oracle.overlap_by_distance(oracle.pair_overlap(idx2, cnt2), cnt2, [0, 1])
     assert r == {1: 0.5}
+
+
+# ---------------------------------------------------------------------------- acceptance (Eq. 2-3)
+
+
+def _dists(g, *shape):
+    p = g.random(shape).astype(np.float64) ** 3 + 1e-3            # a few dominant tokens, none with zero mass
+    p = (p / p.sum(-1, keepdims=True)).astype(np.float32)
+    return p
+
+
+def test_accept_identical_models_accept_every_draft_and_sample_from_the_target():
+    g = np.random.default_rng(51)
+    S, T, V = 6, 5, 37
+    p = _dists(g, S, T, V)
+    tok = g.integers(0, V, (S, T)).astype(np.int32)
+    u, un = g.random((S, T)).astype(np.float32), g.random(S).astype(np.float32)
+    r = oracle.accept(p, p.copy(), tok, None, u, un, want_dist=True)
+    assert r["n_path"].tolist() == [T] * S
+    assert r["path"].tolist() == [list(range(T))] * S
+    assert np.all(r["alpha"][:, 1:] == 1.0) and np.all(np.isnan(r["alpha"][:, 0]))
+    for s in range(S):
+        last = p[s, T - 1].astype(np.float64)
+        np.testing.assert_allclose(r["final_dist"][s], last / last.sum(), rtol=0, atol=1e-15)
+        cdf = np.cumsum(last)
+        assert r["next_token"][s] == int(np.searchsorted(cdf, np.float64(un[s]) * cdf[-1], side="left"))
+
+
+def test_accept_with_a_deterministic_target_is_greedy_prefix_matching():
+    """One-hot target rows: a draft token is kept exactly when it is the target's token, the first mismatch cuts
+    the rest and is replaced by the target's token (norm(max(0, p - q)) is the one-hot itself)."""
+    g = np.random.default_rng(52)
+    S, T, V = 8, 6, 11
+    want = g.integers(0, V, (S, T)).astype(np.int32)               # the target's token after each row
+    p = np.zeros((S, T, V), np.float32)
+    for s in range(S):
+        p[s, np.arange(T), want[s]] = 1.0
+    q = _dists(g, S, T, V)
+    tok = np.zeros((S, T), np.int32)
+    n_match = g.integers(0, T, S)
+    for s in range(S):
+        for i in range(1, T):
+            tok[s, i] = want[s, i - 1] if i <= n_match[s] else (want[s, i - 1] + 1 + g.integers(0, V - 1)) % V
+    r = oracle.accept(p, q, tok, None, g.random((S, T)).astype(np.float32), g.random(S).astype(np.float32))
+    for s in range(S):
+        assert r["n_path"][s] == 1 + n_match[s]
+        assert r["path"][s, :r["n_path"][s]].tolist() == list(range(1 + n_match[s]))
+        assert r["next_token"][s] == want[s, n_match[s]]
+
+
+def test_accept_one_draft_token_keeps_the_target_distribution():
+    """The purpose of Eq. 2-3: the first new token is distributed as the target, whatever the draft model is.
+    Exact check: sum over the draft token d ~ q of  alpha_d [x = d] + (1 - alpha_d) residual_d(x)  equals p(x)."""
+    g = np.random.default_rng(53)
+    V = 9
+    p, q = _dists(g, 1, 2, V), _dists(g, 1, 2, V)
+    out = np.zeros(V)
+    for d in range(V):
+        tok = np.array([[0, d]], np.int32)
+        acc = oracle.accept(p, q, tok, None, np.zeros((1, 2), np.float32), np.zeros(1, np.float32))
+        a = acc["alpha"][0, 1]
+        assert a == min(1.0, float(p[0, 0, d]) / float(q[0, 0, d]))
+        out[d] += float(q[0, 0, d]) * a
+        if a < 1.0:
+            rej = oracle.accept(p, q, tok, None, np.full((1, 2), 0.9999999, np.float32), np.zeros(1, np.float32), want_dist=True)
+            assert rej["n_path"][0] == 1
+            out += float(q[0, 0, d]) * (1.0 - a) * rej["final_dist"][0]
+    np.testing.assert_allclose(out, p[0, 0].astype(np.float64) / p[0, 0].astype(np.float64).sum(), rtol=0, atol=1e-7)
+
+
+def test_accept_two_siblings_keep_the_target_distribution():
+    """Tree step with two children drawn independently from q: try the first, on rejection adjust p and try the
+    second, on rejection adjust again and resample.  The emitted token is again distributed as the target."""
+    g = np.random.default_rng(54)
+    V = 6
+    p, q = _dists(g, 1, 3, V), _dists(g, 1, 3, V)
+    par = np.array([[-1, 0, 0]], np.int32)
+    q0 = q[0, 0].astype(np.float64)
+    out = np.zeros(V)
+    hi = np.float32(0.9999999)
+    for d1 in range(V):
+        for d2 in range(V):
+            w = q0[d1] * q0[d2]
+            tok = np.array([[0, d1, d2]], np.int32)
+            a1 = oracle.accept(p, q, tok, par, np.zeros((1, 3), np.float32), np.zeros(1, np.float32))["alpha"][0, 1]
+            out[d1] += w * a1
+            if a1 == 1.0:
+                continue
+            r2 = oracle.accept(p, q, tok, par, np.array([[0, hi, 0]], np.float32), np.zeros(1, np.float32))
+            a2 = r2["alpha"][0, 2]
+            assert a2 == 0.0 or r2["path"][0, :2].tolist() == [0, 2]      # a repeated rejected token has no mass left
+            out[d2] += w * (1 - a1) * a2
+            if a2 == 1.0:
+                continue
+            r3 = oracle.accept(p, q, tok, par, np.array([[0, hi, hi]], np.float32), np.zeros(1, np.float32), want_dist=True)
+            assert r3["n_path"][0] == 1
+            out += w * (1 - a1) * (1 - a2) * r3["final_dist"][0]
+    want = p[0, 0].astype(np.float64)
+    np.testing.assert_allclose(out, want / want.sum(), rtol=0, atol=1e-7)
+
+
+def test_accept_inverts_the_cumulative_sum_and_walks_a_tree():
+    g = np.random.default_rng(55)
+    S, T, V = 5, 7, 23
+    p, q = _dists(g, S, T, V), _dists(g, S, T, V)
+    par = np.full((S, T), -1, np.int32)
+    for s in range(S):
+        for i in range(1, T):
+            par[s, i] = g.integers(0, i)
+    tok = g.integers(0, V, (S, T)).astype(np.int32)
+    u, un = g.random((S, T)).astype(np.float32), g.random(S).astype(np.float32)
+    r = oracle.accept(p, q, tok, par, u, un, want_dist=True)
+    for s in range(S):
+        n = r["n_path"][s]
+        path = r["path"][s, :n]
+        assert path[0] == 0 and all(par[s, path[k]] == path[k - 1] for k in range(1, n))     # a root-to-node path
+        assert all(u[s, c] < r["alpha"][s, c] for c in path[1:])
+        tried = ~np.isnan(r["alpha"][s])
+        assert all(par[s, c] in path for c in np.nonzero(tried)[0])                          # only children of kept rows
+        assert all(u[s, c] >= r["alpha"][s, c] for c in np.nonzero(tried)[0] if c not in path)
+        cdf = np.cumsum(r["final_dist"][s])
+        x = r["next_token"][s]
+        lo = cdf[x - 1] if x > 0 else 0.0
+        assert lo - 1e-12 <= np.float64(un[s]) <= cdf[x] + 1e-12
+    with pytest.raises(ValueError):
+        oracle.accept(p, q, np.full((S, T), V, np.int32), par, u, un)
