@@ -553,6 +553,13 @@ def run_variants(args):
         "attn_first_token_per_head": lambda: sv.sv_verify_attn(g, q, kv, dk, dv, None, idx, cnt, out, workspace=ws),
         "attn_shared_budget": lambda: sv.sv_verify_attn(g, q, kv, dk, dv, None, idx_g, cnt_g, out, workspace=ws),
     }
+    # acceptance step (Eq. 2-3) on the same batch and draft length, Llama-3.1 vocabulary
+    ac = si.make_accept_case(S, T, 128256, seed=2100)
+    ad = {k: (None if v is None else torch.from_numpy(v).to(dev)) for k, v in ac.items()}
+    a_path = torch.zeros((S, T), dtype=torch.int32, device=dev)
+    a_n, a_next = torch.zeros(S, dtype=torch.int32, device=dev), torch.zeros(S, dtype=torch.int32, device=dev)
+    calls["accept_chain_vocab128256"] = lambda: sv.sv_accept(ad["p_target"], ad["p_draft"], ad["tokens"], None, ad["u_accept"],
+                                                             ad["u_next"], a_path, a_n, a_next)
     us = {}
     with torch.cuda.stream(stream):
         for name, fn in calls.items():
@@ -587,6 +594,7 @@ def run_variants(args):
         "timing": "median of 15 replays of a CUDA graph holding one call (1, 2 or n_draft kernel launches), L2 evicted "
                   "before each replay, CUDA events on the launching stream",
         "us_per_call": us,
+        "accept_rows_kept": a_n.cpu().tolist(),
         "shared_budget_blocks_per_head": {"min": int(cg.min()), "max": int(cg.max()), "mean": float(cg.mean())},
         "overlap_ratio_by_distance": {str(d): float(np.mean(v)) for d, v in sorted(ratios.items())},
         "overlap_note": "i.i.d. synthetic queries share only the planted blocks; the paper's > 0.8 is a property of "

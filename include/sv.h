@@ -270,6 +270,35 @@ SV_API sv_status sv_select_blocks_global(const sv_geom *geom, const void *q, con
                                          int32_t n_local, int32_t *out_idx, int32_t *out_cnt, int32_t max_sel,
                                          float *scores, void *stream);
 
+/*
+ * Acceptance of the draft tokens after verification (Section 2.1, Eq. 2-3), chains and trees.
+ *
+ * Rows of a step: row 0 is the token accepted in the previous step (the root), rows 1..n_draft-1 the draft
+ * tokens; parent[s][i] < i is the row a draft token continues (NULL: the chain parent[i] = i - 1).
+ *   p_target  dev float [S][n_draft][vocab]: the target model's distribution of the token that follows row i
+ *   p_draft   dev float [S][n_draft][vocab]: the draft model's distribution the children of row i were drawn from
+ *   tokens    dev int32 [S][n_draft] token ids of the rows (ids outside the vocabulary are clamped)
+ *   u_accept  dev float [S][n_draft], u_next dev float [S]: uniform numbers in [0, 1) supplied by the caller
+ * Walk from the root: the children of the current row are tried in row order; child c with token x is kept
+ * when u_accept[c] < min(1, p(x) / q(x)) (Eq. 2) and the walk moves to c; a rejected child replaces p by
+ * norm(max(0, p - q)) (Eq. 3) before the next sibling is tried (a residual without mass leaves p unchanged;
+ * q(x) = 0 accepts).  When no child is kept the next token is drawn from the current p -- after a rejection the
+ * adjusted distribution, after a fully accepted path the target's own -- as the smallest x with p(x) > 0 and
+ * sum_{y <= x} p(y) >= u_next * sum_y p(y).  The paper states Eq. 2-3 for a chain; the sibling rule is the
+ * multi-round form that keeps the emitted token distributed as the target when siblings are drawn
+ * independently from q.
+ *   path        dev int32 [S][n_draft]: rows whose tokens are kept, root first (so n_path >= 1), -1 padded; it is
+ *               the accept_idx / n_accept pair sv_kv_append takes
+ *   n_path      dev int32 [S]; next_token dev int32 [S]
+ *   alpha       optional dev float [S][n_draft]: the acceptance probability of every child that was tried
+ *               (other entries are left untouched)
+ * fp32 arithmetic with fixed summation order (results are reproducible run to run).  n_draft <= 32
+ * (SV_ERR_UNSUPPORTED), vocab a multiple of 4 and 16-byte aligned distributions (SV_ERR_ALIGN).  One launch.
+ */
+SV_API sv_status sv_accept(int32_t n_seq, int32_t n_draft, int32_t vocab, const float *p_target, const float *p_draft,
+                           const int32_t *tokens, const int32_t *parent, const float *u_accept, const float *u_next,
+                           int32_t *path, int32_t *n_path, int32_t *next_token, float *alpha, void *stream);
+
 /* Number of KV splits (CTAs per (sequence, KV head)) sv_verify_attn uses for this geometry. */
 SV_API int32_t sv_verify_attn_splits(const sv_geom *geom, int32_t max_sel);
 

@@ -23,7 +23,7 @@ SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in sc
 
 EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
            "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
-           "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global")
+           "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global", "sv_accept")
 
 
 class SvError(RuntimeError):
@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.sv_token_overlap.argtypes = [gp, vp, vp, i32, vp, vp]
     lib.sv_select_blocks_global.restype = ctypes.c_int
     lib.sv_select_blocks_global.argtypes = [gp, vp, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]
+    lib.sv_accept.restype = ctypes.c_int
+    lib.sv_accept.argtypes = [i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sv_verify_attn_noalloc.restype = ctypes.c_int
     lib.sv_verify_attn_noalloc.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     return lib
@@ -232,6 +234,21 @@ def sv_select_blocks_global(geom: sv_geom, q, reps, seq_lens, budget_blocks, n_s
                                         _ptr(out_idx, torch.int32, "out_idx"), _ptr(out_cnt, torch.int32, "out_cnt"),
                                         int(out_idx.shape[-1]), _ptr(scores, torch.float32, "scores"), _stream(stream)),
            "sv_select_blocks_global")
+
+
+def sv_accept(p_target, p_draft, tokens, parent, u_accept, u_next, path, n_path, next_token, alpha=None, stream=None) -> None:
+    """Acceptance walk (Eq. 2-3).  p_target, p_draft float32 [S][T][V]; tokens int32 [S][T]; parent int32 [S][T] or
+    None (chain); u_accept float32 [S][T]; u_next float32 [S]; outputs path int32 [S][T], n_path int32 [S],
+    next_token int32 [S], optional alpha float32 [S][T]."""
+    S, T, V = (int(x) for x in p_target.shape)
+    if tuple(p_draft.shape) != (S, T, V) or tuple(tokens.shape) != (S, T) or tuple(path.shape) != (S, T):
+        raise ValueError("sv_accept: shapes disagree")
+    _check(_lib.sv_accept(S, T, V, _ptr(p_target, torch.float32, "p_target"), _ptr(p_draft, torch.float32, "p_draft"),
+                          _ptr(tokens, torch.int32, "tokens"), _ptr(parent, torch.int32, "parent"),
+                          _ptr(u_accept, torch.float32, "u_accept"), _ptr(u_next, torch.float32, "u_next"),
+                          _ptr(path, torch.int32, "path"), _ptr(n_path, torch.int32, "n_path"),
+                          _ptr(next_token, torch.int32, "next_token"), _ptr(alpha, torch.float32, "alpha"),
+                          _stream(stream)), "sv_accept")
 
 
 def sv_pick_anchors(inter, uni, n_anchors: int):

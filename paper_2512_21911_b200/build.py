@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsv.so")
 SOURCES = ["sv_api.cu", "block_reps.cu", "select_blocks.cu", "verify_attn.cu", "verify_attn_tc.cu", "kv_append.cu", "anchor_calib.cu",
-           "select_variants.cu"]
+           "select_variants.cu", "accept.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -241,3 +241,32 @@ def make_layer(geom: dict, layer: int = 0, sharp: bool = False, tail_fill: Optio
 def shrink(w: Workload, **kw) -> Workload:
     """A copy of a workload with some fields replaced (tests use smaller contexts of the same shape)."""
     return replace(w, **kw)
+
+
+def make_accept_case(n_seq, n_draft, vocab, seed=2000, tree=False, temperature=0.35, draft_noise=0.2):
+    """Seeded inputs for the acceptance step: target and draft distributions per row (softmax of correlated
+    Gaussian logits, peaked like language-model outputs: `temperature` sharpens, `draft_noise` is how far the
+    draft model's logits stray from the target's), draft tokens drawn from the draft distribution of their
+    parent row, and the uniform numbers the step consumes.  Row 0 is the root.  float32 / int32 arrays."""
+    g = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, n_seq, n_draft, vocab])))
+    lt = g.standard_normal((n_seq, n_draft, vocab)) / temperature
+    ld = lt + draft_noise * g.standard_normal((n_seq, n_draft, vocab)) / temperature
+
+    def softmax(z):
+        z = z - z.max(-1, keepdims=True)
+        e = np.exp(z)
+        return (e / e.sum(-1, keepdims=True)).astype(np.float32)
+
+    p_target, p_draft = softmax(lt), softmax(ld)
+    parent = np.full((n_seq, n_draft), -1, np.int32)
+    for s in range(n_seq):
+        for i in range(1, n_draft):
+            parent[s, i] = g.integers(0, i) if tree else i - 1
+    tokens = np.zeros((n_seq, n_draft), np.int32)
+    for s in range(n_seq):
+        tokens[s, 0] = g.integers(0, vocab)
+        for i in range(1, n_draft):
+            q = p_draft[s, parent[s, i]].astype(np.float64)
+            tokens[s, i] = g.choice(vocab, p=q / q.sum())
+    return dict(p_target=p_target, p_draft=p_draft, tokens=tokens, parent=parent if tree else None,
+                u_accept=g.random((n_seq, n_draft), dtype=np.float32), u_next=g.random(n_seq, dtype=np.float32))

@@ -653,3 +653,109 @@ def test_per_token_retrieval_and_overlap_parity(sv, name):
     np.testing.assert_array_equal(inter.cpu().numpy(), oracle.pair_overlap(idx_h, cnt_h))
     ratios = oracle.overlap_by_distance(inter.cpu().numpy(), cnt_h, np.arange(T))
     assert all(0.0 <= v <= 1.0 for v in ratios.values())
+
+
+# ---------------------------------------------------------------------------- acceptance (Eq. 2-3)
+
+
+def _settle_accept_case(c, margin=1e-4):
+    """Move the uniform numbers away from the decision boundaries (as seen by the fp64 oracle) so that fp32 and
+    fp64 must take the same decisions; returns the oracle's result for the settled inputs."""
+    for _ in range(8):
+        r = oracle.accept(c["p_target"], c["p_draft"], c["tokens"], c["parent"], c["u_accept"], c["u_next"], want_dist=True)
+        moved = False
+        a = r["alpha"]
+        close = ~np.isnan(a) & (np.abs(c["u_accept"].astype(np.float64) - a) < margin) & (a < 1.0)
+        if close.any():
+            c["u_accept"][close] = np.clip(a[close] + 20 * margin, 0, 0.999).astype(np.float32)
+            moved = True
+        for s in range(c["u_next"].shape[0]):
+            cdf = np.cumsum(r["final_dist"][s])
+            x = int(r["next_token"][s])
+            lo = cdf[x - 1] if x > 0 else 0.0
+            if min(c["u_next"][s] - lo, cdf[x] - c["u_next"][s]) < 1e-5 and cdf[x] - lo > 4e-5:
+                c["u_next"][s] = np.float32(0.5 * (lo + cdf[x]))
+                moved = True
+        if not moved:
+            return r
+    raise AssertionError("could not settle the uniform numbers")
+
+
+def _gpu_accept(sv, c):
+    S, T, V = c["p_target"].shape
+    dev = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    path = torch.full((S, T), -9, dtype=torch.int32, device="cuda")
+    n_path = torch.full((S,), -9, dtype=torch.int32, device="cuda")
+    nxt = torch.full((S,), -9, dtype=torch.int32, device="cuda")
+    alpha = torch.full((S, T), float("nan"), device="cuda")
+    sv.sv_accept(dev(c["p_target"]), dev(c["p_draft"]), dev(c["tokens"]), dev(c["parent"]), dev(c["u_accept"]),
+                 dev(c["u_next"]), path, n_path, nxt, alpha)
+    torch.cuda.synchronize()
+    return path.cpu().numpy(), n_path.cpu().numpy(), nxt.cpu().numpy(), alpha.cpu().numpy()
+
+
+def _check_accept(c, r, got):
+    path, n_path, nxt, alpha = got
+    np.testing.assert_array_equal(n_path, r["n_path"])
+    np.testing.assert_array_equal(path, r["path"])
+    tried = ~np.isnan(r["alpha"])
+    np.testing.assert_array_equal(np.isnan(alpha), ~tried)
+    np.testing.assert_allclose(alpha[tried], r["alpha"][tried], rtol=2e-5, atol=1e-7)
+    for s in range(nxt.shape[0]):
+        if nxt[s] == r["next_token"][s]:
+            continue
+        # a different token is acceptable only next to the oracle's on the cumulative sum, within fp32 summation error
+        cdf = np.cumsum(r["final_dist"][s])
+        x = int(nxt[s])
+        lo = cdf[x - 1] if x > 0 else 0.0
+        assert r["final_dist"][s, x] > 0 and lo - 1e-5 <= c["u_next"][s] <= cdf[x] + 1e-5, (s, x, r["next_token"][s])
+    assert np.mean(nxt == r["next_token"]) >= 0.9
+
+
+@pytest.mark.parametrize("S,T,V,tree", [(4, 5, 512, False), (3, 8, 4096, True), (2, 16, 32768, True),
+                                         (5, 6, 10240, False), (2, 1, 2048, False), (1, 32, 8192, True)])
+def test_accept_parity(sv, S, T, V, tree):
+    """Acceptance walk against the oracle: kept rows bit-exact, acceptance probabilities to fp32 accuracy, the
+    drawn token equal (or adjacent within fp32 summation error on the cumulative sum).  Vocabularies from one CTA
+    per sequence (512) to clusters of 8 (32768), ragged per-thread segments (10240)."""
+    c = si.make_accept_case(S, T, V, seed=2000 + V + T, tree=tree)
+    r = _settle_accept_case(c)
+    _check_accept(c, r, _gpu_accept(sv, c))
+
+
+def test_accept_special_cases(sv):
+    """Identical models keep the whole chain; a one-hot target is greedy matching; a rejected token that repeats
+    among the siblings has no mass left; all-rejecting uniform numbers walk every sibling."""
+    c = si.make_accept_case(3, 6, 1024, seed=7)
+    c["p_draft"] = c["p_target"].copy()
+    r = _settle_accept_case(c)
+    got = _gpu_accept(sv, c)
+    assert got[1].tolist() == [6, 6, 6]
+    _check_accept(c, r, got)
+    # one-hot target
+    c = si.make_accept_case(4, 6, 1024, seed=8)
+    want = np.random.default_rng(3).integers(0, 1024, (4, 6))
+    c["p_target"][:] = 0
+    for s in range(4):
+        c["p_target"][s, np.arange(6), want[s]] = 1.0
+        c["tokens"][s, 1:3] = want[s, 0:2]                     # two matches, then whatever the draft drew
+    r = _settle_accept_case(c)
+    got = _gpu_accept(sv, c)
+    _check_accept(c, r, got)
+    assert all(got[1][s] >= 3 and got[2][s] == want[s, got[1][s] - 1] for s in range(4))
+    # siblings: every child rejected, one token repeated
+    c = si.make_accept_case(2, 5, 2048, seed=9, tree=True)
+    c["parent"][:] = np.array([-1, 0, 0, 0, 0], np.int32)
+    c["tokens"][:, 2] = c["tokens"][:, 1]
+    c["u_accept"][:] = 0.9995
+    r = _settle_accept_case(c)
+    got = _gpu_accept(sv, c)
+    _check_accept(c, r, got)
+
+
+@pytest.mark.parametrize("tree", [False, True])
+def test_accept_full_vocabulary(sv, tree):
+    """Llama-3.1 vocabulary (128256 entries), batch and draft length of the benchmark workload."""
+    c = si.make_accept_case(4, 8, 128256, seed=11, tree=tree)
+    r = _settle_accept_case(c)
+    _check_accept(c, r, _gpu_accept(sv, c))

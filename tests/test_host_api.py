@@ -84,6 +84,13 @@ def test_argument_validation_without_device(svb):
                                        0x7000, None) == 6
     assert lib.sv_token_overlap(ctypes.byref(svb.make_geom(1, 32, 8, 128, 64, 32768, 32)), 0x1000, 0x2000, 16, 0x3000,
                                 None) == 6
+    # acceptance: missing outputs, too many rows, vocabulary not a multiple of 4, misaligned distributions
+    acc = lambda S, T, V, pt=0x1000, out=0x7000: lib.sv_accept(S, T, V, pt, 0x2000, 0x3000, None, 0x4000, 0x5000, out,
+                                                               0x8000, 0x9000, None, None)
+    assert acc(1, 8, 1024, out=None) == 1
+    assert acc(0, 8, 1024) == 2 and acc(1, 0, 1024) == 2 and acc(1, 8, 0) == 2
+    assert acc(1, 33, 1024) == 6
+    assert acc(1, 8, 1022) == 3 and acc(1, 8, 1024, pt=0x1004) == 3
     # attention: missing output
     kv = svb.sv_kv(0x1000, 0x2000, 0x3000, 0x4000, 4)
     assert lib.sv_verify_attn(ctypes.byref(g), 0x1000, ctypes.byref(kv), 0x1000, 0x1000, None, None, None, 0, 0.0,
