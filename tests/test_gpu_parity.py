@@ -759,3 +759,48 @@ def test_accept_full_vocabulary(sv, tree):
     c = si.make_accept_case(4, 8, 128256, seed=11, tree=tree)
     r = _settle_accept_case(c)
     _check_accept(c, r, _gpu_accept(sv, c))
+
+
+def test_accept_feeds_kv_append(sv):
+    """One decoding step end to end on the GPU: verify-attention on the selected blocks, acceptance, commit of the
+    kept rows (root + accepted drafts) to the paged cache -- cache, lengths and representatives against the oracle
+    run on the same inputs."""
+    w = si.shrink(SMALL["cfg2_small"], n_draft=8)
+    geom = si.make_geometry(w)
+    c = si.make_layer(geom)
+    S, Hkv, T, B = w.n_seq, w.n_kv_heads, w.n_draft, w.block_size
+    # room for the commit: one more table column with fresh pages
+    bt = np.concatenate([c["block_table"], np.zeros((S, 1), np.int32)], axis=1)
+    for s in range(S):
+        bt[s, c["n_blocks"][s]] = c["n_pages"] + s
+    pad = np.zeros((S,) + c["k_pool"].shape[1:], np.uint16)
+    k_pool, v_pool = np.concatenate([c["k_pool"], pad]), np.concatenate([c["v_pool"], pad])
+    NB = bt.shape[1]
+    g = sv.make_geom(S, w.n_q_heads, Hkv, 128, B, NB, T)
+    kp, vp = bf16_dev(k_pool), bf16_dev(v_pool)
+    btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(c["seq_lens"]).cuda()
+    kv = sv.make_kv(kp, vp, btd, sld)
+    reps = torch.zeros((S, Hkv, NB, 128), device="cuda")
+    sv.sv_block_reps(g, kv, reps)
+    a = si.make_accept_case(S, T, 4096, seed=77)
+    r = _settle_accept_case(a)
+    dev = lambda x: None if x is None else torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    path = torch.zeros((S, T), dtype=torch.int32, device="cuda")
+    n_path, nxt = torch.zeros(S, dtype=torch.int32, device="cuda"), torch.zeros(S, dtype=torch.int32, device="cuda")
+    sv.sv_accept(dev(a["p_target"]), dev(a["p_draft"]), dev(a["tokens"]), None, dev(a["u_accept"]), dev(a["u_next"]),
+                 path, n_path, nxt)
+    new_len = torch.zeros_like(sld)
+    sv.sv_kv_append(g, kp, vp, btd, sld, bf16_dev(c["draft_k"]), bf16_dev(c["draft_v"]), path, n_path, new_len, reps)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(path.cpu().numpy(), r["path"])
+    ko, vo = k_pool.copy(), v_pool.copy()
+    reps_o = oracle.block_reps(ko, bt, c["seq_lens"])
+    len_o = oracle.kv_append(ko, vo, bt, c["seq_lens"], c["draft_k"], c["draft_v"], r["path"], r["n_path"], reps_o)
+    np.testing.assert_array_equal(new_len.cpu().numpy(), len_o)
+    assert np.all(len_o == c["seq_lens"] + r["n_path"]) and np.all(r["n_path"] >= 1)
+    np.testing.assert_array_equal(kp.cpu().view(torch.int16).numpy().view(np.uint16), ko)
+    np.testing.assert_array_equal(vp.cpu().view(torch.int16).numpy().view(np.uint16), vo)
+    rg = reps.cpu().numpy()
+    for s in range(S):
+        nbn = (int(len_o[s]) + B - 1) // B
+        np.testing.assert_allclose(rg[s, :, :nbn], reps_o[s, :, :nbn], rtol=0, atol=2e-6)
