@@ -271,6 +271,21 @@ SV_API sv_status sv_select_blocks_global(const sv_geom *geom, const void *q, con
                                          float *scores, void *stream);
 
 /*
+ * Representatives stored in bfloat16 (storage variant; halves the bytes block selection reads).
+ * sv_block_reps_bf16 is sv_block_reps with the fp32 mean rounded once to bfloat16 (nearest, ties to even):
+ *   reps_bf16 dev bf16 [S][Hkv][max_blocks][head_dim].  sv_select_blocks_bf16reps is sv_select_blocks reading
+ * that array; scores are still accumulated in fp32.  sv_kv_append refreshes fp32 representatives only: after
+ * a commit, rebuild the grown blocks of a bfloat16 array with sv_block_reps_bf16 on their block range.
+ */
+SV_API sv_status sv_block_reps_bf16(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
+                                    void *reps_bf16, void *stream);
+SV_API sv_status sv_select_blocks_bf16reps(const sv_geom *geom, const void *q, const void *reps_bf16,
+                                           const int32_t *seq_lens, const int32_t *budget_blocks, int32_t n_sink,
+                                           int32_t n_local, int32_t reuse_prev, const int32_t *prev_idx,
+                                           const int32_t *prev_cnt, int32_t *out_idx, int32_t *out_cnt,
+                                           int32_t max_sel, float *out_scores, void *stream);
+
+/*
  * Acceptance of the draft tokens after verification (Section 2.1, Eq. 2-3), chains and trees.
  *
  * Rows of a step: row 0 is the token accepted in the previous step (the root), rows 1..n_draft-1 the draft

@@ -336,3 +336,17 @@ def accept(p_target, p_draft, tokens, parent, u_accept, u_next, want_dist=False)
         raise ValueError("token id outside the vocabulary")
     assert rc == 0, rc
     return dict(path=path, n_path=n_path, next_token=nxt, alpha=alpha, final_dist=dist)
+
+
+def round_bf16(x):
+    """Nearest bfloat16 (ties to even) of fp64 values, returned as fp64."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty_like(x)
+    rc = _load().svo_round_bf16(ctypes.c_int64(x.size), _p(x, np.float64), _p(y, np.float64))
+    assert rc == 0, rc
+    return y
+
+
+def block_reps_bf16(k_pool, block_table, seq_lens):
+    """Block representatives kept in bfloat16: the fp64 means of Eq. 5 rounded once."""
+    return round_bf16(block_reps(k_pool, block_table, seq_lens))

@@ -684,3 +684,26 @@ int svo_accept(int S, int T, int V, const float *p_target, const float *p_draft,
     free(p);
     return 0;
 }
+
+/*
+ * Representatives stored in bfloat16 (storage variant of Eq. 5's block representative): the fp64 mean is
+ * rounded once, to the nearest bfloat16 (8 significand bits), ties to even; scores are then taken with the
+ * rounded values.  Magnitudes here are far from the bfloat16 range limits; subnormal results are not handled
+ * specially (frexp/ldexp keep them exact anyway).
+ */
+int svo_round_bf16(int64_t n, const double *x, double *y)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        double v = x[i];
+        if (v == 0.0 || !isfinite(v)) {
+            y[i] = v;
+            continue;
+        }
+        int e;
+        double m = frexp(v, &e);          /* v = m * 2^e, 0.5 <= |m| < 1 */
+        double scaled = ldexp(m, 8);      /* 8 significand bits: |scaled| in [128, 256) */
+        double r = nearbyint(scaled);     /* default rounding mode: to nearest, ties to even */
+        y[i] = ldexp(r, e - 8);
+    }
+    return 0;
+}

@@ -23,7 +23,8 @@ SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in sc
 
 EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
            "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
-           "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global", "sv_accept")
+           "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global", "sv_accept",
+           "sv_block_reps_bf16", "sv_select_blocks_bf16reps")
 
 
 class SvError(RuntimeError):
@@ -77,6 +78,10 @@ def _load() -> ctypes.CDLL:
     lib.sv_token_overlap.argtypes = [gp, vp, vp, i32, vp, vp]
     lib.sv_select_blocks_global.restype = ctypes.c_int
     lib.sv_select_blocks_global.argtypes = [gp, vp, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]
+    lib.sv_block_reps_bf16.restype = ctypes.c_int
+    lib.sv_block_reps_bf16.argtypes = [gp, kp, i32, i32, vp, vp]
+    lib.sv_select_blocks_bf16reps.restype = ctypes.c_int
+    lib.sv_select_blocks_bf16reps.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
     lib.sv_accept.restype = ctypes.c_int
     lib.sv_accept.argtypes = [i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sv_verify_attn_noalloc.restype = ctypes.c_int
@@ -137,6 +142,28 @@ def sv_block_reps(geom: sv_geom, kv: sv_kv, reps: torch.Tensor, block_begin: int
                   stream=None) -> None:
     _check(_lib.sv_block_reps(ctypes.byref(geom), ctypes.byref(kv), block_begin, block_end,
                               _ptr(reps, torch.float32, "reps"), _stream(stream)), "sv_block_reps")
+
+
+def sv_block_reps_bf16(geom: sv_geom, kv: sv_kv, reps_bf16: torch.Tensor, block_begin: int = 0, block_end: int = -1,
+                       stream=None) -> None:
+    """sv_block_reps with the representatives stored in bfloat16."""
+    _check(_lib.sv_block_reps_bf16(ctypes.byref(geom), ctypes.byref(kv), block_begin, block_end,
+                                   _ptr(reps_bf16, torch.bfloat16, "reps_bf16"), _stream(stream)), "sv_block_reps_bf16")
+
+
+def sv_select_blocks_bf16reps(geom: sv_geom, q, reps_bf16, seq_lens, budget_blocks, n_sink: int, n_local: int, out_idx,
+                              out_cnt, reuse_prev: bool = False, prev_idx=None, prev_cnt=None, out_scores=None,
+                              stream=None) -> None:
+    """sv_select_blocks reading bfloat16 representatives."""
+    _check(_lib.sv_select_blocks_bf16reps(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"),
+                                          _ptr(reps_bf16, torch.bfloat16, "reps_bf16"),
+                                          _ptr(seq_lens, torch.int32, "seq_lens"),
+                                          _ptr(budget_blocks, torch.int32, "budget_blocks"), n_sink, n_local,
+                                          1 if reuse_prev else 0, _ptr(prev_idx, torch.int32, "prev_idx"),
+                                          _ptr(prev_cnt, torch.int32, "prev_cnt"), _ptr(out_idx, torch.int32, "out_idx"),
+                                          _ptr(out_cnt, torch.int32, "out_cnt"), int(out_idx.shape[-1]),
+                                          _ptr(out_scores, torch.float32, "out_scores"), _stream(stream)),
+           "sv_select_blocks_bf16reps")
 
 
 def sv_select_blocks(geom: sv_geom, q, reps, seq_lens, budget_blocks, n_sink: int, n_local: int, out_idx, out_cnt,

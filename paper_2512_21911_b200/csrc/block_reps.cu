@@ -15,11 +15,12 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kRowGroups = kThreads / 16;   // 16 threads cover one 256-byte key row
 
-template <int B>
+// OutT: float (the default representatives) or __nv_bfloat16 (storage variant: the fp32 mean rounded once).
+template <int B, typename OutT>
 __global__ void __launch_bounds__(kThreads) block_reps_kernel(const uint4 *__restrict__ k_pool,
                                                               const int32_t *__restrict__ block_table,
                                                               const int32_t *__restrict__ seq_lens,
-                                                              float *__restrict__ reps, int Hkv, int NBmax,
+                                                              OutT *__restrict__ reps, int Hkv, int NBmax,
                                                               int block_begin, int block_end)
 {
     const int s = blockIdx.z, h = blockIdx.y;
@@ -61,14 +62,15 @@ __global__ void __launch_bounds__(kThreads) block_reps_kernel(const uint4 *__res
         float sum = 0.f;
 #pragma unroll
         for (int g = 0; g < kRowGroups; ++g) sum += part[g][threadIdx.x];
-        reps[(((size_t)s * Hkv + h) * NBmax + b) * 128 + threadIdx.x] = sum / (float)cnt;
+        reps[(((size_t)s * Hkv + h) * NBmax + b) * 128 + threadIdx.x] = static_cast<OutT>(sum / (float)cnt);
     }
 }
 
 }  // namespace
 
-extern "C" sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
-                                   float *reps, void *stream)
+template <typename OutT>
+static sv_status launch_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
+                                   OutT *reps, void *stream)
 {
     sv_status st = svh::check_geom(geom);
     if (st != SV_OK) return st;
@@ -91,9 +93,21 @@ extern "C" sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t
     const uint4 *pool = static_cast<const uint4 *>(kv->k_pool);
     const cudaError_t e =
         geom->block_size == 64
-            ? cudaLaunchKernelEx(&cfg, block_reps_kernel<64>, pool, kv->block_table, kv->seq_lens, reps,
+            ? cudaLaunchKernelEx(&cfg, block_reps_kernel<64, OutT>, pool, kv->block_table, kv->seq_lens, reps,
                                  (int)geom->n_kv_heads, (int)geom->max_blocks, (int)block_begin, (int)block_end)
-            : cudaLaunchKernelEx(&cfg, block_reps_kernel<128>, pool, kv->block_table, kv->seq_lens, reps,
+            : cudaLaunchKernelEx(&cfg, block_reps_kernel<128, OutT>, pool, kv->block_table, kv->seq_lens, reps,
                                  (int)geom->n_kv_heads, (int)geom->max_blocks, (int)block_begin, (int)block_end);
     return e == cudaSuccess ? svh::launch_status() : SV_ERR_CUDA;
+}
+
+extern "C" sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
+                                   float *reps, void *stream)
+{
+    return launch_block_reps<float>(geom, kv, block_begin, block_end, reps, stream);
+}
+
+extern "C" sv_status sv_block_reps_bf16(const sv_geom *geom, const sv_kv *kv, int32_t block_begin, int32_t block_end,
+                                        void *reps_bf16, void *stream)
+{
+    return launch_block_reps<__nv_bfloat16>(geom, kv, block_begin, block_end, static_cast<__nv_bfloat16 *>(reps_bf16), stream);
 }

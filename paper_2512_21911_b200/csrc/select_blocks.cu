@@ -51,7 +51,7 @@ __device__ __forceinline__ uint32_t order_key(float x)
 
 struct SelectParams {
     const __nv_bfloat16 *q;   // [S][T][Hq][128]
-    const float *reps;        // [S][Hkv][NBmax][128]
+    const void *reps;         // [S][Hkv][NBmax][128], float or bfloat16
     const int32_t *seq_lens;
     const int32_t *budget;
     int32_t *out_idx;
@@ -94,6 +94,8 @@ __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t
 // keys straight into CTA 0's shared memory (distributed shared memory), then signals an mbarrier there
 // and exits; CTA 0 selects.  The only cluster-wide barrier is split (arrive early, wait late) so that
 // its latency hides behind the loads.
+// kBf16: the representatives are stored in bfloat16 (storage variant); scores are fp32 either way.
+template <bool kBf16>
 __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
 {
     cg::cluster_group cluster = cg::this_cluster();
@@ -121,11 +123,23 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // before any global request is in flight
     SEL_STAMP(11);
     const int b0 = rank * p.chunk;
-    const float4 *rbase = reinterpret_cast<const float4 *>(p.reps + ((size_t)s * p.Hkv + h) * p.NBmax * 128);
+    constexpr int kRowBytes = kBf16 ? 256 : 512, kLaneBytes = kRowBytes / 32;
+    const char *rbase = static_cast<const char *>(p.reps) + ((size_t)s * p.Hkv + h) * p.NBmax * kRowBytes;
+    auto row_ptr = [&](int row) { return rbase + (size_t)row * kRowBytes + lane * kLaneBytes; };
+    auto load_row = [&](int row) {
+        if constexpr (kBf16) {
+            const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(row_ptr(row)));
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
+            return make_float4(lo.x, lo.y, hi.x, hi.y);
+        } else {
+            return __ldg(reinterpret_cast<const float4 *>(row_ptr(row)));
+        }
+    };
     int b = b0 + warp * kRowsPerIter;
 #pragma unroll
     for (int i = 0; i < kRowsPerIter; ++i)
-        if (b + i < min(b0 + p.chunk, p.NBmax)) svk::prefetch_l2(rbase + (size_t)(b + i) * 32 + lane);
+        if (b + i < min(b0 + p.chunk, p.NBmax)) svk::prefetch_l2(row_ptr(b + i));
     const int G = p.Hq / p.Hkv;
     const __nv_bfloat16 *q0 = p.q + ((size_t)s * p.T * p.Hq + (size_t)h * G) * 128;
     if (tid < G * 2) svk::prefetch_l2(q0 + tid * 64);
@@ -141,7 +155,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     auto load_rows = [&](int bb, int hi) {
 #pragma unroll
         for (int i = 0; i < kRowsPerIter; ++i)
-            r[i] = (bb + i < hi) ? __ldg(rbase + (size_t)(bb + i) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+            r[i] = (bb + i < hi) ? load_row(bb + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     };
     load_rows(b, min(b0 + p.chunk, p.NBmax));
     float qsum = 0.f;
@@ -310,11 +324,10 @@ __global__ void copy_selection_kernel(const int32_t *__restrict__ prev_idx, cons
 
 }  // namespace
 
-extern "C" sv_status sv_select_blocks(const sv_geom *geom, const void *q, const float *reps, const int32_t *seq_lens,
-                                      const int32_t *budget_blocks, int32_t n_sink, int32_t n_local,
-                                      int32_t reuse_prev, const int32_t *prev_idx, const int32_t *prev_cnt,
-                                      int32_t *out_idx, int32_t *out_cnt, int32_t max_sel, float *out_scores,
-                                      void *stream)
+static sv_status select_impl(const sv_geom *geom, const void *q, const void *reps, bool reps_bf16, const int32_t *seq_lens,
+                             const int32_t *budget_blocks, int32_t n_sink, int32_t n_local, int32_t reuse_prev,
+                             const int32_t *prev_idx, const int32_t *prev_cnt, int32_t *out_idx, int32_t *out_cnt,
+                             int32_t max_sel, float *out_scores, void *stream)
 {
     sv_status st = svh::check_geom(geom);
     if (st != SV_OK) return st;
@@ -355,7 +368,9 @@ extern "C" sv_status sv_select_blocks(const sv_geom *geom, const void *q, const 
 
     const size_t smem = (size_t)CL * chunk * sizeof(uint32_t);
     if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        (reps_bf16 ? cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                   : cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+            cudaSuccess)
         return SV_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CL, geom->n_kv_heads, geom->n_seq);
@@ -370,6 +385,28 @@ extern "C" sv_status sv_select_blocks(const sv_geom *geom, const void *q, const 
     svh::pdl_attribute(attr + 1);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, select_kernel, p) != cudaSuccess) return SV_ERR_CUDA;
+    if ((reps_bf16 ? cudaLaunchKernelEx(&cfg, select_kernel<true>, p) : cudaLaunchKernelEx(&cfg, select_kernel<false>, p)) !=
+        cudaSuccess)
+        return SV_ERR_CUDA;
     return svh::launch_status();
+}
+
+extern "C" sv_status sv_select_blocks(const sv_geom *geom, const void *q, const float *reps, const int32_t *seq_lens,
+                                      const int32_t *budget_blocks, int32_t n_sink, int32_t n_local,
+                                      int32_t reuse_prev, const int32_t *prev_idx, const int32_t *prev_cnt,
+                                      int32_t *out_idx, int32_t *out_cnt, int32_t max_sel, float *out_scores,
+                                      void *stream)
+{
+    return select_impl(geom, q, reps, false, seq_lens, budget_blocks, n_sink, n_local, reuse_prev, prev_idx, prev_cnt,
+                       out_idx, out_cnt, max_sel, out_scores, stream);
+}
+
+extern "C" sv_status sv_select_blocks_bf16reps(const sv_geom *geom, const void *q, const void *reps_bf16,
+                                               const int32_t *seq_lens, const int32_t *budget_blocks, int32_t n_sink,
+                                               int32_t n_local, int32_t reuse_prev, const int32_t *prev_idx,
+                                               const int32_t *prev_cnt, int32_t *out_idx, int32_t *out_cnt,
+                                               int32_t max_sel, float *out_scores, void *stream)
+{
+    return select_impl(geom, q, reps_bf16, true, seq_lens, budget_blocks, n_sink, n_local, reuse_prev, prev_idx, prev_cnt,
+                       out_idx, out_cnt, max_sel, out_scores, stream);
 }

@@ -804,3 +804,52 @@ def test_accept_feeds_kv_append(sv):
     for s in range(S):
         nbn = (int(len_o[s]) + B - 1) // B
         np.testing.assert_allclose(rg[s, :, :nbn], reps_o[s, :, :nbn], rtol=0, atol=2e-6)
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg1_small", "cfg2_small", "cfg3_small"])
+def test_bf16_representatives_parity(sv, name):
+    """Representatives stored in bfloat16: the GPU rounds its fp32 mean, the oracle its fp64 mean -- equal except
+    where the two means straddle a rounding boundary (one bfloat16 step, rare); scores to fp32 accuracy of the
+    rounded values; block lists bit-exact wherever the oracle's boundary gap exceeds the measured score error."""
+    w = SMALL[name]
+    geom = si.make_geometry(w)
+    c = si.make_layer(geom)
+    d = Dev(sv, c)
+    S, Hkv, NB, max_sel = w.n_seq, w.n_kv_heads, c["max_blocks"], geom["max_sel"]
+    reps16 = torch.zeros((S, Hkv, NB, 128), dtype=torch.bfloat16, device="cuda")
+    sv.sv_block_reps_bf16(d.geom, d.kv, reps16)
+    idx = torch.full((S, Hkv, max_sel), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((S, Hkv), -7, dtype=torch.int32, device="cuda")
+    sc = torch.zeros((S, Hkv, NB), device="cuda")
+    sv.sv_select_blocks_bf16reps(d.geom, d.q, reps16, d.seq_lens, d.budget, 1, 1, idx, cnt, out_scores=sc)
+    torch.cuda.synchronize()
+    reps_o = oracle.block_reps_bf16(c["k_pool"], c["block_table"], c["seq_lens"])
+    sc_o = oracle.scores(oracle.group_query(c["q"], Hkv), reps_o, c["seq_lens"], w.block_size)
+    idx_o, cnt_o = oracle.select(sc_o, c["seq_lens"], c["budget"], w.block_size, 1, 1, max_sel)
+    rg = bf16_host(reps16)
+    idx_h, cnt_h, sc_h = idx.cpu().numpy(), cnt.cpu().numpy(), sc.cpu().numpy()
+    n_val = n_diff = 0
+    exact = 0
+    for s in range(S):
+        nb = int(c["n_blocks"][s])
+        a, b = rg[s, :, :nb], reps_o[s, :, :nb]
+        step = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(b), 1e-30))) - 7)     # one bfloat16 step at that magnitude
+        assert np.all(np.abs(a - b) <= step * 1.0000001)
+        n_val += a.size
+        n_diff += int((a != b).sum())
+        err = float(np.abs(sc_h[s, :, :nb] - sc_o[s, :, :nb]).max())
+        np.testing.assert_array_equal(cnt_h[s], cnt_o[s])
+        for h in range(Hkv):
+            N = int(cnt_o[s, h])
+            free = np.sort(sc_o[s, h, 1:nb - 1])[::-1]
+            k = N - 2
+            gap = np.inf if (N >= nb or k <= 0 or k >= free.size) else free[k - 1] - free[k]
+            got = idx_h[s, h, :N]
+            assert np.all(np.diff(got) > 0) and got[0] == 0 and got[-1] == nb - 1
+            if gap > 2.5 * err + 1e-12:
+                np.testing.assert_array_equal(got, idx_o[s, h, :N])
+                exact += 1
+            else:
+                assert all(b_ in (0, nb - 1) or sc_o[s, h, b_] >= free[k - 1] - 2.5 * err - 1e-12 for b_ in got)
+    assert n_diff <= max(2, n_val // 2000), (n_diff, n_val)
+    assert exact >= (S * Hkv * 3) // 4

@@ -25,7 +25,7 @@ def svb():
 def test_exports_every_declared_symbol(svb):
     header = open(os.path.join(ROOT, "include", "sv.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(sv_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(sv_[a-z0-9_]+)\s*\(", header))
     assert declared == set(svb.EXPORTS)
     lib = ctypes.CDLL(svb.LIB_PATH)
     for name in declared:

@@ -808,3 +808,24 @@ def test_accept_inverts_the_cumulative_sum_and_walks_a_tree():
         assert lo - 1e-12 <= np.float64(un[s]) <= cdf[x] + 1e-12
     with pytest.raises(ValueError):
         oracle.accept(p, q, np.full((S, T), V, np.int32), par, u, un)
+
+
+def test_round_bf16_is_nearest_representable_with_ties_to_even():
+    g = np.random.default_rng(61)
+    x = np.concatenate([g.standard_normal(4000) * 10.0 ** g.integers(-6, 6, 4000), [0.0, 1.0, -1.0, 255.0, 256.5]])
+    y = oracle.round_bf16(x)
+    # representable: a float32 whose low 16 bits are zero
+    bits = y.astype(np.float32).view(np.uint32)
+    assert np.all(y.astype(np.float32).astype(np.float64) == y) and np.all(bits & 0xFFFF == 0)
+    # nearest: no bfloat16 neighbour is closer
+    up = (bits + 0x10000).view(np.float32).astype(np.float64)
+    dn = (bits - 0x10000).view(np.float32).astype(np.float64)
+    nz = x != 0
+    assert np.all(np.abs(y - x)[nz] <= np.abs(up - x)[nz]) and np.all(np.abs(y - x)[nz] <= np.abs(dn - x)[nz])
+    # ties go to the even significand: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert oracle.round_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert oracle.round_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+    assert oracle.round_bf16(np.array([-(1.0 + 2.0 ** -8)]))[0] == -1.0
+    # agrees with the float32 -> bfloat16 conversion of the input generator wherever float32 holds x exactly
+    x32 = x.astype(np.float32)
+    np.testing.assert_array_equal(oracle.round_bf16(x32.astype(np.float64)), si.bf16_bits_to_f64(si.f32_to_bf16_bits(x32)))
