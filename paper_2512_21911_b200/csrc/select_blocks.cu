@@ -43,6 +43,19 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kRowsPerIter = 4;   // independent representative rows a warp has in flight
 
+// Histogram bin -> shared-memory slot: one pad word per 32 bins, so that a warp whose lane j reads bins
+// 8j .. 8j+7 (the scan below) touches 32 different banks with every load.
+constexpr int kHistSlots = 256 + 8;
+constexpr int kFastChunks = 4;   // fast selection path: up to 4 keys per thread (2048 blocks)
+constexpr int kFastCap = 32;     // ... and at most this many keys left at the boundary after the histogram levels
+__device__ __forceinline__ uint32_t hist_slot(uint32_t bin) { return bin + (bin >> 5); }
+
+// inverse of order_key (defined below): the score a key was made from
+__device__ __forceinline__ float key_score(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+
 __device__ __forceinline__ uint32_t order_key(float x)
 {
     const uint32_t u = __float_as_uint(x + 0.0f);   // -0 -> +0
@@ -106,7 +119,10 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
 
     extern __shared__ __align__(16) uint32_t keys_all[];         // [CL*chunk] keys of all blocks (used in CTA 0)
     __shared__ float qbar[128];
-    __shared__ uint32_t hist[4][256];
+    __shared__ uint32_t hist[4][kHistSlots];
+    __shared__ unsigned long long cand[kFastCap];   // (key, ~block index) of the keys at the boundary (fast path)
+    __shared__ uint32_t cand_n;
+    __shared__ uint32_t pass_bin[3];               // boundary bin of a radix pass: index, keys still to take in it, its size
     __shared__ uint32_t warp_sel[kWarps], warp_eq[kWarps];
     __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: one arrival per CTA of the cluster
 
@@ -118,7 +134,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         svk::mbar_init(svk::smem_u32(&keys_ready), CL);
         svk::mbar_fence_init();
     }
-    for (int i = tid; i < 4 * 256; i += kThreads) (&hist[0][0])[i] = 0;
+    for (int i = tid; i < 4 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
     SEL_STAMP(10);
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // before any global request is in flight
     SEL_STAMP(11);
@@ -214,76 +230,235 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) return;   // gave up: leave the output untouched
     SEL_STAMP(5);
 
-    // exact radix select of the N-th largest key: up to 4 passes of 8 bits, one histogram per pass.  Every
-    // warp scans the histogram itself (one block barrier per pass), and the passes stop as soon as the
-    // boundary bin is taken whole (then every key with the prefix found so far is kept).
-    uint32_t prefix = 0, mask = 0, remaining = (uint32_t)N;
+    // ---- fast path (up to kFastChunks * 512 blocks, scores not all equal) -----------------------------------
+    // The scores of one (sequence, KV head) are mapped linearly onto 0..65535 (monotone in the score, so the
+    // order is kept; equal codes are possible, equal scores are not split).  One histogram pass over the upper
+    // 8 bits of the code finds the boundary bin: unlike the raw float bits, the codes spread over all 256 bins,
+    // so plain shared-memory atomics rarely collide and the boundary bin holds only a few keys.  Those few are
+    // ranked against one another by their exact keys (ties: smaller block index first), which settles the
+    // selection exactly.  A boundary bin with more than kFastCap keys (outliers stretching the range) falls
+    // through to the general radix select below.
+    if (nb <= kFastChunks * kThreads) {
+        uint32_t kk[kFastChunks], kmin = 0xFFFFFFFFu, kmax = 0u;
+#pragma unroll
+        for (int c = 0; c < kFastChunks; ++c) {
+            const int bb = c * kThreads + tid;
+            kk[c] = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
+            if (kk[c] != 0xFFFFFFFFu) kmin = min(kmin, kk[c]), kmax = max(kmax, kk[c]);
+        }
+        kmin = __reduce_min_sync(0xffffffffu, kmin);
+        kmax = __reduce_max_sync(0xffffffffu, kmax);
+        if (lane == 0) warp_sel[warp] = kmin, warp_eq[warp] = kmax;
+        if (tid == 0) cand_n = 0;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) kmin = min(kmin, warp_sel[w]), kmax = max(kmax, warp_eq[w]);
+        const float xmin = key_score(kmin), xmax = key_score(kmax);
+        const float scale = 65535.f / (xmax - xmin);
+        const uint32_t R = (uint32_t)(N - forced);   // evictable blocks to keep: 0 <= R < number of evictable blocks
+        if (kmin < kmax && scale > 0.f && scale < 3.0e38f) {   // block-uniform
+            uint32_t q[kFastChunks];   // 16-bit code of the score; 0x10000 = forced or absent
+#pragma unroll
+            for (int c = 0; c < kFastChunks; ++c)
+                q[c] = kk[c] == 0xFFFFFFFFu ? 0x10000u : min(65535u, (uint32_t)((key_score(kk[c]) - xmin) * scale));
+            // level 0: upper byte of the code over all evictable keys; level 1 (only when the boundary bin of
+            // level 0 is too crowded to rank directly): lower byte over the keys of that bin
+            uint32_t bound = 0x100u, need = R, in_bin = 0;   // boundary prefix of the code, keys to keep / present at it
+            int shift = 8;
+            bool settled = R == 0;   // nothing evictable is kept: every code is below the boundary 0x100
 #pragma unroll 1
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        // one shared-memory atomic per distinct digit per warp (scores share their leading bits, so
-        // un-aggregated atomics would pile onto a single bin)
+            for (int lvl = 0; lvl < 2 && !settled; ++lvl) {
+                shift = 8 - 8 * lvl;
+#pragma unroll
+                for (int c = 0; c < kFastChunks; ++c)
+                    if (q[c] < 0x10000u && (lvl == 0 || (q[c] >> 8) == bound))
+                        atomicAdd(&hist[lvl][hist_slot((q[c] >> shift) & 255u)], 1u);
+                __syncthreads();
+                if (warp == 0) {   // lane j owns bins 255-8j .. 248-8j (descending)
+                    uint32_t c8[8], tot = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        c8[i] = hist[lvl][hist_slot(255 - 8 * lane - i)];
+                        tot += c8[i];
+                    }
+                    uint32_t incl = tot;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += v;
+                    }
+                    uint32_t above = incl - tot;
+                    if (above < need && need <= incl) {   // exactly one lane
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (above < need && need <= above + c8[i]) {
+                                pass_bin[0] = 255 - 8 * lane - i;
+                                pass_bin[1] = need - above;
+                                pass_bin[2] = c8[i];
+                            }
+                            above += c8[i];
+                        }
+                    }
+                }
+                __syncthreads();
+                bound = lvl == 0 ? pass_bin[0] : ((bound << 8) | pass_bin[0]);
+                need = pass_bin[1];
+                in_bin = pass_bin[2];
+                settled = need == in_bin || in_bin <= (uint32_t)kFastCap;
+                __syncthreads();   // pass_bin is rewritten by the next level
+            }
+            if (settled) {   // block-uniform
+                const bool rank_them = need < in_bin;   // otherwise every key at the boundary prefix is kept
+                if (rank_them) {
+                    // the few keys at the boundary: order them exactly, by key, ties by smaller block index
+#pragma unroll
+                    for (int c = 0; c < kFastChunks; ++c)
+                        if ((q[c] >> shift) == bound) {
+                            const uint32_t bb = (uint32_t)(c * kThreads + tid);
+                            cand[atomicAdd(&cand_n, 1u)] = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
+                        }
+                    __syncthreads();
+                }
+                bool sel[kFastChunks];
+#pragma unroll
+                for (int c = 0; c < kFastChunks; ++c) {
+                    const uint32_t bb = (uint32_t)(c * kThreads + tid);
+                    const uint32_t pc = q[c] >> shift;   // forced / absent: 0x10000 >> shift is above every boundary
+                    sel[c] = bb < (uint32_t)nb && pc > bound;
+                    if (bb < (uint32_t)nb && pc == bound) {
+                        sel[c] = true;
+                        if (rank_them) {
+                            const unsigned long long mine = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
+                            uint32_t rk = 0;
+#pragma unroll 4
+                            for (uint32_t t = 0; t < in_bin; ++t) rk += cand[t] > mine ? 1u : 0u;
+                            sel[c] = rk < need;
+                        }
+                    }
+                }
+                SEL_STAMP(7);
+                // ascending compaction
+                uint32_t base = 0;
+#pragma unroll
+                for (int c = 0; c < kFastChunks; ++c) {
+                    if (c * kThreads < nb) {   // block-uniform
+                        const uint32_t ballot = __ballot_sync(0xffffffffu, sel[c]);
+                        if (lane == 0) warp_sel[warp] = __popc(ballot);
+                        __syncthreads();
+                        uint32_t before = 0, total = 0;
+#pragma unroll
+                        for (int w = 0; w < kWarps; ++w) {
+                            const uint32_t v = warp_sel[w];
+                            if (w < warp) before += v;
+                            total += v;
+                        }
+                        if (sel[c]) out[base + before + __popc(ballot & ((1u << lane) - 1u))] = c * kThreads + tid;
+                        base += total;
+                        __syncthreads();
+                    }
+                }
+                if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
+                SEL_STAMP(8);
+                return;
+            }
+            // fall through: the fast path used hist[0] and hist[1]; clear them for the radix passes
+            for (int i = tid; i < 2 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
+            __syncthreads();
+        }
+    }
+
+    // Exact radix select of the boundary key among the evictable blocks (the forced ones carry 0xFFFFFFFF and
+    // are kept without taking part).  The keys of one (sequence, KV head) share their leading bits (same sign,
+    // neighbouring exponents), so the digits start at the highest bit in which any two keys differ: the first
+    // 8-bit pass then spreads the keys over the bins (shared-memory atomics rarely collide) and usually leaves a
+    // boundary bin of a few keys, so that the second pass ends the search.  Every warp scans the histogram itself
+    // (one block barrier per pass); the passes stop as soon as the boundary bin is taken whole.
+    uint32_t k_and = 0xFFFFFFFFu, k_or = 0u;
+    for (int c0 = 0; c0 < nb; c0 += kThreads) {
+        const int bb = c0 + tid;
+        const uint32_t k = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
+        if (k != 0xFFFFFFFFu) k_and &= k, k_or |= k;
+    }
+    k_and = __reduce_and_sync(0xffffffffu, k_and);
+    k_or = __reduce_or_sync(0xffffffffu, k_or);
+    if (lane == 0) warp_sel[warp] = k_and, warp_eq[warp] = k_or;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) k_and &= warp_sel[w], k_or |= warp_eq[w];
+    __syncthreads();   // warp_sel / warp_eq are reused by the compaction
+    const uint32_t diff = k_and ^ k_or;
+    uint32_t remaining = (uint32_t)(N - forced);        // evictable blocks to keep (N < nb here, so fewer than there are)
+    int lo = diff ? 32 - __clz(diff) : 0;               // undecided low bits
+    uint32_t mask = lo == 32 ? 0u : ~((1u << lo) - 1u); // bits decided so far: the common leading bits
+    uint32_t prefix = k_and & mask;
+#pragma unroll 1
+    for (int pass = 0; pass < 4 && lo > 0 && remaining > 0; ++pass) {
+        const int width = min(8, lo), shift = lo - width;
+        const uint32_t dmask = (1u << width) - 1u;
         for (int c0 = 0; c0 < nb; c0 += kThreads) {
             const int bb = c0 + tid;
-            const uint32_t k = bb < nb ? keys_all[bb] : 0u;
-            const bool cand = bb < nb && (k & mask) == prefix;
-            const uint32_t digit = cand ? ((k >> shift) & 255u) : 256u;
+            const uint32_t k = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
+            const bool cand = k != 0xFFFFFFFFu && (k & mask) == prefix;
+            // one shared-memory atomic per distinct digit per warp: keys of similar magnitude pile onto few bins
+            const uint32_t digit = cand ? ((k >> shift) & dmask) : 256u;
             const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-            if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[pass][digit], (uint32_t)__popc(peers));
+            if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[pass][hist_slot(digit)], (uint32_t)__popc(peers));
         }
         __syncthreads();
-        // lane j owns bins 255-8j .. 248-8j (descending)
-        uint32_t c[8], tot = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            c[i] = hist[pass][255 - 8 * lane - i];
-            tot += c[i];
-        }
-        uint32_t incl = tot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        const uint32_t excl = incl - tot;
-        uint32_t found = 0;   // (bin << 16) | (bin count << 0 ... ) packed below
-        uint32_t bin = 0, rem_in_bin = 0, bin_count = 0;
-        if (excl < remaining && remaining <= incl) {   // exactly one lane
-            uint32_t above = excl;
+        // warp 0 scans the histogram (the other warps would only compete for issue slots) and publishes the
+        // boundary bin; lane j owns bins 255-8j .. 248-8j (descending)
+        if (warp == 0) {
+            uint32_t c[8], tot = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                if (above < remaining && remaining <= above + c[i]) {
-                    bin = 255 - 8 * lane - i;
-                    rem_in_bin = remaining - above;
-                    bin_count = c[i];
-                    found = 1;
+                c[i] = hist[pass][hist_slot(255 - 8 * lane - i)];
+                tot += c[i];
+            }
+            uint32_t incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const uint32_t excl = incl - tot;
+            if (excl < remaining && remaining <= incl) {   // exactly one lane
+                uint32_t above = excl;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (above < remaining && remaining <= above + c[i]) {
+                        pass_bin[0] = 255 - 8 * lane - i;
+                        pass_bin[1] = remaining - above;
+                        pass_bin[2] = c[i];
+                    }
+                    above += c[i];
                 }
-                above += c[i];
             }
         }
-        const uint32_t src = __ffs(__ballot_sync(0xffffffffu, found != 0)) - 1;
-        bin = __shfl_sync(0xffffffffu, bin, src);
-        rem_in_bin = __shfl_sync(0xffffffffu, rem_in_bin, src);
-        bin_count = __shfl_sync(0xffffffffu, bin_count, src);
+        __syncthreads();
+        const uint32_t bin = pass_bin[0], rem_in_bin = pass_bin[1], bin_count = pass_bin[2];
+        // (pass_bin is rewritten only after the next pass's barrier)
         prefix |= bin << shift;
-        mask |= 0xFFu << shift;
+        mask |= dmask << shift;
         remaining = rem_in_bin;
+        lo = shift;
         SEL_STAMP(14 + pass);
-        if (remaining == bin_count) break;   // the whole boundary bin is kept: lower digits cannot matter
+        if (remaining == bin_count) break;   // the whole boundary bin is kept: lower bits cannot matter
     }
-    // keys whose masked part exceeds the prefix are kept; of those equal to it, the first `remaining` in
-    // index order (all of them after an early stop)
+    // evictable keys whose decided bits exceed the prefix are kept; of those equal to it, the first `remaining`
+    // in index order (all of them after an early stop, none when only the forced blocks fit the budget)
     SEL_STAMP(7);
-    const uint32_t thr = prefix;          // N-th largest key (its bits under the mask)
-    const uint32_t take_eq = remaining;   // how many keys equal to thr under the mask are kept (smallest indices first)
+    const uint32_t thr = prefix;
+    const uint32_t take_eq = remaining;
 
     // ascending compaction
     uint32_t base_sel = 0, base_eq = 0;
     for (int c0 = 0; c0 < nb; c0 += kThreads) {
         const int bb = c0 + tid;
-        const uint32_t k = bb < nb ? (keys_all[bb] & mask) : 0u;
-        const bool gt = bb < nb && k > thr;
-        const bool eq = bb < nb && k == thr;
+        const uint32_t key = bb < nb ? keys_all[bb] : 0u;
+        const bool is_forced = bb < nb && key == 0xFFFFFFFFu;
+        const uint32_t k = key & mask;
+        const bool gt = is_forced || (bb < nb && k > thr);
+        const bool eq = bb < nb && !is_forced && k == thr;
         const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
         const uint32_t gt_ballot = __ballot_sync(0xffffffffu, gt);
         if (lane == 0) {
@@ -350,8 +525,11 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     if (n_sink + n_local > max_sel) return SV_ERR_BUDGET;
     if (geom->max_blocks > svh::kMaxBlocksSelect) return SV_ERR_UNSUPPORTED;
 
+    // CTAs per (sequence, KV head): at least 32 blocks each, and no more CTAs than two per SM can hold at once
+    // (512 threads x 60 registers: two CTAs per SM) -- a second wave costs more than the shorter slices save
+    const int pairs = geom->n_seq * geom->n_kv_heads;
     int CL = 1;
-    while (CL < 8 && geom->max_blocks / (CL * 2) >= 32) CL *= 2;
+    while (CL < 8 && geom->max_blocks / (CL * 2) >= 32 && pairs * CL * 2 <= 2 * svh::sm_count()) CL *= 2;
     const int per = (geom->max_blocks + CL - 1) / CL;
     const int chunk = (per + kWarps * kRowsPerIter - 1) / (kWarps * kRowsPerIter) * (kWarps * kRowsPerIter);
 

@@ -48,6 +48,21 @@ inline void pdl_attribute(cudaLaunchAttribute *attr)
     attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;
 }
 
+// SMs of the current device (148 when there is no device to ask).
+inline int sm_count()
+{
+    static const int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
+            v = 148;
+        }
+        return v;
+    }();
+    return n;
+}
+
 inline sv_status launch_status()
 {
     return cudaGetLastError() == cudaSuccess ? SV_OK : SV_ERR_CUDA;

@@ -611,17 +611,7 @@ bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
     return true;
 }
 
-int sm_count()
-{
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
-            v = 148;
-        return v;
-    }();
-    return n;
-}
+using svh::sm_count;
 
 // Blocks per CTA are minimised subject to one CTA per SM; then the fewest splits that achieve it.
 int choose_splits(const sv_geom *g, int n_blocks)
