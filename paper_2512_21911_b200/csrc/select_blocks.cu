@@ -12,6 +12,8 @@
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "sv_host.h"
 #include "sv_ptx.cuh"
 
@@ -46,7 +48,6 @@ constexpr int kRowsPerIter = 4;   // independent representative rows a warp has 
 // Histogram bin -> shared-memory slot: one pad word per 32 bins, so that a warp whose lane j reads bins
 // 8j .. 8j+7 (the scan below) touches 32 different banks with every load.
 constexpr int kHistSlots = 256 + 8;
-constexpr int kFastChunks = 4;   // fast selection path: up to 4 keys per thread (2048 blocks)
 constexpr int kFastCap = 32;     // ... and at most this many keys left at the boundary after the histogram levels
 __device__ __forceinline__ uint32_t hist_slot(uint32_t bin) { return bin + (bin >> 5); }
 
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) return;   // gave up: leave the output untouched
     SEL_STAMP(5);
 
-    // ---- fast path (up to kFastChunks * 512 blocks, scores not all equal) -----------------------------------
+    // ---- fast path (up to 2048 blocks = 4 keys per thread, scores not all equal) -----------------------------------
     // The scores of one (sequence, KV head) are mapped linearly onto 0..65535 (monotone in the score, so the
     // order is kept; equal codes are possible, equal scores are not split).  One histogram pass over the upper
     // 8 bits of the code finds the boundary bin: unlike the raw float bits, the codes spread over all 256 bins,
@@ -238,10 +239,12 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     // ranked against one another by their exact keys (ties: smaller block index first), which settles the
     // selection exactly.  A boundary bin with more than kFastCap keys (outliers stretching the range) falls
     // through to the general radix select below.
-    if (nb <= kFastChunks * kThreads) {
-        uint32_t kk[kFastChunks], kmin = 0xFFFFFFFFu, kmax = 0u;
+    // NC = keys per thread (1, 2 or 4); returns true when the selection has been written
+    const auto fast_select = [&](auto nc_tag) -> bool {
+        constexpr int NC = decltype(nc_tag)::value;
+        uint32_t kk[NC], kmin = 0xFFFFFFFFu, kmax = 0u;
 #pragma unroll
-        for (int c = 0; c < kFastChunks; ++c) {
+        for (int c = 0; c < NC; ++c) {
             const int bb = c * kThreads + tid;
             kk[c] = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
             if (kk[c] != 0xFFFFFFFFu) kmin = min(kmin, kk[c]), kmax = max(kmax, kk[c]);
@@ -257,9 +260,9 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         const float scale = 65535.f / (xmax - xmin);
         const uint32_t R = (uint32_t)(N - forced);   // evictable blocks to keep: 0 <= R < number of evictable blocks
         if (kmin < kmax && scale > 0.f && scale < 3.0e38f) {   // block-uniform
-            uint32_t q[kFastChunks];   // 16-bit code of the score; 0x10000 = forced or absent
+            uint32_t q[NC];   // 16-bit code of the score; 0x10000 = forced or absent
 #pragma unroll
-            for (int c = 0; c < kFastChunks; ++c)
+            for (int c = 0; c < NC; ++c)
                 q[c] = kk[c] == 0xFFFFFFFFu ? 0x10000u : min(65535u, (uint32_t)((key_score(kk[c]) - xmin) * scale));
             // level 0: upper byte of the code over all evictable keys; level 1 (only when the boundary bin of
             // level 0 is too crowded to rank directly): lower byte over the keys of that bin
@@ -270,7 +273,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
             for (int lvl = 0; lvl < 2 && !settled; ++lvl) {
                 shift = 8 - 8 * lvl;
 #pragma unroll
-                for (int c = 0; c < kFastChunks; ++c)
+                for (int c = 0; c < NC; ++c)
                     if (q[c] < 0x10000u && (lvl == 0 || (q[c] >> 8) == bound))
                         atomicAdd(&hist[lvl][hist_slot((q[c] >> shift) & 255u)], 1u);
                 __syncthreads();
@@ -312,16 +315,16 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                 if (rank_them) {
                     // the few keys at the boundary: order them exactly, by key, ties by smaller block index
 #pragma unroll
-                    for (int c = 0; c < kFastChunks; ++c)
+                    for (int c = 0; c < NC; ++c)
                         if ((q[c] >> shift) == bound) {
                             const uint32_t bb = (uint32_t)(c * kThreads + tid);
                             cand[atomicAdd(&cand_n, 1u)] = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
                         }
                     __syncthreads();
                 }
-                bool sel[kFastChunks];
+                bool sel[NC];
 #pragma unroll
-                for (int c = 0; c < kFastChunks; ++c) {
+                for (int c = 0; c < NC; ++c) {
                     const uint32_t bb = (uint32_t)(c * kThreads + tid);
                     const uint32_t pc = q[c] >> shift;   // forced / absent: 0x10000 >> shift is above every boundary
                     sel[c] = bb < (uint32_t)nb && pc > bound;
@@ -340,7 +343,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                 // ascending compaction
                 uint32_t base = 0;
 #pragma unroll
-                for (int c = 0; c < kFastChunks; ++c) {
+                for (int c = 0; c < NC; ++c) {
                     if (c * kThreads < nb) {   // block-uniform
                         const uint32_t ballot = __ballot_sync(0xffffffffu, sel[c]);
                         if (lane == 0) warp_sel[warp] = __popc(ballot);
@@ -359,12 +362,20 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                 }
                 if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
                 SEL_STAMP(8);
-                return;
+                return true;
             }
             // fall through: the fast path used hist[0] and hist[1]; clear them for the radix passes
             for (int i = tid; i < 2 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
             __syncthreads();
         }
+        return false;
+    };
+    if (nb <= kThreads) {
+        if (fast_select(std::integral_constant<int, 1>{})) return;
+    } else if (nb <= 2 * kThreads) {
+        if (fast_select(std::integral_constant<int, 2>{})) return;
+    } else if (nb <= 4 * kThreads) {
+        if (fast_select(std::integral_constant<int, 4>{})) return;
     }
 
     // Exact radix select of the boundary key among the evictable blocks (the forced ones carry 0xFFFFFFFF and
