@@ -56,16 +56,16 @@ constexpr int kThreads = 384;
 constexpr int kUnit = 64;                        // keys per unit
 constexpr int kTile = kUnit * 128;               // bytes of one [64 rows][64 bf16] half tile (8 KB)
 constexpr int kStageBytes = 4 * kTile;           // K lo/hi + V lo/hi
-constexpr int kStages = 4;
+constexpr int kStages = 5;
 constexpr int kQBytes = 2 * 128 * 128;           // Q: two halves [128 rows][64 bf16]
 constexpr int kPBytes = 128 * 128;               // P: [128 rows][64 bf16]
 constexpr int kOffQ = kStages * kStageBytes;
 constexpr int kOffP = kOffQ + kQBytes;
-constexpr int kOffDraft = kOffP + 2 * kPBytes;   // draft unit: same layout as a stage
-constexpr int kOffMisc = kOffDraft + kStageBytes;
+constexpr int kOffDraft = 0;                     // the draft unit is the first occupant of ring stage 0 (last split only)
+constexpr int kOffMisc = kOffP + 2 * kPBytes;
 constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
-static_assert(20 <= 32, "one lane of the producer warp per barrier");
+static_assert(2 * kStages + 10 <= 32, "one lane of the producer warp per barrier");
 constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns
 constexpr int kMergeStride = 132;                // floats per row of the cross-warpgroup merge buffer
 
@@ -155,6 +155,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
             const int j0 = (int)((long long)split * n_sel / p.splits);
             const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+            const int off = has_draft ? 1 : 0;
             bool dead = false;
             for (int base = j0; base < j1; base += 32) {
                 const int j = base + lane;
@@ -174,8 +175,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const int t0 = __shfl_sync(0xffffffffu, tok0, i);
                     if (lane == 0 && !dead) {
                         for (int uo = 0; uo < upb; ++uo) {
-                            const int u = (base - j0 + i) * upb + uo;
-                            const int stage = u % kStages, it = u / kStages;
+                            const int u = (base - j0 + i) * upb + uo;   // ring unit; the draft unit (if any) came first
+                            const int stage = (u + off) % kStages, it = (u + off) / kStages;
                             if (it > 0 && (*abort_flag || !mbar_wait_bounded(bar(kEmpty + stage), (it - 1) & 1))) {
                                 dead = true;
                                 *abort_flag = 1;
@@ -221,10 +222,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint64_t d_hi = dq & 0xFFFFFFFF00000000ull;
                     for (int u = 0; u < n_total && !dead; ++u) {
                         const int g = u & 1, k = u >> 1;
-                        const bool ring = u >= off;
-                        const int stage = ring ? (u - off) % kStages : 0;
-                        const int it = ring ? (u - off) / kStages : 0;
-                        if (*abort_flag || (ring && !mbar_wait_bounded(bar(kFull + stage), it & 1)) ||
+                        const int stage = u % kStages, it = u / kStages;
+                        if (*abort_flag || !mbar_wait_bounded(bar(kFull + stage), it & 1) ||
                             (k > 0 && !mbar_wait_bounded(bar(kSFree + g), (k - 1) & 1))) {
                             dead = true;
                             *abort_flag = 1;
@@ -232,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             break;
                         }
                         tc_fence_after_sync();
-                        const uint32_t k_lo = dk_lo + (uint32_t)((ring ? stage * kStageBytes : kOffDraft) >> 4);
+                        const uint32_t k_lo = dk_lo + (uint32_t)((stage * kStageBytes) >> 4);
                         const uint32_t d = tmem_base + g * kUnit;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
@@ -253,8 +252,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint64_t dp_hi = dp & 0xFFFFFFFF00000000ull, dv_hi = dv & 0xFFFFFFFF00000000ull;
                     for (int u = 0; u < n_total && !dead; ++u) {
                         const int g = u & 1, k = u >> 1;
-                        const bool ring = u >= off;
-                        const int stage = ring ? (u - off) % kStages : 0;
+                        const int stage = u % kStages;
                         if (*abort_flag || !mbar_wait_bounded(bar(kPReady + g), k & 1)) {
                             dead = true;
                             *abort_flag = 1;
@@ -262,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             break;
                         }
                         tc_fence_after_sync();
-                        const uint32_t v_lo = dv_lo + (uint32_t)((ring ? stage * kStageBytes : kOffDraft) >> 4);
+                        const uint32_t v_lo = dv_lo + (uint32_t)((stage * kStageBytes) >> 4);
                         const uint32_t p_lo = dp_lo + (uint32_t)((g * kPBytes) >> 4);
                         const uint32_t d = tmem_base + 128 + g * 128;
 #pragma unroll
@@ -270,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             tc_mma_bf16(d, dp_hi | (p_lo + (uint32_t)((kk * 32) >> 4)), dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)),
                                         idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);   // the warpgroup's first unit starts O
                         tc_commit(bar(kOReady + g));
-                        if (ring) tc_commit(bar(kEmpty + stage));
+                        tc_commit(bar(kEmpty + stage));
                         if (u < 24) TC_STAMP(56 + u);
                     }
                 }
@@ -378,6 +376,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     fence_proxy_async();   // the tensor cores read these tiles through the async proxy
     named_bar_sync(2, 256);
     if (lane == 0) mbar_arrive(bar(kStaged));
+    if (has_draft && tid == 0) mbar_arrive(bar(kFull + 0));   // the draft unit fills stage 0 in place of a TMA load
     if (tid == 0) TC_STAMP(2);
 
     const int wg = warp >> 2, quad = warp & 3;
@@ -444,7 +443,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (lane == 0) mbar_arrive(bar(kSFree + wg));   // the next S of this warpgroup may be issued
 
         const bool is_draft = u < off;
-        const int stage = is_draft ? 0 : (u - off) % kStages;
+        const int stage = u % kStages;
         const int nvalid = is_draft ? p.T : min(meta[stage], kUnit);
         uint8_t *pbuf = smem + kOffP + wg * kPBytes;
         float sc[NH][16], factor[NH];
