@@ -2,8 +2,9 @@
 
 A thin driver over the C-ABI calls: it owns the per-layer representatives, the shared block list,
 the split-KV workspace and the outputs, and enqueues, per layer, ``sv_select_blocks`` (anchor
-layers) or the reuse of the previous layer's list (Eq. 9), then ``sv_verify_attn``.  All compute is in
-the library's kernels; this class only holds buffers and calls them in order.
+layers) or the reuse of the previous layer's list (Eq. 9), then ``sv_verify_attn``; after verification,
+``accept`` (Eq. 2-3) and ``commit`` (append the kept rows to the cache) close the decoding step.  All compute
+is in the library's kernels; this class only holds buffers and calls them in order.
 """
 from __future__ import annotations
 
@@ -102,6 +103,30 @@ class SparseVerifier:
                         sv.sv_block_reps(self.geom, self.kv[l], self.reps[l], sv.SV_TAIL_BLOCK)
         for l in range(self.n_layers):
             self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l])
+
+    def accept(self, p_target, p_draft, tokens, u_accept, u_next):
+        """Acceptance of the step's draft tokens (Eq. 2-3).  Returns (path [S][T], n_path [S], next_token [S]):
+        the rows whose K/V enter the cache (root first) and the token drawn after the kept path."""
+        S, T = int(self.geom.n_seq), int(self.geom.n_draft)
+        dev = p_target.device
+        path = torch.empty((S, T), dtype=torch.int32, device=dev)
+        n_path = torch.empty((S,), dtype=torch.int32, device=dev)
+        next_token = torch.empty((S,), dtype=torch.int32, device=dev)
+        sv.sv_accept(p_target, p_draft, tokens, self.parent, u_accept, u_next, path, n_path, next_token)
+        return path, n_path, next_token
+
+    def commit(self, draft_k, draft_v, path, n_path) -> None:
+        """Append the kept rows' K/V of every layer to the paged cache (one sv_kv_append per layer, which also
+        refreshes the representatives of the blocks that grew) and advance the sequence lengths.  The block table
+        must already hold pages for the blocks the sequences grow into.  draft_k/v: [layers][S][T][Hkv][D]."""
+        new_len = torch.empty_like(self.seq_lens)
+        for l in range(self.n_layers):
+            k_pool, v_pool = self._pools[l]
+            sv.sv_kv_append(self.geom, k_pool, v_pool, self.block_table, self.seq_lens, draft_k[l], draft_v[l], path,
+                            n_path, new_len, self.reps[l])
+        self.seq_lens.copy_(new_len)          # every layer has read the old lengths by now (same stream)
+        if self._stack_kv is not None:
+            self._stack_lens.copy_(self.seq_lens.repeat(self.n_layers))
 
     def dense_step(self, q, draft_k, draft_v, out) -> None:
         for l in range(self.n_layers):

@@ -853,3 +853,68 @@ def test_bf16_representatives_parity(sv, name):
                 assert all(b_ in (0, nb - 1) or sc_o[s, h, b_] >= free[k - 1] - 2.5 * err - 1e-12 for b_ in got)
     assert n_diff <= max(2, n_val // 2000), (n_diff, n_val)
     assert exact >= (S * Hkv * 3) // 4
+
+
+def test_engine_two_decoding_steps(sv):
+    """SparseVerifier over a 2-layer stack: verify -> accept -> commit -> verify again.  The second step's block
+    lists and attention must equal the oracle's on the cache the oracle itself appended to."""
+    n_layers = 2
+    w = si.shrink(SMALL["cfg2_small"], n_draft=6, n_layers=n_layers)
+    geom = si.make_geometry(w)
+    layers = [si.make_layer(geom, layer=l) for l in range(n_layers)]
+    S, Hkv, Hq, T, B = w.n_seq, w.n_kv_heads, w.n_q_heads, w.n_draft, w.block_size
+    c0 = layers[0]
+    bt = np.concatenate([c0["block_table"], np.zeros((S, 1), np.int32)], axis=1)      # room to grow into
+    for s in range(S):
+        bt[s, c0["n_blocks"][s]] = c0["n_pages"] + s
+    NB, max_sel = bt.shape[1], geom["max_sel"]
+    pad = np.zeros((S,) + c0["k_pool"].shape[1:], np.uint16)
+    pools = [(np.concatenate([c["k_pool"], pad]), np.concatenate([c["v_pool"], pad])) for c in layers]
+    lens = c0["seq_lens"].copy()
+    eng = sv.SparseVerifier(n_seq=S, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=128, block_size=B, max_blocks=NB, n_draft=T,
+                            n_layers=n_layers, block_table=torch.from_numpy(bt).cuda(), seq_lens=torch.from_numpy(lens).cuda(),
+                            budget_blocks=torch.from_numpy(c0["budget"]).cuda(), max_sel=max_sel, n_sink=1, n_local=1)
+    k_all = torch.stack([bf16_dev(k) for k, _ in pools]).contiguous()
+    v_all = torch.stack([bf16_dev(v) for _, v in pools]).contiguous()
+    eng.set_kv_stack(k_all, v_all)
+    for l in range(n_layers):
+        eng.build_reps(l)
+    stack = lambda key: torch.stack([bf16_dev(c[key]) for c in layers]).contiguous()
+    q, dk, dv = stack("q"), stack("draft_k"), stack("draft_v")
+    out = torch.zeros_like(q)
+    eng.verify_step(q, dk, dv, out)
+    a = si.make_accept_case(S, T, 2048, seed=91)
+    ra = _settle_accept_case(a)
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    path, n_path, nxt = eng.accept(dev(a["p_target"]), dev(a["p_draft"]), dev(a["tokens"]), dev(a["u_accept"]), dev(a["u_next"]))
+    eng.commit(dk, dv, path, n_path)
+    torch.cuda.synchronize()
+    assert int(eng.status.item()) == 0
+    np.testing.assert_array_equal(path.cpu().numpy(), ra["path"])
+    # the oracle's copy of the step
+    new_lens = None
+    for l, c in enumerate(layers):
+        ko, vo = pools[l]
+        new_lens = oracle.kv_append(ko, vo, bt, lens, c["draft_k"], c["draft_v"], ra["path"], ra["n_path"], None)
+    np.testing.assert_array_equal(eng.seq_lens.cpu().numpy(), new_lens)
+    # second step: fresh queries and draft tokens (layer data of another seed), same budgets
+    layers2 = [si.make_layer(geom, layer=10 + l) for l in range(n_layers)]
+    stack2 = lambda key: torch.stack([bf16_dev(c[key]) for c in layers2]).contiguous()
+    q2, dk2, dv2 = stack2("q"), stack2("draft_k"), stack2("draft_v")
+    out2 = torch.zeros_like(q2)
+    lse2 = torch.zeros((S, T, Hq), device="cuda")
+    for l in range(n_layers):
+        eng.verify_layer(l, q2[l], dk2[l], dv2[l], out2[l], lse=lse2)
+        torch.cuda.synchronize()
+        ko, vo = pools[l]
+        idx_o, cnt_o, sc_o = oracle.select_blocks(layers2[l]["q"], ko, bt, new_lens, c0["budget"], 1, 1, max_sel)
+        idx_g, cnt_g = eng.sel_idx.cpu().numpy(), eng.sel_cnt.cpu().numpy()
+        np.testing.assert_array_equal(cnt_g, cnt_o)
+        # the second step's queries were gap-repaired against the un-appended cache: demand the same sets except
+        # at most a couple of boundary blocks, and compare the attention on the GPU's own lists
+        differ = sum(int(set(idx_g[s, h, :cnt_g[s, h]]) != set(idx_o[s, h, :cnt_o[s, h]])) for s in range(S) for h in range(Hkv))
+        assert differ <= max(1, S * Hkv // 20), differ
+        o_ref, lse_ref = oracle.verify_attn(layers2[l]["q"], ko, vo, bt, new_lens, layers2[l]["draft_k"], layers2[l]["draft_v"],
+                                            None, idx_g, cnt_g)
+        check_attn(bf16_host(out2[l]), lse2.cpu().numpy().astype(np.float64), o_ref, lse_ref, f"second step, layer {l}")
+    assert int(eng.status.item()) == 0
