@@ -123,6 +123,7 @@ def run_pipeline(sv, c, n_sink=None, n_local=None, what=""):
 SMALL = {
     # rows = G*T: 16 (1 warp row), 32, 20 (ragged batch), 64, 128 (block 128, tree)
     "cfg0": si.WORKLOADS["cfg0"],
+    "cfg1_full": si.shrink(si.WORKLOADS["cfg1"], n_layers=1),      # the benchmark's layer shape, for the variant tests
     "cfg1_small": si.shrink(si.WORKLOADS["cfg1"], seq_len=(4096, 4096), budget_blocks=20, n_layers=1),
     "cfg2_small": si.shrink(si.WORKLOADS["cfg2"], n_seq=5, seq_len=(700, 3000), budget_blocks=9),
     "rows64": si.shrink(si.WORKLOADS["cfg1"], seq_len=(2500, 2500), budget_blocks=12, n_draft=16, n_layers=1, tree=True),
@@ -550,7 +551,7 @@ def _boundary_gap_global(sc, nb, total, n_sink, n_local):
     return srt[k - 1] - srt[k]
 
 
-@pytest.mark.parametrize("name", ["cfg0", "cfg1_small", "cfg2_small", "cfg3_small"])
+@pytest.mark.parametrize("name", ["cfg0", "cfg1_small", "cfg2_small", "cfg3_small", "cfg1_full"])
 def test_select_global_parity(sv, name):
     """Budget shared by the KV heads: lists bit-exact against the oracle wherever the fp32 scores leave no doubt
     about the boundary pair (checked in the oracle's fp64 scores); counts always add up to budget * Hkv."""
@@ -626,7 +627,7 @@ def test_select_global_ties_and_degenerate_budgets(sv):
         sv.sv_select_blocks_global(d.geom, d.q, d.reps, d.seq_lens, d.budget, 1, 1, idx[:, :, :NB - 1].contiguous(), cnt, sc)
 
 
-@pytest.mark.parametrize("name", ["cfg0", "cfg2_small", "cfg3_small"])
+@pytest.mark.parametrize("name", ["cfg0", "cfg2_small", "cfg3_small", "cfg1_full"])
 def test_per_token_retrieval_and_overlap_parity(sv, name):
     """Every draft token retrieves with its own query; pair intersections bit-exact against the oracle on the
     lists the GPU produced, token 0 equal to the adopted strategy."""
@@ -806,7 +807,7 @@ def test_accept_feeds_kv_append(sv):
         np.testing.assert_allclose(rg[s, :, :nbn], reps_o[s, :, :nbn], rtol=0, atol=2e-6)
 
 
-@pytest.mark.parametrize("name", ["cfg0", "cfg1_small", "cfg2_small", "cfg3_small"])
+@pytest.mark.parametrize("name", ["cfg0", "cfg1_small", "cfg2_small", "cfg3_small", "cfg1_full"])
 def test_bf16_representatives_parity(sv, name):
     """Representatives stored in bfloat16: the GPU rounds its fp32 mean, the oracle its fp64 mean -- equal except
     where the two means straddle a rounding boundary (one bfloat16 step, rare); scores to fp32 accuracy of the
