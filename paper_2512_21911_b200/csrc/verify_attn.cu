@@ -502,11 +502,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 constexpr int kMergeThreads = 64;
 
 // Combine the per-split partials: o = sum_j 2^(m_j - m) o_j / sum_j 2^(m_j - m) l_j.
-// One thread per (row, 4 output dims).  The partials sit in L2; all loads of up to 16 splits are
+// One thread per (row, 4 output dims).  The partials sit in L2; all loads of up to 20 splits are
 // issued before the first use so that the kernel costs one memory round trip, not one per split.
 __global__ void __launch_bounds__(kMergeThreads) merge_splits_kernel(const AttnParams p)
 {
-    constexpr int U = 16;
+    constexpr int U = 20;   // 148 SMs / 8 KV heads = 18 splits still fit one batch
     const int h = blockIdx.y, s = blockIdx.z;
     const int rows = p.G * p.T;
     const int idx = blockIdx.x * kMergeThreads + threadIdx.x;
