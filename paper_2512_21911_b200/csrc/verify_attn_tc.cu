@@ -20,6 +20,8 @@
 // each with its own S / P / O buffers; warp 8 is the TMA producer, one thread of warp 9 issues every
 // S = Q K^T (and the warp owns the TMEM allocation), one thread of warp 10 issues every O += P V.  The
 // third warpgroup gives its registers to the other two (setmaxnreg).  Everything is chained with mbarriers; tcgen05.commit signals MMA completion.
+// At the end warpgroup 0 reads both accumulators from TMEM (warp q of either warpgroup owns lane quadrant q),
+// merges them in registers and writes the rows (or the fp32 partial of its split) out.
 // All waits are bounded; a wait that gives up sets *status and the CTA drains and frees its TMEM.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -536,66 +538,71 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (lane == 0) mbar_arrive(bar(kPReady + wg));
         if (tid == 0 && k < 12) TC_STAMP(92 + k);
     }
-    // fetch this warp's rows of O: 32 output dims 8*jj + 2*qd + e (index 2*jj + e) per slot
-    float o[NH][32];
+    // ------------------------------------------------------------------ combine the two warpgroups, write out
+    // Warp q of either warpgroup owns TMEM lane quadrant q, so warpgroup 0 can read warpgroup 1's accumulator
+    // straight from TMEM: warpgroup 1 only waits for its last PV, leaves its (m, l) in its own (now idle) P tile and
+    // signals; warpgroup 0 fetches both accumulators, merges them in registers and writes the rows out.
+    const int n_sm = 2 * wg_threads;
+    const int t = quad * 32 + lane;
+    float *ml1 = reinterpret_cast<float *>(smem + kOffP + kPBytes);   // [2 * NH][128]: m, l of warpgroup 1's slots
+    if (k > 0) wait_pv(k - 1);   // this warpgroup's accumulator is complete
+    if (wg == 1) {
 #pragma unroll
-    for (int i = 0; i < NH; ++i)
-#pragma unroll
-        for (int d = 0; d < 32; ++d) o[i][d] = 0.f;
-    if (k > 0) {
-        wait_pv(k - 1);
-        if (!dead) {
-            if (tid == 0) TC_STAMP(104);
-#pragma unroll
-            for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo)
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t r[32];
-                    tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + c * 64, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-#pragma unroll
-                            for (int e = 0; e < 2; ++e) o[lo * 2 + hh][(c * 8 + j) * 2 + e] = __uint_as_float(r[4 * j + 2 * hh + e]);
-                }
+        for (int i = 0; i < NH; ++i) {
+            ml1[(2 * i) * 128 + t] = m[i];
+            ml1[(2 * i + 1) * 128 + t] = l[i];
         }
+        tc_fence_before_sync();
+        named_bar_arrive(1, n_sm);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kTmemDone));   // this warpgroup reads TMEM no more
+        return;
     }
+    if (tid == 0) TC_STAMP(104);
+    named_bar_sync(1, n_sm);
+    tc_fence_after_sync();
+    if (tid == 0) TC_STAMP(106);
+    const bool have0 = k > 0 && !dead, have1 = n_total >= 2;   // a warpgroup without units never wrote its accumulator
+    // this warp's rows of O: 32 output dims 8*jj + 2*qd + e (index 2*jj + e) per slot
+    float o[NH][32], w0[NH], w1[NH], row_m[NH], row_l[NH];
+#pragma unroll
+    for (int i = 0; i < NH; ++i) {
+        const float m1 = ml1[(2 * i) * 128 + t], l1 = ml1[(2 * i + 1) * 128 + t];
+        const float M = fmaxf(m[i], m1);
+        const float M_use = (M == -INFINITY) ? 0.f : M;
+        w0[i] = fast_exp2(m[i] - M_use), w1[i] = fast_exp2(m1 - M_use);
+        float lsum = w0[i] * l[i] + w1[i] * l1;
+        lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+        lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+        row_m[i] = M, row_l[i] = lsum;
+    }
+#pragma unroll
+    for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            uint32_t r0[32], r1[32];
+            if (have0) tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + c * 64, r0);
+            if (have1) tmem_ld_16x256b_x8(t_o + 128 + ((uint32_t)(lo * 16) << 16) + c * 64, r1);
+            tmem_ld_wait();
+#pragma unroll
+            for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int i = lo * 2 + hh, x = 4 * j + 2 * hh + e;
+                        const float a = have0 ? w0[i] * __uint_as_float(r0[x]) : 0.f;
+                        const float b = have1 ? w1[i] * __uint_as_float(r1[x]) : 0.f;
+                        o[i][(c * 8 + j) * 2 + e] = a + b;
+                    }
+        }
     if (tid == 0) TC_STAMP(105);
     tc_fence_before_sync();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar(kTmemDone));
-
-    // ------------------------------------------------------------------ merge the two warpgroups, write out
-    const int n_sm = 2 * wg_threads;
-    named_bar_sync(1, n_sm);   // both warpgroups are past their last unit: the ring is free
-    if (tid == 0) TC_STAMP(106);
-    float *mx_buf = reinterpret_cast<float *>(smem);             // [NH*34][128] floats, index k*128 + t
-    const int t = quad * 32 + lane;
-    if (wg == 1) {
-#pragma unroll
-        for (int i = 0; i < NH; ++i) {
-#pragma unroll
-            for (int d = 0; d < 32; ++d) mx_buf[(i * 34 + d) * 128 + t] = o[i][d];
-            mx_buf[(i * 34 + 32) * 128 + t] = m[i];
-            mx_buf[(i * 34 + 33) * 128 + t] = l[i];
-        }
-    }
-    named_bar_sync(1, n_sm);
-    if (tid == 0) TC_STAMP(107);
-    if (wg == 1) return;
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
-        const float m1 = mx_buf[(i * 34 + 32) * 128 + t], l1 = mx_buf[(i * 34 + 33) * 128 + t];
-        const float M = fmaxf(m[i], m1);
-        const float M_use = (M == -INFINITY) ? 0.f : M;
-        const float w0 = fast_exp2(m[i] - M_use), w1 = fast_exp2(m1 - M_use);
-        float lsum = w0 * l[i] + w1 * l1;
-        lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
-        lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-#pragma unroll
-        for (int d = 0; d < 32; ++d) o[i][d] = w0 * o[i][d] + w1 * mx_buf[(i * 34 + d) * 128 + t];
+        const float M = row_m[i], lsum = row_l[i];
         const int row = lrow[i];
         if (row >= rows) continue;
         if (p.splits == 1) {
