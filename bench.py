@@ -299,6 +299,9 @@ def run_gpu(args):
                                                 out[l], workspace=eng.workspace, status_word=eng.status)
                               for l in range(w.n_layers)])
     g_dense = capture(lambda: eng.dense_step(q, dk, dv, out))
+    # full rebuild of the block representatives of every layer (prefill-time cost; the step only refreshes tails)
+    reps_scratch = torch.empty_like(eng.reps[0])
+    g_reps = capture(lambda: [sv.sv_block_reps(eng.geom, eng.kv[l], reps_scratch) for l in range(w.n_layers)])
 
     sampler = ClockSampler(local)
     ms_step = time_replays(g_step, args.steps, max(args.warmup, 3), sampler=sampler)
@@ -306,6 +309,7 @@ def run_gpu(args):
     ms_reuse = time_replays(g_reuse, side, 3)
     ms_attn = time_replays(g_attn, side, 3)
     ms_dense = time_replays(g_dense, max(5, side // 4), 3)
+    ms_reps = time_replays(g_reps, max(5, side // 4), 3)
 
     # End to end: every step copies its inputs (Q, draft K/V of all layers) from pinned host memory and its
     # outputs back.  Two sets of device buffers and three streams (copy-in, compute, copy-out) let the copies of
@@ -366,8 +370,8 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e = (aggregate_over_ranks(x, world, allmax)[0]
-                                                    for x in (ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e))
+    ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e, ms_reps = (aggregate_over_ranks(x, world, allmax)[0]
+                                                             for x in (ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e, ms_reps))
 
     # algorithmic bytes of one sv_verify_attn launch (K+V of the kept tokens and draft tokens, Q in, O out)
     S, T, Hq, Hkv, D, B, N = w.n_seq, w.n_draft, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, w.budget_blocks
@@ -376,6 +380,7 @@ def run_gpu(args):
     attn_bytes = Hkv * (kv_tokens + S * T) * 2 * D * 2 + 2 * S * T * Hq * D * 2
     dense_bytes = Hkv * (int(geom["seq_lens"].sum()) + S * T) * 2 * D * 2 + 2 * S * T * Hq * D * 2
     peak, peak_kind = measured_peaks()
+    reps_bytes = Hkv * int(geom["seq_lens"].sum()) * D * 2 + S * Hkv * geom["max_blocks"] * D * 4
     us_attn = ms_attn * 1e3 / w.n_layers
     us_dense = ms_dense * 1e3 / w.n_layers
     achieved = attn_bytes / (us_attn * 1e-6) / 1e9
@@ -407,6 +412,11 @@ def run_gpu(args):
         "reuse_even_anchors": {"us_per_layer": ms_reuse * 1e3 / w.n_layers, "kernels_per_step": eng_reuse.kernels_per_step(True)},
         "dense_verify": {"us_per_layer": us_dense, "gbs": dense_bytes / (us_dense * 1e-6) / 1e9,
                          "frac": dense_bytes / (us_dense * 1e-6) / 1e9 / peak, "bytes_per_launch": dense_bytes},
+        "block_reps_rebuild": {"us_per_layer": ms_reps * 1e3 / w.n_layers, "bytes_per_launch": reps_bytes,
+                               "gbs": reps_bytes / (ms_reps * 1e-3 / w.n_layers) / 1e9,
+                               "frac": reps_bytes / (ms_reps * 1e-3 / w.n_layers) / 1e9 / peak,
+                               "note": "sv_block_reps over a whole layer (all K read once, fp32 means written); "
+                                       "32 layers = 2 GiB per replay, nothing found in L2"},
         "min_score_gap_over_delta": min_ratio,
     }
 
