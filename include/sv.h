@@ -15,6 +15,11 @@
  *                     and the draft tokens' own K/V                       (Fig. 1)
  *   sv_kv_append      commit of the accepted draft tokens to the cache, with
  *                     the representatives of the grown blocks refreshed (Section 2.1)
+ *   sv_accept         acceptance of the draft tokens after verification (Eq. 2-3)
+ *   sv_anchor_jaccard / sv_pick_anchors   anchor-layer calibration       (Eq. 7-8)
+ *   sv_select_blocks_global / _tokens, sv_token_overlap, sv_block_reps_bf16,
+ *   sv_select_blocks_bf16reps   retrieval variants the paper discusses but does
+ *                     not adopt, for comparison                   (Section 2.2, Eq. 6)
  *
  * Conventions for every entry point
  *   - "dev" pointers are device memory owned by the caller; the library never
