@@ -133,6 +133,8 @@ SMALL = {
     # multi-head attention (G = 1), a wide GQA group (G = 16, 128 rows), block 128 whose tail holds <= 64 tokens
     "mha": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=4, seq_len=(1200, 1200), budget_blocks=6, planted=2),
     "g16": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1500, 1500), budget_blocks=6, n_draft=8, planted=2),
+    # more (sequence, KV head) pairs than SMs: several waves of CTAs, one split each
+    "many_seqs": si.shrink(si.WORKLOADS["cfg2"], n_seq=40, seq_len=(300, 1100), budget_blocks=6, planted=1),
     "b128_short_tail": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(128 * 9 + 30, 128 * 9 + 30), n_q_heads=16, n_kv_heads=4,
                                  budget_blocks=5, n_draft=6, planted=2),
 }
