@@ -921,3 +921,93 @@ def test_engine_two_decoding_steps(sv):
                                             None, idx_g, cnt_g)
         check_attn(bf16_host(out2[l]), lse2.cpu().numpy().astype(np.float64), o_ref, lse_ref, f"second step, layer {l}")
     assert int(eng.status.item()) == 0
+
+
+def test_select_fuzz_exact_scores(sv):
+    """Selection on hand-made score distributions, bit-exact against the oracle including ties.  The query is a unit
+    vector, so a block's score is the first component of its representative exactly (no rounding on either side):
+    normal, heavy-tailed (outliers stretch the score range), coarsely quantised (many ties at the boundary), two far
+    clusters, constant, and block counts on both sides of the 2048-block limit of the fast selection path."""
+    g = np.random.default_rng(77)
+    S, Hkv, Hq, T, B = 2, 2, 4, 3, 64
+    kinds = ["normal", "cauchy", "quantised", "clusters", "constant", "few_distinct", "tiny_range"]
+    for trial in range(42):
+        kind = kinds[trial % len(kinds)]
+        NB = int(g.choice([33, 64, 200, 512, 513, 1024, 1500, 2048, 2049, 3000]))
+        lens = np.array([NB * B - int(g.integers(0, B)), max(B, int(g.integers(NB // 2, NB)) * B - 7)], np.int32)
+        n_sink, n_local = int(g.integers(0, 3)), int(g.integers(0, 3))
+        budget = np.array([int(g.integers(n_sink + n_local + 1, NB)), int(g.integers(n_sink + n_local, NB + 5))], np.int32)
+        max_sel = int(max(budget.max(), 8))
+        if kind == "normal":
+            sc = g.standard_normal((S, Hkv, NB))
+        elif kind == "cauchy":
+            sc = g.standard_cauchy((S, Hkv, NB)) * 0.01
+        elif kind == "quantised":
+            sc = np.round(g.standard_normal((S, Hkv, NB)) * 3) / 8
+        elif kind == "clusters":
+            sc = g.standard_normal((S, Hkv, NB)) * 1e-3 + (g.random((S, Hkv, NB)) < 0.1) * 50.0
+        elif kind == "constant":
+            sc = np.full((S, Hkv, NB), -0.375)
+        elif kind == "few_distinct":
+            sc = g.integers(0, 3, (S, Hkv, NB)).astype(np.float64) - 1.0
+        else:
+            sc = 1.0 + g.random((S, Hkv, NB)) * 1e-6
+        sc = sc.astype(np.float32)
+        reps = np.zeros((S, Hkv, NB, 128), np.float32)
+        reps[..., 0] = sc
+        q = np.zeros((S, T, Hq, 128), np.float32)
+        q[:, 0, :, 0] = 1.0
+        q[:, 1:] = g.standard_normal((S, T - 1, Hq, 128))
+        geom = sv.make_geom(S, Hq, Hkv, 128, B, NB, T)
+        idx = torch.full((S, Hkv, max_sel), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((S, Hkv), -7, dtype=torch.int32, device="cuda")
+        sv.sv_select_blocks(geom, bf16_dev(si.f32_to_bf16_bits(q)), torch.from_numpy(reps).cuda(), torch.from_numpy(lens).cuda(),
+                            torch.from_numpy(budget).cuda(), n_sink, n_local, idx, cnt)
+        torch.cuda.synchronize()
+        sc_o = sc.astype(np.float64)
+        eff = np.minimum(np.maximum(budget, n_sink + n_local), max_sel).astype(np.int32)   # the library's documented clamp
+        idx_o, cnt_o = oracle.select(sc_o, lens, eff, B, n_sink, n_local, max_sel)
+        np.testing.assert_array_equal(cnt.cpu().numpy(), cnt_o, err_msg=f"trial {trial} {kind} NB={NB}")
+        ih = idx.cpu().numpy()
+        for s in range(S):
+            for h in range(Hkv):
+                np.testing.assert_array_equal(ih[s, h, :cnt_o[s, h]], idx_o[s, h, :cnt_o[s, h]],
+                                              err_msg=f"trial {trial} {kind} NB={NB} s={s} h={h} budget={budget[s]}")
+
+
+def test_select_global_fuzz_exact_scores(sv):
+    """The shared-budget variant on the same hand-made score distributions, bit-exact including ties across heads."""
+    g = np.random.default_rng(78)
+    S, Hkv, Hq, T, B = 2, 4, 4, 2, 64
+    for trial in range(18):
+        NB = int(g.choice([40, 200, 512, 1000]))
+        lens = np.array([NB * B - int(g.integers(0, B)), max(B, int(g.integers(NB // 2, NB)) * B - 7)], np.int32)
+        n_sink, n_local = int(g.integers(0, 2)), int(g.integers(0, 3))
+        budget = np.array([int(g.integers(n_sink + n_local, NB)), int(g.integers(n_sink + n_local, NB + 3))], np.int32)
+        kind = trial % 4
+        if kind == 0:
+            sc = g.standard_normal((S, Hkv, NB))
+        elif kind == 1:
+            sc = np.round(g.standard_normal((S, Hkv, NB)) * 2) / 4            # many ties, also across heads
+        elif kind == 2:
+            sc = g.standard_cauchy((S, Hkv, NB)) * 0.01
+        else:
+            sc = np.full((S, Hkv, NB), 0.25)
+        sc = sc.astype(np.float32)
+        reps = np.zeros((S, Hkv, NB, 128), np.float32)
+        reps[..., 0] = sc
+        q = np.zeros((S, T, Hq, 128), np.float32)
+        q[:, 0, :, 0] = 1.0
+        geom = sv.make_geom(S, Hq, Hkv, 128, B, NB, T)
+        idx = torch.full((S, Hkv, NB), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((S, Hkv), -7, dtype=torch.int32, device="cuda")
+        scd = torch.zeros((S, Hkv, NB), device="cuda")
+        sv.sv_select_blocks_global(geom, bf16_dev(si.f32_to_bf16_bits(q)), torch.from_numpy(reps).cuda(),
+                                   torch.from_numpy(lens).cuda(), torch.from_numpy(budget).cuda(), n_sink, n_local, idx, cnt, scd)
+        torch.cuda.synchronize()
+        idx_o, cnt_o = oracle.select_global(sc.astype(np.float64), lens, budget, B, n_sink, n_local, NB)
+        np.testing.assert_array_equal(cnt.cpu().numpy(), cnt_o, err_msg=f"trial {trial}")
+        ih = idx.cpu().numpy()
+        for s in range(S):
+            for h in range(Hkv):
+                np.testing.assert_array_equal(ih[s, h, :cnt_o[s, h]], idx_o[s, h, :cnt_o[s, h]], err_msg=f"trial {trial} s={s} h={h}")
