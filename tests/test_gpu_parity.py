@@ -1011,3 +1011,30 @@ def test_select_global_fuzz_exact_scores(sv):
         for s in range(S):
             for h in range(Hkv):
                 np.testing.assert_array_equal(ih[s, h, :cnt_o[s, h]], idx_o[s, h, :cnt_o[s, h]], err_msg=f"trial {trial} s={s} h={h}")
+
+
+def test_pipeline_fuzz_random_shapes(sv):
+    """reps -> select -> attention on randomly drawn shapes (batch, GQA group, draft length, chain / tree, block size,
+    ragged lengths, budgets, forced blocks), each compared stage by stage with the oracle."""
+    g = np.random.default_rng(2024)
+    done = 0
+    for trial in range(40):
+        Hkv = int(g.choice([1, 2, 4]))
+        G = int(g.choice([1, 2, 4, 8]))
+        T = int(g.choice([1, 2, 3, 5, 8, 13, 16]))
+        if G * T > 128:
+            continue
+        B = int(g.choice([64, 128]))
+        S = int(g.integers(1, 5))
+        lo = int(g.integers(3 * B, 12 * B))
+        hi = lo + int(g.integers(0, 10 * B))
+        n_sink, n_local = int(g.integers(0, 3)), int(g.integers(0, 3))
+        nb_min = (lo + B - 1) // B
+        budget = int(g.integers(max(1, n_sink + n_local), nb_min + 3))
+        w = si.Workload(f"fuzz{trial}", S, (lo, hi), Hkv * G, Hkv, 128, B, budget, T, bool(g.integers(0, 2)), 1,
+                        max(1, min(2, budget - n_sink - n_local)), 5000 + trial, n_sink, n_local)
+        geom = si.make_geometry(w)
+        c = si.make_layer(geom, sharp=bool(trial & 1))
+        run_pipeline(sv, c, what=f"fuzz {trial}: S={S} Hkv={Hkv} G={G} T={T} B={B} L={lo}..{hi} N={budget} sink={n_sink} local={n_local}")
+        done += 1
+    assert done >= 25
