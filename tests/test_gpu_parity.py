@@ -1038,3 +1038,20 @@ def test_pipeline_fuzz_random_shapes(sv):
         run_pipeline(sv, c, what=f"fuzz {trial}: S={S} Hkv={Hkv} G={G} T={T} B={B} L={lo}..{hi} N={budget} sink={n_sink} local={n_local}")
         done += 1
     assert done >= 25
+
+
+def test_accept_fuzz(sv):
+    """Acceptance walk on random small cases: trees with several siblings per row, every draft length, vocabularies that
+    leave ragged per-thread segments, draft models from identical to unrelated."""
+    g = np.random.default_rng(99)
+    for trial in range(36):
+        S = int(g.integers(1, 6))
+        T = int(g.integers(1, 17))
+        V = 4 * int(g.integers(2, 1500))
+        c = si.make_accept_case(S, T, V, seed=300 + trial, tree=bool(trial % 3), draft_noise=float(g.choice([0.0, 0.1, 0.5, 2.0])))
+        if trial % 5 == 0 and T > 2:                       # a bushy tree: every draft row hangs off the root
+            c["parent"] = np.tile(np.array([-1] + [0] * (T - 1), np.int32), (S, 1))
+        if trial % 7 == 0:
+            c["u_accept"][:] = 0.9995                       # reject as much as possible
+        r = _settle_accept_case(c)
+        _check_accept(c, r, _gpu_accept(sv, c))
