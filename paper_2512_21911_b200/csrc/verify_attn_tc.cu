@@ -307,7 +307,6 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     }
     grid_dependency_wait();
-    grid_launch_dependents();   // the next kernel may be scheduled; it waits for this grid before reading
     {
         // real rows: all loads of a thread are in flight together
         const int n_q = rows * 16, n_d = has_draft ? 2 * p.T * 16 : 0;
@@ -545,6 +544,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int n_sm = 2 * wg_threads;
     const int t = quad * 32 + lane;
     float *ml1 = reinterpret_cast<float *>(smem + kOffP + kPBytes);   // [2 * NH][128]: m, l of warpgroup 1's slots
+    // Only now may the dependent kernel (the split merge) be scheduled: released at the start, its small CTAs would all
+    // become resident on the few SMs this grid leaves idle and later do the whole merge from there; released here,
+    // they spread over the SMs that the attention CTAs are about to vacate.
+    grid_launch_dependents();
     if (k > 0) wait_pv(k - 1);   // this warpgroup's accumulator is complete
     if (wg == 1) {
 #pragma unroll
