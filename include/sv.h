@@ -56,7 +56,7 @@ typedef enum {
     SV_ERR_ALIGN = 3,       /* a pointer is not aligned as required */
     SV_ERR_BUDGET = 4,      /* n_sink + n_local exceeds max_sel */
     SV_ERR_WORKSPACE = 5,   /* workspace_bytes is smaller than sv_workspace_bytes() */
-    SV_ERR_UNSUPPORTED = 6, /* head_dim != 128, block_size not 64/128, more than 128 query rows per KV head ... */
+    SV_ERR_UNSUPPORTED = 6, /* head_dim != 128, block_size not 64/128, more than 64 draft tokens, more than 8 row tiles ... */
     SV_ERR_CUDA = 7,        /* a CUDA call or kernel launch failed */
     SV_ERR_SCRATCH_LIMIT = 8 /* sv_verify_attn_noalloc: the problem needs more scratch than the built-in buffer holds */
 } sv_status;
@@ -72,7 +72,8 @@ typedef struct {
     int32_t head_dim;   /* D, must be 128 */
     int32_t block_size; /* B: tokens per KV block (Eq. 4), 64 or 128 */
     int32_t max_blocks; /* NBmax: row stride of block_table / reps / scores */
-    int32_t n_draft;    /* T: draft tokens verified per sequence, 1..32, with G*T <= 128 */
+    int32_t n_draft;    /* T: draft tokens verified per sequence, 1..64; the G*T query rows of a KV head are processed
+                           in tiles of at most 128 rows, at most 8 tiles (G <= 128) */
 } sv_geom;
 
 /*
@@ -312,7 +313,7 @@ SV_API sv_status sv_select_blocks_bf16reps(const sv_geom *geom, const void *q, c
  *   n_path      dev int32 [S]; next_token dev int32 [S]
  *   alpha       optional dev float [S][n_draft]: the acceptance probability of every child that was tried
  *               (other entries are left untouched)
- * fp32 arithmetic with fixed summation order (results are reproducible run to run).  n_draft <= 32
+ * fp32 arithmetic with fixed summation order (results are reproducible run to run).  n_draft <= 64
  * (SV_ERR_UNSUPPORTED), vocab a multiple of 4 and 16-byte aligned distributions (SV_ERR_ALIGN).  One launch.
  */
 SV_API sv_status sv_accept(int32_t n_seq, int32_t n_draft, int32_t vocab, const float *p_target, const float *p_draft,

@@ -24,7 +24,7 @@ namespace {
 
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
-constexpr int kMaxRows = 32;     // draft rows per step (the ancestor masks of the attention kernel are 32 bits)
+constexpr int kMaxRows = 64;     // draft rows per step (the ancestor masks of the attention kernel are 64 bits)
 constexpr int kMaxCluster = 8;
 
 struct AcceptParams {

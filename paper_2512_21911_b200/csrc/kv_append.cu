@@ -3,7 +3,7 @@
 // verification attention (Section 2.1: the accepted prefix of the draft is kept; Section 3.1: blocks are cut
 // from the current cache).
 //
-// One CTA per (KV head, sequence).  At most 32 tokens are appended per sequence, so at most two blocks are
+// One CTA per (KV head, sequence).  At most 64 tokens are appended per sequence, so at most two blocks are
 // touched: the rows are copied with 128-bit loads/stores (K and V), then the one or two affected block
 // means are recomputed from the pool exactly as sv_block_reps does (fp32 sums in a fixed order), which keeps
 // them bit-identical to a full rebuild.  Traffic: n*512 bytes copied + at most 2*B*256 bytes re-read per

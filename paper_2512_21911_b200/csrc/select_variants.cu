@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(kOverlapThreads) token_overlap_kernel(const in
     const int words = (NBmax + 31) >> 5;
     svk::grid_dependency_wait();
     svk::grid_launch_dependents();
-    __shared__ int n_of[32];
+    __shared__ int n_of[64];
     for (int i = threadIdx.x; i < T * words; i += kOverlapThreads) bitmap[i] = 0u;
     if (threadIdx.x < T) n_of[threadIdx.x] = min(max(cnt[((size_t)threadIdx.x * S + s) * Hkv + h], 0), max_sel);
     __syncthreads();

@@ -9,11 +9,24 @@
 namespace svh {
 
 constexpr int kHeadDim = 128;
-constexpr int kMaxRows = 128;      // G * T rows packed per KV head
-constexpr int kMaxDraft = 32;      // ancestor masks are 32-bit
+constexpr int kMaxRows = 128;      // query rows (G * draft tokens) packed into one M = 128 tile
+constexpr int kMaxRowTiles = 8;    // row tiles per (sequence, KV head): G * T <= 1024 at most
+constexpr int kMaxDraft = 64;      // ancestor masks are 64-bit; the draft tokens form one 64-key unit
 constexpr int kMaxBlocksSelect = 32768;
 
 inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Draft tokens whose G query rows fit one M = 128 row tile, and the number of such tiles.
+inline int tokens_per_tile(const sv_geom *g)
+{
+    const int G = g->n_q_heads / g->n_kv_heads;
+    return G * g->n_draft <= kMaxRows ? g->n_draft : (kMaxRows / G > 0 ? kMaxRows / G : 1);
+}
+inline int row_tiles(const sv_geom *g)
+{
+    const int tt = tokens_per_tile(g);
+    return (g->n_draft + tt - 1) / tt;
+}
 
 inline sv_status check_geom(const sv_geom *g)
 {
@@ -24,7 +37,7 @@ inline sv_status check_geom(const sv_geom *g)
     if (g->head_dim != kHeadDim) return SV_ERR_UNSUPPORTED;
     if (g->block_size != 64 && g->block_size != 128) return SV_ERR_UNSUPPORTED;
     if (g->n_draft > kMaxDraft) return SV_ERR_UNSUPPORTED;
-    if ((g->n_q_heads / g->n_kv_heads) * g->n_draft > kMaxRows) return SV_ERR_UNSUPPORTED;
+    if (g->n_q_heads / g->n_kv_heads > kMaxRows || row_tiles(g) > kMaxRowTiles) return SV_ERR_UNSUPPORTED;
     if (g->n_seq > 65535 || g->n_kv_heads > 65535) return SV_ERR_SHAPE;
     return SV_OK;
 }

@@ -613,16 +613,6 @@ bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
 
 using svh::sm_count;
 
-// Blocks per CTA are minimised subject to one CTA per SM; then the fewest splits that achieve it.
-int choose_splits(const sv_geom *g, int n_blocks)
-{
-    const int pairs = g->n_seq * g->n_kv_heads;
-    const int per_pair = sm_count() / pairs;
-    if (per_pair <= 1 || n_blocks <= 1) return 1;
-    const int blocks_per_cta = (n_blocks + per_pair - 1) / per_pair;
-    return (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
-}
-
 // The tcgen05 kernel is the product path.  Setting SV_ATTN_IMPL=mma in the environment (read once)
 // selects the older mma.sync kernel, kept for A/B comparisons of the two tensor-core paths.
 bool use_tensor_memory_path()
@@ -632,6 +622,16 @@ bool use_tensor_memory_path()
         return !(v && v[0] == 'm');
     }();
     return tc;
+}
+
+// Blocks per CTA are minimised subject to one CTA per SM; then the fewest splits that achieve it.
+int choose_splits(const sv_geom *g, int n_blocks)
+{
+    const int pairs = g->n_seq * g->n_kv_heads * (use_tensor_memory_path() ? svh::row_tiles(g) : 1);
+    const int per_pair = sm_count() / pairs;
+    if (per_pair <= 1 || n_blocks <= 1) return 1;
+    const int blocks_per_cta = (n_blocks + per_pair - 1) / per_pair;
+    return (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
 }
 
 template <int WM, int MT, int WT>
@@ -721,12 +721,15 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
     p.status = status_word;
     p.T = geom->n_draft, p.Hq = geom->n_q_heads, p.Hkv = geom->n_kv_heads, p.G = G, p.B = geom->block_size;
     p.NBmax = geom->max_blocks, p.max_sel = max_sel, p.splits = splits;
+    p.Tt = svh::tokens_per_tile(geom), p.tiles = svh::row_tiles(geom);
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;   // 1/sqrt(128)
     p.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     dim3 grid(splits, geom->n_kv_heads, geom->n_seq);
     cudaError_t e;
+    if (!use_tensor_memory_path() && (rows > svh::kMaxRows || geom->n_draft > 32)) return SV_ERR_UNSUPPORTED;
+    if (use_tensor_memory_path()) grid.x = splits * p.tiles;   // one CTA per (row tile, split)
     if (use_tensor_memory_path())
         e = launch_attn_tc(tk, tv, p, grid, cs);          // tcgen05 + TMEM, rows padded to one M = 128 tile
     else if (rows <= 16)

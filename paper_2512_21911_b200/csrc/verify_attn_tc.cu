@@ -96,16 +96,18 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint8_t *misc = smem + kOffMisc;
     const uint32_t bars = smem0 + kOffMisc;                               // kNumBars x 8 bytes
     int *meta = reinterpret_cast<int *>(misc + 256);                      // [kStages] valid keys per stage
-    uint32_t *anc = reinterpret_cast<uint32_t *>(misc + 320);             // [32] visible-draft masks
+    unsigned long long *anc = reinterpret_cast<unsigned long long *>(misc + 512);   // [64] visible-draft masks
     volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 448);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 456);
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
-    const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+    // blockIdx.x = row tile * splits + split: the query rows of draft tokens i0 .. i0 + Tq - 1, a slice of the blocks
+    const int tile = blockIdx.x / p.splits, split = blockIdx.x - tile * p.splits, h = blockIdx.y, s = blockIdx.z;
+    const int i0 = tile * p.Tt, Tq = min(p.Tt, p.T - i0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int upb = p.B / kUnit;
     const bool has_draft = split == p.splits - 1;
-    const int rows = p.G * p.T;
+    const int rows = p.G * Tq;                               // query rows of this tile
     constexpr int RPQ = 8 * NH;                              // query rows per TMEM lane quadrant
     const int n_active = min(4, (rows + RPQ - 1) / RPQ);     // warps per softmax warpgroup that own real rows
 
@@ -317,7 +319,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (idx < n_q) {
                 const int r = idx >> 4, c = idx & 15;
                 const int i = r / p.G, g = r - i * p.G;
-                v[x] = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
+                v[x] = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i0 + i) * p.Hq + h * p.G + g) * 128) + c);
             }
         }
         uint4 w[4];
@@ -330,18 +332,18 @@ __global__ void __launch_bounds__(kThreads, 1)
                 w[x] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
             }
         }
-        if (has_draft && tid < 32) {
-            uint32_t mask = 0;
+        if (has_draft && tid < 64) {
+            unsigned long long mask = 0;
             if (tid < p.T) {
                 if (p.parent) {
                     int a = tid;
                     for (int step = 0; step < p.T && a >= 0; ++step) {
-                        mask |= 1u << a;
+                        mask |= 1ull << a;
                         const int nxt = p.parent[(size_t)s * p.T + a];
                         a = nxt < a ? nxt : -1;   // parents must precede their children
                     }
                 } else {
-                    mask = (tid == 31) ? 0xFFFFFFFFu : ((1u << (tid + 1)) - 1u);
+                    mask = (tid == 63) ? ~0ull : ((1ull << (tid + 1)) - 1ull);
                 }
             }
             anc[tid] = mask;
@@ -365,7 +367,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int i = r / p.G, g = r - i * p.G;
             const int tr = (r / RPQ) * 32 + (r % RPQ);
             *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) =
-                __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
+                __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i0 + i) * p.Hq + h * p.G + g) * 128) + c);
         }
         for (int idx = tid + 4 * 256; idx < n_d; idx += 256) {
             const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
@@ -386,15 +388,15 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t t_lane = (uint32_t)(quad * 32) << 16;
     const uint32_t t_s = tmem_base + t_lane + wg * kUnit;
     const uint32_t t_o = tmem_base + t_lane + 128 + wg * 128;
-    const uint32_t all_t = (p.T == 32) ? 0xFFFFFFFFu : ((1u << p.T) - 1u);
+    const unsigned long long all_t = (p.T == 64) ? ~0ull : ((1ull << p.T) - 1ull);
     const int wg_threads = n_active * 32;
-    uint32_t vis[NH];
+    unsigned long long vis[NH];
     int trow[NH], lrow[NH];
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
         lrow[i] = quad * RPQ + 8 * i + lr;
         trow[i] = quad * 32 + 8 * i + lr;
-        vis[i] = (has_draft && lrow[i] < rows) ? anc[lrow[i] / p.G] : all_t;
+        vis[i] = (has_draft && lrow[i] < rows) ? anc[i0 + lrow[i] / p.G] : all_t;
     }
 
     const int L = p.seq_lens[s];
@@ -462,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     for (int e = 0; e < 2; ++e) {
                         const int col = 8 * j + 2 * qd + e;
                         bool ok = col < nvalid;
-                        if (is_draft) ok = ok && col < 32 && ((vis[i] >> (col & 31)) & 1u);
+                        if (is_draft) ok = ok && ((vis[i] >> col) & 1ull);
                         if (!ok) sc[i][2 * j + e] = -INFINITY;
                     }
             }
@@ -610,14 +612,14 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (row >= rows) continue;
         if (p.splits == 1) {
             const int ii = row / p.G, g = row - ii * p.G;
-            const size_t orow = ((size_t)s * p.T + ii) * p.Hq + h * p.G + g;
+            const size_t orow = ((size_t)s * p.T + i0 + ii) * p.Hq + h * p.G + g;
             const float inv = 1.f / lsum;
             uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + qd;
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) dst[4 * jj] = pack_bf16(o[i][2 * jj] * inv, o[i][2 * jj + 1] * inv);
             if (p.lse && qd == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
         } else {
-            const size_t prow = (((size_t)s * p.Hkv + h) * p.splits + split) * rows + row;
+            const size_t prow = (((size_t)s * p.Hkv + h) * p.splits + split) * (p.G * p.T) + i0 * p.G + row;
             float2 *dst = reinterpret_cast<float2 *>(p.ws_o + prow * 128) + qd;
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) dst[4 * jj] = make_float2(o[i][2 * jj], o[i][2 * jj + 1]);
@@ -655,7 +657,7 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
 cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                            cudaStream_t stream)
 {
-    const int rows = p.G * p.T;
+    const int rows = p.G * p.Tt;   // rows of a full row tile
     if (rows <= 32) return launch_tc<1>(tm_k, tm_v, p, grid, stream);
     if (rows <= 64) return launch_tc<2>(tm_k, tm_v, p, grid, stream);
     return launch_tc<4>(tm_k, tm_v, p, grid, stream);

@@ -133,6 +133,11 @@ SMALL = {
     # multi-head attention (G = 1), a wide GQA group (G = 16, 128 rows), block 128 whose tail holds <= 64 tokens
     "mha": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=4, seq_len=(1200, 1200), budget_blocks=6, planted=2),
     "g16": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1500, 1500), budget_blocks=6, n_draft=8, planted=2),
+    # more than 128 query rows per KV head (several row tiles) and more than 32 draft tokens (64-bit ancestor masks)
+    "t60_tree": si.shrink(si.WORKLOADS["cfg1"], seq_len=(3000, 3000), budget_blocks=10, n_draft=60, n_layers=1, tree=True, planted=3),
+    "t40_chain_2seq": si.shrink(si.WORKLOADS["cfg2"], n_seq=2, seq_len=(900, 2100), budget_blocks=7, n_draft=40, planted=2),
+    "g8_t24_b128": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(2000, 4000), budget_blocks=6, n_draft=24, planted=2),
+    "g16_t64": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1100, 1100), budget_blocks=5, n_draft=64, tree=True, planted=2),
     # more (sequence, KV head) pairs than SMs: several waves of CTAs, one split each
     "many_seqs": si.shrink(si.WORKLOADS["cfg2"], n_seq=40, seq_len=(300, 1100), budget_blocks=6, planted=1),
     "b128_short_tail": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(128 * 9 + 30, 128 * 9 + 30), n_q_heads=16, n_kv_heads=4,
@@ -404,7 +409,8 @@ def test_mma_sync_attention_path_stays_green():
         pytest.skip("already running on the mma.sync path")
     env = dict(os.environ, SV_ATTN_IMPL="mma")
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-q", "-x", "-m", "gpu", "-k",
-                        "pipeline_parity_small or more_splits or empty_prefix"], env=env, capture_output=True, text=True,
+                        "(pipeline_parity_small or more_splits or empty_prefix) and not t60 and not t40 and not g8_t24 and not g16_t64"],
+                       env=env, capture_output=True, text=True,   # the older kernel stops at 128 query rows / 32 draft tokens
                        cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
@@ -716,7 +722,7 @@ def _check_accept(c, r, got):
 
 
 @pytest.mark.parametrize("S,T,V,tree", [(4, 5, 512, False), (3, 8, 4096, True), (2, 16, 32768, True),
-                                         (5, 6, 10240, False), (2, 1, 2048, False), (1, 32, 8192, True)])
+                                         (5, 6, 10240, False), (2, 1, 2048, False), (1, 32, 8192, True), (2, 64, 4096, True), (1, 60, 2048, False)])
 def test_accept_parity(sv, S, T, V, tree):
     """Acceptance walk against the oracle: kept rows bit-exact, acceptance probabilities to fp32 accuracy, the
     drawn token equal (or adjacent within fp32 summation error on the cumulative sum).  Vocabularies from one CTA

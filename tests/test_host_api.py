@@ -55,13 +55,15 @@ def test_argument_validation_without_device(svb):
     assert lib.sv_block_reps(ctypes.byref(g), ctypes.byref(null_kv), 0, -1, None, None) == 1      # SV_ERR_NULL
     bad = svb.make_geom(1, 8, 3, 128, 64, 64, 4)
     assert lib.sv_block_reps(ctypes.byref(bad), ctypes.byref(null_kv), 0, -1, None, None) == 2    # SV_ERR_SHAPE
-    for kw, code in ((dict(head_dim=64), 6), (dict(block_size=32), 6), (dict(n_draft=33), 6), (dict(n_draft=0), 2)):
+    for kw, code in ((dict(head_dim=64), 6), (dict(block_size=32), 6), (dict(n_draft=65), 6), (dict(n_draft=0), 2)):
         args = dict(n_seq=1, n_q_heads=8, n_kv_heads=2, head_dim=128, block_size=64, max_blocks=64, n_draft=4)
         args.update(kw)
         gg = svb.make_geom(**args)
         assert lib.sv_block_reps(ctypes.byref(gg), ctypes.byref(null_kv), 0, -1, None, None) == code
-    big = svb.make_geom(1, 64, 2, 128, 64, 64, 8)        # 32 * 8 = 256 query rows per KV head
+    big = svb.make_geom(1, 64, 2, 128, 64, 64, 64)       # G = 32: 4 draft tokens per row tile, 16 tiles
     assert lib.sv_block_reps(ctypes.byref(big), ctypes.byref(null_kv), 0, -1, None, None) == 6
+    ok = svb.make_geom(1, 64, 2, 128, 64, 64, 8)         # 32 * 8 = 256 query rows per KV head: two row tiles
+    assert lib.sv_block_reps(ctypes.byref(ok), ctypes.byref(null_kv), 0, -1, None, None) == 1      # only the pointers are missing
     # misaligned pool pointer
     kv = svb.sv_kv(0x1008, 0x2000, 0x3000, 0x4000, 4)
     assert lib.sv_block_reps(ctypes.byref(g), ctypes.byref(kv), 0, -1, 0x5000, None) == 3        # SV_ERR_ALIGN
@@ -89,7 +91,7 @@ def test_argument_validation_without_device(svb):
                                                                0x8000, 0x9000, None, None)
     assert acc(1, 8, 1024, out=None) == 1
     assert acc(0, 8, 1024) == 2 and acc(1, 0, 1024) == 2 and acc(1, 8, 0) == 2
-    assert acc(1, 33, 1024) == 6
+    assert acc(1, 65, 1024) == 6
     assert acc(1, 8, 1022) == 3 and acc(1, 8, 1024, pt=0x1004) == 3
     # attention: missing output
     kv = svb.sv_kv(0x1000, 0x2000, 0x3000, 0x4000, 4)
