@@ -22,8 +22,8 @@ struct AttnParams {
     float *ws_ml;   // [S][Hkv][splits][rows][2]
     int32_t *status;
     int T, Hq, Hkv, G, B, NBmax, max_sel, splits;
-    int Tt, tiles;   // tcgen05 kernel: draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
     float scale_log2;
+    int Tt, tiles;   // tcgen05 kernel: draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
 };
 
 // tcgen05 / TMEM attention kernel (verify_attn_tc.cu): rows = G*T <= 128 packed as one M=128 tile.

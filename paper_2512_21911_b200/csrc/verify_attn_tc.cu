@@ -85,7 +85,10 @@ enum Bar {
 };
 
 // NH = 8-row groups per TMEM lane quadrant that hold real query rows: 1 (rows <= 32), 2 (<= 64), 4 (<= 128).
-template <int NH>
+// kWide: more than one row tile per (sequence, KV head) or more than 32 draft tokens (64-bit ancestor masks).  The
+// common case keeps split = blockIdx.x, plain row arithmetic and 32-bit masks: deriving the split from a division
+// costs 3 % on long loops, and the wider mask code 7 % at 128 rows.
+template <int NH, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
     verify_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                           const AttnParams p)
@@ -96,14 +99,16 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint8_t *misc = smem + kOffMisc;
     const uint32_t bars = smem0 + kOffMisc;                               // kNumBars x 8 bytes
     int *meta = reinterpret_cast<int *>(misc + 256);                      // [kStages] valid keys per stage
-    unsigned long long *anc = reinterpret_cast<unsigned long long *>(misc + 512);   // [64] visible-draft masks
+    unsigned long long *anc = reinterpret_cast<unsigned long long *>(misc + 512);   // [64] visible-draft masks (kWide)
+    uint32_t *anc32 = reinterpret_cast<uint32_t *>(misc + 320);                     // [32] the same, up to 32 draft tokens
     volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 448);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 456);
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
     // blockIdx.x = row tile * splits + split: the query rows of draft tokens i0 .. i0 + Tq - 1, a slice of the blocks
-    const int tile = blockIdx.x / p.splits, split = blockIdx.x - tile * p.splits, h = blockIdx.y, s = blockIdx.z;
-    const int i0 = tile * p.Tt, Tq = min(p.Tt, p.T - i0);
+    const int tile = kWide ? blockIdx.x / p.splits : 0;
+    const int split = kWide ? blockIdx.x - tile * p.splits : blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+    const int i0 = kWide ? tile * p.Tt : 0, Tq = kWide ? min(p.Tt, p.T - i0) : p.T;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int upb = p.B / kUnit;
     const bool has_draft = split == p.splits - 1;
@@ -332,7 +337,23 @@ __global__ void __launch_bounds__(kThreads, 1)
                 w[x] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
             }
         }
-        if (has_draft && tid < 64) {
+        if (!kWide && has_draft && tid < 32) {
+            uint32_t mask = 0;
+            if (tid < p.T) {
+                if (p.parent) {
+                    int a = tid;
+                    for (int step = 0; step < p.T && a >= 0; ++step) {
+                        mask |= 1u << a;
+                        const int nxt = p.parent[(size_t)s * p.T + a];
+                        a = nxt < a ? nxt : -1;   // parents must precede their children
+                    }
+                } else {
+                    mask = (tid == 31) ? 0xFFFFFFFFu : ((1u << (tid + 1)) - 1u);
+                }
+            }
+            anc32[tid] = mask;
+        }
+        if (kWide && has_draft && tid < 64) {
             unsigned long long mask = 0;
             if (tid < p.T) {
                 if (p.parent) {
@@ -388,15 +409,25 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t t_lane = (uint32_t)(quad * 32) << 16;
     const uint32_t t_s = tmem_base + t_lane + wg * kUnit;
     const uint32_t t_o = tmem_base + t_lane + 128 + wg * 128;
-    const unsigned long long all_t = (p.T == 64) ? ~0ull : ((1ull << p.T) - 1ull);
     const int wg_threads = n_active * 32;
-    unsigned long long vis[NH];
+    // per slot, the draft tokens the row may see: kWide: bit 2j + e <-> this thread's column 8j + 2qd + e; else bit = token
+    uint32_t vis[NH];
     int trow[NH], lrow[NH];
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
         lrow[i] = quad * RPQ + 8 * i + lr;
         trow[i] = quad * 32 + 8 * i + lr;
-        vis[i] = (has_draft && lrow[i] < rows) ? anc[i0 + lrow[i] / p.G] : all_t;
+        if constexpr (kWide) {
+            const unsigned long long all_t = (p.T == 64) ? ~0ull : ((1ull << p.T) - 1ull);
+            const unsigned long long row_vis = (has_draft && lrow[i] < rows) ? anc[i0 + lrow[i] / p.G] : all_t;
+            uint32_t mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mine |= (uint32_t)((row_vis >> (8 * j + 2 * qd)) & 3ull) << (2 * j);
+            vis[i] = mine;
+        } else {
+            const uint32_t all_t = (p.T == 32) ? 0xFFFFFFFFu : ((1u << p.T) - 1u);
+            vis[i] = (has_draft && lrow[i] < rows) ? anc32[lrow[i] / p.G] : all_t;
+        }
     }
 
     const int L = p.seq_lens[s];
@@ -464,7 +495,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                     for (int e = 0; e < 2; ++e) {
                         const int col = 8 * j + 2 * qd + e;
                         bool ok = col < nvalid;
-                        if (is_draft) ok = ok && ((vis[i] >> col) & 1ull);
+                        if constexpr (kWide) {
+                            if (is_draft) ok = ok && ((vis[i] >> (2 * j + e)) & 1u);
+                        } else {
+                            if (is_draft) ok = ok && col < 32 && ((vis[i] >> (col & 31)) & 1u);
+                        }
                         if (!ok) sc[i][2 * j + e] = -INFINITY;
                     }
             }
@@ -631,13 +666,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 }  // namespace
 
-template <int NH>
+template <int NH, bool kWide>
 static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                              cudaStream_t stream)
 {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(verify_attn_tc_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -651,16 +686,21 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
     attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH>, tm_k, tm_v, p);
+    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide>, tm_k, tm_v, p);
 }
 
 cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                            cudaStream_t stream)
 {
     const int rows = p.G * p.Tt;   // rows of a full row tile
-    if (rows <= 32) return launch_tc<1>(tm_k, tm_v, p, grid, stream);
-    if (rows <= 64) return launch_tc<2>(tm_k, tm_v, p, grid, stream);
-    return launch_tc<4>(tm_k, tm_v, p, grid, stream);
+    if (p.tiles > 1 || p.T > 32) {
+        if (rows <= 32) return launch_tc<1, true>(tm_k, tm_v, p, grid, stream);
+        if (rows <= 64) return launch_tc<2, true>(tm_k, tm_v, p, grid, stream);
+        return launch_tc<4, true>(tm_k, tm_v, p, grid, stream);
+    }
+    if (rows <= 32) return launch_tc<1, false>(tm_k, tm_v, p, grid, stream);
+    if (rows <= 64) return launch_tc<2, false>(tm_k, tm_v, p, grid, stream);
+    return launch_tc<4, false>(tm_k, tm_v, p, grid, stream);
 }
 
 }  // namespace svk
