@@ -503,9 +503,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                         if (!ok) sc[i][2 * j + e] = -INFINITY;
                     }
             }
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) mx = fmaxf(mx, sc[i][c]);
+            // 16 columns with 3-input maxima: 8 instructions instead of 15
+            const float x0 = max3f(sc[i][0], sc[i][1], sc[i][2]), x1 = max3f(sc[i][3], sc[i][4], sc[i][5]);
+            const float x2 = max3f(sc[i][6], sc[i][7], sc[i][8]), x3 = max3f(sc[i][9], sc[i][10], sc[i][11]);
+            const float x4 = max3f(sc[i][12], sc[i][13], sc[i][14]);
+            float mx = fmaxf(max3f(x0, x1, x2), max3f(x3, x4, sc[i][15]));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
             const float um = mx * p.scale_log2;
@@ -550,15 +552,20 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
         for (int i = 0; i < NH; ++i) {
             const float m_use = (m[i] == -INFINITY) ? 0.f : m[i];
-            float lsum = 0.f;
+            // two columns per instruction: x = s * scale - m and the running sums as packed fp32 pairs
+            const unsigned long long scale2 = f2_pack(p.scale_log2, p.scale_log2), neg_m2 = f2_pack(-m_use, -m_use);
+            unsigned long long lsum2 = f2_pack(0.f, 0.f);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float p0 = fast_exp2(fmaf(sc[i][2 * j], p.scale_log2, -m_use));
-                const float p1 = fast_exp2(fmaf(sc[i][2 * j + 1], p.scale_log2, -m_use));
-                lsum += p0 + p1;
+                float x0, x1;
+                f2_unpack(f2_fma(f2_pack(sc[i][2 * j], sc[i][2 * j + 1]), scale2, neg_m2), x0, x1);
+                const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                lsum2 = f2_add(lsum2, f2_pack(p0, p1));
                 *reinterpret_cast<uint32_t *>(pbuf + swz128(trow[i], j) + 4 * qd) = pack_bf16(p0, p1);
             }
-            l[i] += lsum;
+            float ls0, ls1;
+            f2_unpack(lsum2, ls0, ls1);
+            l[i] += ls0 + ls1;
         }
         if (!is_draft && nvalid < kUnit) {
             // zero the value rows past the end of the sequence (0 * junk must stay 0)
