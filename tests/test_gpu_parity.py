@@ -1061,3 +1061,54 @@ def test_accept_fuzz(sv):
             c["u_accept"][:] = 0.9995                       # reject as much as possible
         r = _settle_accept_case(c)
         _check_accept(c, r, _gpu_accept(sv, c))
+
+
+def test_benchmark_step_under_cuda_graph_replay(sv):
+    """The launch configuration the benchmark times: a stack of full-size cfg1 layers with their pools in one
+    allocation, one step (tail refresh of all layers in one launch, then select + attention + merge per layer, chained
+    with programmatic dependent launch) captured in a CUDA graph and replayed.  Every layer's output after the third
+    replay against the oracle on sampled rows; the last layer's block list exact."""
+    n_layers = 3
+    w = si.shrink(si.WORKLOADS["cfg1"], n_layers=n_layers)
+    geom = si.make_geometry(w)
+    layers = [si.make_layer(geom, layer=l, sharp=bool(l & 1)) for l in range(n_layers)]
+    eng = sv.SparseVerifier(n_seq=w.n_seq, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=128,
+                            block_size=w.block_size, max_blocks=geom["max_blocks"], n_draft=w.n_draft, n_layers=n_layers,
+                            block_table=torch.from_numpy(geom["block_table"]).cuda(),
+                            seq_lens=torch.from_numpy(geom["seq_lens"]).cuda(),
+                            budget_blocks=torch.from_numpy(geom["budget"]).cuda(), max_sel=geom["max_sel"],
+                            n_sink=w.n_sink, n_local=w.n_local)
+    k_all = torch.stack([bf16_dev(c["k_pool"]) for c in layers]).contiguous()
+    v_all = torch.stack([bf16_dev(c["v_pool"]) for c in layers]).contiguous()
+    eng.set_kv_stack(k_all, v_all)
+    for l in range(n_layers):
+        eng.build_reps(l)
+    q = torch.stack([bf16_dev(c["q"]) for c in layers]).contiguous()
+    dk = torch.stack([bf16_dev(c["draft_k"]) for c in layers]).contiguous()
+    dv = torch.stack([bf16_dev(c["draft_v"]) for c in layers]).contiguous()
+    out = torch.zeros_like(q)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            eng.verify_step(q, dk, dv, out, refresh_tail=True)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            eng.verify_step(q, dk, dv, out, refresh_tail=True)
+        out.zero_()
+        for _ in range(3):
+            graph.replay()
+        stream.synchronize()
+    assert int(eng.status.item()) == 0
+    g = np.random.default_rng(17)
+    for l, c in enumerate(layers):
+        idx_ref, cnt_ref, _ = oracle_select(c, w.n_sink, w.n_local, geom["max_sel"])
+        smp = np.stack([np.zeros(24, np.int64), g.integers(0, w.n_draft, 24), g.integers(0, w.n_q_heads, 24)], axis=1).astype(np.int32)
+        o_ref, _ = oracle_attn(c, idx_ref, cnt_ref, samples=smp)
+        o = bf16_host(out[l])
+        o_s = np.stack([o[s, i, hq] for s, i, hq in smp])
+        rel = np.linalg.norm(o_s - o_ref, axis=-1) / np.linalg.norm(o_ref, axis=-1)
+        assert rel.max() <= 1e-2 and np.abs(o_s - o_ref).max() <= 1e-2, (l, rel.max())
+        if l == n_layers - 1:
+            np.testing.assert_array_equal(eng.sel_cnt.cpu().numpy(), cnt_ref)
+            np.testing.assert_array_equal(eng.sel_idx.cpu().numpy(), idx_ref)
