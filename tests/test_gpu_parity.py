@@ -1112,3 +1112,33 @@ def test_benchmark_step_under_cuda_graph_replay(sv):
         if l == n_layers - 1:
             np.testing.assert_array_equal(eng.sel_cnt.cpu().numpy(), cnt_ref)
             np.testing.assert_array_equal(eng.sel_idx.cpu().numpy(), idx_ref)
+
+
+def test_select_at_the_largest_supported_block_count(sv):
+    """32768 blocks per sequence (a 2M-token context at block 64): the general radix path with keys of all CTAs of the
+    cluster in CTA 0's shared memory, exact against the oracle; one more block is refused."""
+    g = np.random.default_rng(5)
+    S, Hkv, Hq, T, B, NB = 1, 1, 2, 2, 64, 32768
+    sc = (g.standard_normal((S, Hkv, NB)) * 0.5).astype(np.float32)
+    sc[0, 0, ::997] = 0.125                                           # some exact ties
+    reps = np.zeros((S, Hkv, NB, 128), np.float32)
+    reps[..., 0] = sc
+    q = np.zeros((S, T, Hq, 128), np.float32)
+    q[:, 0, :, 0] = 1.0
+    lens = np.array([NB * B - 5], np.int32)
+    for N in (3, 700, 5000):
+        budget = np.array([N], np.int32)
+        geom = sv.make_geom(S, Hq, Hkv, 128, B, NB, T)
+        idx = torch.full((S, Hkv, N), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((S, Hkv), -7, dtype=torch.int32, device="cuda")
+        sv.sv_select_blocks(geom, bf16_dev(si.f32_to_bf16_bits(q)), torch.from_numpy(reps).cuda(), torch.from_numpy(lens).cuda(),
+                            torch.from_numpy(budget).cuda(), 1, 2, idx, cnt)
+        torch.cuda.synchronize()
+        idx_o, cnt_o = oracle.select(sc.astype(np.float64), lens, budget, B, 1, 2, N)
+        np.testing.assert_array_equal(cnt.cpu().numpy(), cnt_o)
+        np.testing.assert_array_equal(idx.cpu().numpy(), idx_o)
+    too_big = sv.make_geom(S, Hq, Hkv, 128, B, NB + 1, T)
+    with pytest.raises(sv.SvError):
+        sv.sv_select_blocks(too_big, bf16_dev(si.f32_to_bf16_bits(q)), torch.zeros((S, Hkv, NB + 1, 128), device="cuda"),
+                            torch.from_numpy(lens).cuda(), torch.from_numpy(np.array([8], np.int32)).cuda(), 1, 2,
+                            torch.zeros((S, Hkv, 8), dtype=torch.int32, device="cuda"), torch.zeros((S, Hkv), dtype=torch.int32, device="cuda"))
