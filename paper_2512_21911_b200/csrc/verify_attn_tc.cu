@@ -6,9 +6,10 @@
 //
 //   S[128 x 64]  = Q[128 x 128] . K^T     8 x tcgen05.mma (M128 N64 K16), operands in shared memory
 //                                         (Q, K: K-major, 128-byte swizzle), accumulator in TMEM
-//   softmax      four threads per query row (tcgen05.ld 16x256b: the mma.sync accumulator fragment
-//                layout): mask, running max / sum in fp32 with quad shuffles, P rounded to bf16 into
-//                shared memory (K-major, 128-byte swizzle)
+//   softmax      up to 64 query rows: four threads per row (tcgen05.ld 16x256b, the mma.sync accumulator
+//                fragment layout, rows spread over all four lane quadrants): mask, running max / sum in
+//                fp32 with quad shuffles; 65-128 rows: one thread per row (tcgen05.ld 32x32b), no shuffles,
+//                16-byte P stores.  P rounded to bf16 into shared memory (K-major, 128-byte swizzle)
 //   O[128x128]  += P[128 x 64] . V        4 x tcgen05.mma (M128 N128 K16), V read MN-major from the
 //                                         tile exactly as TMA stored it; O stays in TMEM for the whole
 //                                         kernel.  The exponentials use a reference maximum that is only
@@ -413,6 +414,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     // per slot, the draft tokens the row may see: kWide: bit 2j + e <-> this thread's column 8j + 2qd + e; else bit = token
     uint32_t vis[NH];
     int trow[NH], lrow[NH];
+    unsigned long long row_vis = ~0ull;   // NH == 4: the draft tokens row quad * 32 + lane may see
+    if constexpr (NH == 4) {
+        const int r = quad * 32 + lane;
+        if (has_draft && r < rows) row_vis = kWide ? anc[i0 + r / p.G] : (unsigned long long)anc32[r / p.G];
+    }
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
         lrow[i] = quad * RPQ + 8 * i + lr;
@@ -468,18 +474,97 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (dead) break;
         if (tid == 0 && k < 12) TC_STAMP(80 + k);
         tc_fence_after_sync();
-        uint32_t sr[NH == 4 ? 2 : 1][32];
+        const bool is_draft = u < off;
+        const int stage = u % kStages;
+        const int nvalid = is_draft ? p.T : min(meta[stage], kUnit);
+        uint8_t *pbuf = smem + kOffP + wg * kPBytes;
+        if constexpr (NH == 4) {
+        // 128 query rows: one thread per row (tcgen05.ld 32x32b), no shuffles, 16-byte P stores; m[0] / l[0] hold
+        // the row's state until the loop ends
+        uint32_t sr[2][32];
+        tmem_ld_x32(t_s, sr[0]);
+        tmem_ld_x32(t_s + 32, sr[1]);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kSFree + wg));   // the next S of this warpgroup may be issued
+        float sc[64];
+#pragma unroll
+        for (int c = 0; c < 64; ++c) sc[c] = __uint_as_float(sr[c >> 5][c & 31]);
+        if (is_draft || nvalid < kUnit) {
+#pragma unroll
+            for (int c = 0; c < 64; ++c) {
+                bool ok = c < nvalid;
+                if (is_draft) ok = ok && ((row_vis >> c) & 1ull);
+                if (!ok) sc[c] = -INFINITY;
+            }
+        }
+        float mx4[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) mx4[a] = max3f(sc[16 * a], sc[16 * a + 1], sc[16 * a + 2]);
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+#pragma unroll
+            for (int c = 3; c < 15; c += 2) mx4[a] = max3f(mx4[a], sc[16 * a + c], sc[16 * a + c + 1]);
+            mx4[a] = fmaxf(mx4[a], sc[16 * a + 15]);
+        }
+        const float um = fmaxf(max3f(mx4[0], mx4[1], mx4[2]), mx4[3]) * p.scale_log2;
+        float factor = 1.f;
+        bool move = false;
+        if (um > m[0] + kLazy || (m[0] == -INFINITY && um > -INFINITY)) {
+            factor = fast_exp2(m[0] - um);   // 0 when there was no reference
+            m[0] = um;
+            l[0] *= factor;
+            move = true;
+        }
+        if (k > 0) {
+            wait_pv(k - 1);
+            if (dead) break;
+        }
+        if (k > 0 && __any_sync(0xffffffffu, move)) {
+            // rare: rescale this thread's row of O in TMEM
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld_x32(t_o + c * 32, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int x = 0; x < 32; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * factor);
+                tmem_st_x32(t_o + c * 32, r);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+        }
+        {
+            const float m_use = (m[0] == -INFINITY) ? 0.f : m[0];
+            const unsigned long long scale2 = f2_pack(p.scale_log2, p.scale_log2), neg_m2 = f2_pack(-m_use, -m_use);
+            unsigned long long lsum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
+            const uint32_t row = (uint32_t)(quad * 32 + lane);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float x0, x1;
+                    f2_unpack(f2_fma(f2_pack(sc[8 * j + 2 * e], sc[8 * j + 2 * e + 1]), scale2, neg_m2), x0, x1);
+                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                    lsum2[e & 1] = f2_add(lsum2[e & 1], f2_pack(p0, p1));
+                    pk[e] = pack_bf16(p0, p1);
+                }
+                *reinterpret_cast<uint4 *>(pbuf + swz128(row, j)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            float ls0, ls1;
+            f2_unpack(f2_add(lsum2[0], lsum2[1]), ls0, ls1);
+            l[0] += ls0 + ls1;
+        }
+        } else {
+        uint32_t sr[1][32];
         tmem_ld_16x256b_x8(t_s, sr[0]);
-        if constexpr (NH == 4) tmem_ld_16x256b_x8(t_s + (16u << 16), sr[1]);
         tmem_ld_wait();
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kSFree + wg));   // the next S of this warpgroup may be issued
 
-        const bool is_draft = u < off;
-        const int stage = u % kStages;
-        const int nvalid = is_draft ? p.T : min(meta[stage], kUnit);
-        uint8_t *pbuf = smem + kOffP + wg * kPBytes;
         float sc[NH][16], factor[NH];
         bool move = false;
 #pragma unroll
@@ -567,6 +652,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             f2_unpack(lsum2, ls0, ls1);
             l[i] += ls0 + ls1;
         }
+        }
         if (!is_draft && nvalid < kUnit) {
             // zero the value rows past the end of the sequence (0 * junk must stay 0)
             const int t = quad * 32 + lane;
@@ -580,6 +666,16 @@ __global__ void __launch_bounds__(kThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kPReady + wg));
         if (tid == 0 && k < 12) TC_STAMP(92 + k);
+    }
+    if constexpr (NH == 4) {
+        // back to the four-threads-per-row slots the read-out uses: slot i of this thread is row 8 i + lane / 4 of the warp
+        const float m_row = m[0], l_row = l[0];
+#pragma unroll
+        for (int i = 0; i < NH; ++i) {
+            m[i] = __shfl_sync(0xffffffffu, m_row, 8 * i + lr);
+            const float lv = __shfl_sync(0xffffffffu, l_row, 8 * i + lr);
+            l[i] = qd == 0 ? lv : 0.f;   // the read-out sums l over the four threads of a row
+        }
     }
     // ------------------------------------------------------------------ combine the two warpgroups, write out
     // Warp q of either warpgroup owns TMEM lane quadrant q, so warpgroup 0 can read warpgroup 1's accumulator
