@@ -32,9 +32,20 @@
 #include "attn_common.cuh"
 #include "sv_ptx.cuh"
 
+#ifndef SV_TRACE_U0
+#define SV_TRACE_U0 0
+#endif
 #ifdef SV_TRACE
-// Development aid (never compiled into the library): cycle stamps of the first CTAs.
+// Development aid (never compiled into the library): cycle stamps of the first CTAs (units SV_TRACE_U0 .. + 23) and
+// the wall-clock start / end of every CTA.
 __device__ long long g_sv_trace_tc[32 * 128];
+__device__ long long g_sv_trace_cta[1024 * 2];
+extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_cta()
+{
+    long long *p = nullptr;
+    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace_cta);
+    return p;
+}
 extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_tc()
 {
     long long *p = nullptr;
@@ -45,6 +56,12 @@ extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_tc(
     do {                                                                                   \
         const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);   \
         if (cta_ < 32 && (slot) < 128) g_sv_trace_tc[cta_ * 128 + (slot)] = clock64();     \
+        if ((slot) == 0 || (slot) == 120) {                                                \
+            long long ns_;                                                                 \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_));                        \
+            if (cta_ < 32) g_sv_trace_tc[cta_ * 128 + ((slot) == 0 ? 121 : 122)] = ns_;    \
+            if (cta_ < 1024) g_sv_trace_cta[cta_ * 2 + ((slot) == 0 ? 0 : 1)] = ns_;       \
+        }                                                                                  \
     } while (0)
 #else
 #define TC_STAMP(slot) \
@@ -56,6 +73,7 @@ namespace svk {
 namespace {
 
 constexpr int kThreads = 384;
+constexpr int kTraceU0 = SV_TRACE_U0;
 constexpr int kUnit = 64;                        // keys per unit
 constexpr int kTile = kUnit * 128;               // bytes of one [64 rows][64 bf16] half tile (8 KB)
 constexpr int kStageBytes = 4 * kTile;           // K lo/hi + V lo/hi
@@ -70,7 +88,6 @@ constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 static_assert(2 * kStages + 10 <= 32, "one lane of the producer warp per barrier");
 constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns
-constexpr int kMergeStride = 132;                // floats per row of the cross-warpgroup merge buffer
 
 // barrier slots (8 bytes each) inside the misc area
 enum Bar {
@@ -200,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             const int y = r0 + uo * kUnit;
                             // an empty unit (block 128, tail of at most 64 tokens) is still loaded:
                             // it keeps the unit sequence uniform and is fully masked downstream
-                            if (u < 24) TC_STAMP(8 + u);
+                            if (u >= kTraceU0 && u < kTraceU0 + 24) TC_STAMP(8 + u - kTraceU0);
                             mbar_arrive_expect_tx(fb, kStageBytes);
                             tma_load_2d(dst, &tm_k, 0, y, fb, policy);
                             tma_load_2d(dst + kTile, &tm_k, 64, y, fb, policy);
@@ -250,7 +267,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             tc_mma_bf16(d, d_hi | (dq_lo + qo), d_hi | (k_lo + ko), idesc_s, ks > 0);
                         }
                         tc_commit(bar(kSReady + g));
-                        if (u < 24) TC_STAMP(32 + u);
+                        if (u >= kTraceU0 && u < kTraceU0 + 24) TC_STAMP(32 + u - kTraceU0);
                     }
                     // free TMEM only after every softmax warp has finished reading it
                     if (!mbar_wait_bounded(bar(kTmemDone), 0) && p.status) atomicOr(p.status, 16);
@@ -279,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                                         idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);   // the warpgroup's first unit starts O
                         tc_commit(bar(kOReady + g));
                         tc_commit(bar(kEmpty + stage));
-                        if (u < 24) TC_STAMP(56 + u);
+                        if (u >= kTraceU0 && u < kTraceU0 + 24) TC_STAMP(56 + u - kTraceU0);
                     }
                 }
             }
@@ -472,7 +489,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (p.status && lane == 0) atomicOr(p.status, 2);
         }
         if (dead) break;
-        if (tid == 0 && k < 12) TC_STAMP(80 + k);
+        if (tid == 0 && k >= kTraceU0 / 2 && k < kTraceU0 / 2 + 12) TC_STAMP(80 + k - kTraceU0 / 2);
         tc_fence_after_sync();
         const bool is_draft = u < off;
         const int stage = u % kStages;
@@ -665,7 +682,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kPReady + wg));
-        if (tid == 0 && k < 12) TC_STAMP(92 + k);
+        if (tid == 0 && k >= kTraceU0 / 2 && k < kTraceU0 / 2 + 12) TC_STAMP(92 + k - kTraceU0 / 2);
     }
     if constexpr (NH == 4) {
         // back to the four-threads-per-row slots the read-out uses: slot i of this thread is row 8 i + lane / 4 of the warp
