@@ -133,6 +133,9 @@ SMALL = {
     # multi-head attention (G = 1), a wide GQA group (G = 16, 128 rows), block 128 whose tail holds <= 64 tokens
     "mha": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=4, seq_len=(1200, 1200), budget_blocks=6, planted=2),
     "g16": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1500, 1500), budget_blocks=6, n_draft=8, planted=2),
+    # 65-128 rows (one softmax thread per row) with idle warps and padding rows: 80 rows (3 of 4 warps), 104 rows
+    "rows80_tree": si.shrink(si.WORKLOADS["cfg1"], seq_len=(2100, 2100), budget_blocks=9, n_draft=20, n_layers=1, tree=True, planted=2),
+    "rows104": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(1500, 2600), budget_blocks=5, n_draft=13, planted=2),
     # more than 128 query rows per KV head (several row tiles) and more than 32 draft tokens (64-bit ancestor masks)
     "t60_tree": si.shrink(si.WORKLOADS["cfg1"], seq_len=(3000, 3000), budget_blocks=10, n_draft=60, n_layers=1, tree=True, planted=3),
     "t40_chain_2seq": si.shrink(si.WORKLOADS["cfg2"], n_seq=2, seq_len=(900, 2100), budget_blocks=7, n_draft=40, planted=2),
