@@ -695,71 +695,65 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     }
     // ------------------------------------------------------------------ combine the two warpgroups, write out
-    // Warp q of either warpgroup owns TMEM lane quadrant q, so warpgroup 0 can read warpgroup 1's accumulator
-    // straight from TMEM: warpgroup 1 only waits for its last PV, leaves its (m, l) in its own (now idle) P tile and
-    // signals; warpgroup 0 fetches both accumulators, merges them in registers and writes the rows out.
+    // Warp q of either warpgroup owns TMEM lane quadrant q, so each warpgroup can read the other's accumulator straight
+    // from TMEM: both wait for their last PV, exchange (m, l) through their own (now idle) P tiles, and then each merges
+    // and writes one half of the 128 output columns of every row.
     const int n_sm = 2 * wg_threads;
     const int t = quad * 32 + lane;
-    float *ml1 = reinterpret_cast<float *>(smem + kOffP + kPBytes);   // [2 * NH][128]: m, l of warpgroup 1's slots
+    float *ml_mine = reinterpret_cast<float *>(smem + kOffP + wg * kPBytes);          // [2 * NH][128]: m, l per slot
+    float *ml_other = reinterpret_cast<float *>(smem + kOffP + (wg ^ 1) * kPBytes);
     // Only now may the dependent kernel (the split merge) be scheduled: released at the start, its small CTAs would all
     // become resident on the few SMs this grid leaves idle and later do the whole merge from there; released here,
     // they spread over the SMs that the attention CTAs are about to vacate.
     grid_launch_dependents();
     if (k > 0) wait_pv(k - 1);   // this warpgroup's accumulator is complete
-    if (wg == 1) {
 #pragma unroll
-        for (int i = 0; i < NH; ++i) {
-            ml1[(2 * i) * 128 + t] = m[i];
-            ml1[(2 * i + 1) * 128 + t] = l[i];
-        }
-        tc_fence_before_sync();
-        named_bar_arrive(1, n_sm);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(kTmemDone));   // this warpgroup reads TMEM no more
-        return;
+    for (int i = 0; i < NH; ++i) {
+        ml_mine[(2 * i) * 128 + t] = m[i];
+        ml_mine[(2 * i + 1) * 128 + t] = l[i];
     }
+    tc_fence_before_sync();
     if (tid == 0) TC_STAMP(104);
     named_bar_sync(1, n_sm);
     tc_fence_after_sync();
     if (tid == 0) TC_STAMP(106);
-    const bool have0 = k > 0 && !dead, have1 = n_total >= 2;   // a warpgroup without units never wrote its accumulator
-    // this warp's rows of O: 32 output dims 8*jj + 2*qd + e (index 2*jj + e) per slot
-    float o[NH][32], w0[NH], w1[NH], row_m[NH], row_l[NH];
+    // a warpgroup without units never wrote its accumulator
+    const bool have_mine = k > 0 && !dead, have_other = n_total >= (wg == 0 ? 2 : 1);
+    const uint32_t t_o_other = tmem_base + t_lane + 128 + (wg ^ 1) * 128;
+    // this warp's rows of O, the warpgroup's half of the columns: 16 output dims 64 wg + 8 j + 2 qd + e (index 2 j + e)
+    float o[NH][16], row_m[NH], row_l[NH];
 #pragma unroll
-    for (int i = 0; i < NH; ++i) {
-        const float m1 = ml1[(2 * i) * 128 + t], l1 = ml1[(2 * i + 1) * 128 + t];
-        const float M = fmaxf(m[i], m1);
-        const float M_use = (M == -INFINITY) ? 0.f : M;
-        w0[i] = fast_exp2(m[i] - M_use), w1[i] = fast_exp2(m1 - M_use);
-        float lsum = w0[i] * l[i] + w1[i] * l1;
-        lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
-        lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-        row_m[i] = M, row_l[i] = lsum;
-    }
+    for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo) {
+        uint32_t r0[32], r1[32];
+        if (have_mine) tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + wg * 64, r0);
+        if (have_other) tmem_ld_16x256b_x8(t_o_other + ((uint32_t)(lo * 16) << 16) + wg * 64, r1);
 #pragma unroll
-    for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo)
+        for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh) {
+            const int i = lo * 2 + hh;
+            const float m1 = ml_other[(2 * i) * 128 + t], l1 = ml_other[(2 * i + 1) * 128 + t];
+            const float M = fmaxf(m[i], m1);
+            const float M_use = (M == -INFINITY) ? 0.f : M;
+            const float w0 = fast_exp2(m[i] - M_use), w1 = fast_exp2(m1 - M_use);
+            float lsum = w0 * l[i] + w1 * l1;
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            row_m[i] = M, row_l[i] = lsum;
+            if (hh == 0) tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            uint32_t r0[32], r1[32];
-            if (have0) tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + c * 64, r0);
-            if (have1) tmem_ld_16x256b_x8(t_o + 128 + ((uint32_t)(lo * 16) << 16) + c * 64, r1);
-            tmem_ld_wait();
+            for (int j = 0; j < 8; ++j)
 #pragma unroll
-            for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh)
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int i = lo * 2 + hh, x = 4 * j + 2 * hh + e;
-                        const float a = have0 ? w0[i] * __uint_as_float(r0[x]) : 0.f;
-                        const float b = have1 ? w1[i] * __uint_as_float(r1[x]) : 0.f;
-                        o[i][(c * 8 + j) * 2 + e] = a + b;
-                    }
+                for (int e = 0; e < 2; ++e) {
+                    const int x = 4 * j + 2 * hh + e;
+                    const float a = have_mine ? w0 * __uint_as_float(r0[x]) : 0.f;
+                    const float b = have_other ? w1 * __uint_as_float(r1[x]) : 0.f;
+                    o[i][2 * j + e] = a + b;
+                }
         }
+    }
     if (tid == 0) TC_STAMP(105);
     tc_fence_before_sync();
     __syncwarp();
-    if (lane == 0) mbar_arrive(bar(kTmemDone));
+    if (lane == 0) mbar_arrive(bar(kTmemDone));   // this warp reads TMEM no more
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
         const float M = row_m[i], lsum = row_l[i];
@@ -769,16 +763,16 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int ii = row / p.G, g = row - ii * p.G;
             const size_t orow = ((size_t)s * p.T + i0 + ii) * p.Hq + h * p.G + g;
             const float inv = 1.f / lsum;
-            uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + qd;
+            uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + wg * 32 + qd;
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) dst[4 * jj] = pack_bf16(o[i][2 * jj] * inv, o[i][2 * jj + 1] * inv);
-            if (p.lse && qd == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
+            for (int j = 0; j < 8; ++j) dst[4 * j] = pack_bf16(o[i][2 * j] * inv, o[i][2 * j + 1] * inv);
+            if (p.lse && wg == 0 && qd == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
         } else {
             const size_t prow = (((size_t)s * p.Hkv + h) * p.splits + split) * (p.G * p.T) + i0 * p.G + row;
-            float2 *dst = reinterpret_cast<float2 *>(p.ws_o + prow * 128) + qd;
+            float2 *dst = reinterpret_cast<float2 *>(p.ws_o + prow * 128) + wg * 32 + qd;
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) dst[4 * jj] = make_float2(o[i][2 * jj], o[i][2 * jj + 1]);
-            if (qd == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
+            for (int j = 0; j < 8; ++j) dst[4 * j] = make_float2(o[i][2 * j], o[i][2 * j + 1]);
+            if (wg == 0 && qd == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
         }
     }
     if (tid == 0) TC_STAMP(120);
