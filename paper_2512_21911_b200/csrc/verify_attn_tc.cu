@@ -134,6 +134,21 @@ __global__ void __launch_bounds__(kThreads, 1)
     constexpr int RPQ = 8 * NH;                              // query rows per TMEM lane quadrant
     const int n_active = min(4, (rows + RPQ - 1) / RPQ);     // warps per softmax warpgroup that own real rows
 
+    // r / G for the small row indices of this kernel (0 <= r < 8192, 1 <= G <= 128) without an integer division:
+    // (r + 0.5) / G is at least 0.5 / G >= 2^-8 away from the next integer, far more than the fp32 rounding error
+    // First block of split k's slice of a list of n blocks.  With 65-128 rows the draft tokens' unit of the last split
+    // costs about as much as three ordinary units (masking 64 columns per thread, a first pass through that code), so
+    // there the list is cut as if it were that much longer and the last slice comes out shorter.
+    auto slice_begin = [&](int k, int n) {
+        if constexpr (NH == 4) {
+            const int w_draft = (3 + upb - 1) / upb;
+            return min(n, (int)((long long)k * (n + w_draft) / p.splits));
+        } else {
+            return (int)((long long)k * n / p.splits);
+        }
+    };
+    const float inv_g = 1.f / (float)p.G;
+    auto div_g = [&](int r) { return (int)(((float)r + 0.5f) * inv_g); };
     if (tid == 0) TC_STAMP(0);
     // The TMA producer warp initialises the barriers and runs ahead; everybody else meets it at a named
     // barrier (the producer only arrives), with the TMEM allocation done by warp 9 on the way.
@@ -173,15 +188,15 @@ __global__ void __launch_bounds__(kThreads, 1)
             grid_dependency_wait();   // the block list is written by the kernel just before
             // First batch of block indices speculatively, assuming the list is full (cnt == max_sel): its
             // load then overlaps the loads of the count and the length instead of following them.
-            const int j0_spec = (int)((long long)split * p.max_sel / p.splits);
+            const int j0_spec = slice_begin(split, p.max_sel);
             int blk_spec = 0;
             if (p.sel_idx && j0_spec + lane < p.max_sel)
                 blk_spec = p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j0_spec + lane];
             const int L = p.seq_lens[s];
             const int nb = min((L + p.B - 1) / p.B, p.NBmax);
             const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-            const int j0 = (int)((long long)split * n_sel / p.splits);
-            const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+            const int j0 = slice_begin(split, n_sel);
+            const int j1 = slice_begin(split + 1, n_sel);
             const int off = has_draft ? 1 : 0;
             bool dead = false;
             for (int base = j0; base < j1; base += 32) {
@@ -236,8 +251,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                 grid_dependency_wait();
                 const int nb = min((L + p.B - 1) / p.B, p.NBmax);
                 const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-                const int j0 = (int)((long long)split * n_sel / p.splits);
-                const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+                const int j0 = slice_begin(split, n_sel);
+                const int j1 = slice_begin(split + 1, n_sel);
                 const int off = has_draft ? 1 : 0;
                 const int n_total = (j1 - j0) * upb + off;
                 bool dead = !mbar_wait_bounded(bar(kStaged), 0);
@@ -332,29 +347,33 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     }
     grid_dependency_wait();
+    if (tid == 0) TC_STAMP(3);
     {
-        // real rows: all loads of a thread are in flight together
+        // real rows: all loads of a thread are in flight together (16-byte chunks: Q up to 128 rows x 16, draft K and
+        // V up to 64 tokens x 16 each)
+        constexpr int kQB = NH == 4 ? 8 : 4, kDB = kWide ? 8 : 4;
         const int n_q = rows * 16, n_d = has_draft ? 2 * p.T * 16 : 0;
-        uint4 v[4];
+        uint4 v[kQB];
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
+        for (int x = 0; x < kQB; ++x) {
             const int idx = tid + x * 256;
             if (idx < n_q) {
                 const int r = idx >> 4, c = idx & 15;
-                const int i = r / p.G, g = r - i * p.G;
+                const int i = div_g(r), g = r - i * p.G;
                 v[x] = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i0 + i) * p.Hq + h * p.G + g) * 128) + c);
             }
         }
-        uint4 w[4];
+        uint4 w[kDB];
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
+        for (int x = 0; x < kDB; ++x) {
             const int idx = tid + x * 256;
             if (idx < n_d) {
-                const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
+                const int which = (idx >> 4) >= p.T, r = (idx >> 4) - which * p.T, c = idx & 15;   // K rows, then V rows
                 const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
                 w[x] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
             }
         }
+        if (tid == 0) TC_STAMP(4);
         if (!kWide && has_draft && tid < 32) {
             uint32_t mask = 0;
             if (tid < p.T) {
@@ -388,33 +407,24 @@ __global__ void __launch_bounds__(kThreads, 1)
             anc[tid] = mask;
         }
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
+        for (int x = 0; x < kQB; ++x) {
             const int idx = tid + x * 256;
             if (idx < n_q) {
                 const int r = idx >> 4, c = idx & 15;
                 const int tr = (r / RPQ) * 32 + (r % RPQ);
                 *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = v[x];
             }
+        }
+#pragma unroll
+        for (int x = 0; x < kDB; ++x) {
+            const int idx = tid + x * 256;
             if (idx < n_d) {
-                const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
+                const int which = (idx >> 4) >= p.T, r = (idx >> 4) - which * p.T, c = idx & 15;
                 *reinterpret_cast<uint4 *>(smem + kOffDraft + which * (2 * kTile) + (c >> 3) * kTile + swz128(r, c & 7)) = w[x];
             }
         }
-        // shapes with more than 64 query rows or more than 16 draft tokens: the remaining chunks
-        for (int idx = tid + 4 * 256; idx < n_q; idx += 256) {
-            const int r = idx >> 4, c = idx & 15;
-            const int i = r / p.G, g = r - i * p.G;
-            const int tr = (r / RPQ) * 32 + (r % RPQ);
-            *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) =
-                __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i0 + i) * p.Hq + h * p.G + g) * 128) + c);
-        }
-        for (int idx = tid + 4 * 256; idx < n_d; idx += 256) {
-            const int which = idx / (p.T * 16), r = (idx >> 4) % p.T, c = idx & 15;
-            const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
-            *reinterpret_cast<uint4 *>(smem + kOffDraft + which * (2 * kTile) + (c >> 3) * kTile + swz128(r, c & 7)) =
-                __ldg(reinterpret_cast<const uint4 *>(src) + c);
-        }
     }
+    if (tid == 0) TC_STAMP(5);
     fence_proxy_async();   // the tensor cores read these tiles through the async proxy
     named_bar_sync(2, 256);
     if (lane == 0) mbar_arrive(bar(kStaged));
@@ -434,7 +444,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     unsigned long long row_vis = ~0ull;   // NH == 4: the draft tokens row quad * 32 + lane may see
     if constexpr (NH == 4) {
         const int r = quad * 32 + lane;
-        if (has_draft && r < rows) row_vis = kWide ? anc[i0 + r / p.G] : (unsigned long long)anc32[r / p.G];
+        if (has_draft && r < rows) row_vis = kWide ? anc[i0 + div_g(r)] : (unsigned long long)anc32[div_g(r)];
     }
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
@@ -442,22 +452,22 @@ __global__ void __launch_bounds__(kThreads, 1)
         trow[i] = quad * 32 + 8 * i + lr;
         if constexpr (kWide) {
             const unsigned long long all_t = (p.T == 64) ? ~0ull : ((1ull << p.T) - 1ull);
-            const unsigned long long row_vis = (has_draft && lrow[i] < rows) ? anc[i0 + lrow[i] / p.G] : all_t;
+            const unsigned long long row_vis = (has_draft && lrow[i] < rows) ? anc[i0 + div_g(lrow[i])] : all_t;
             uint32_t mine = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) mine |= (uint32_t)((row_vis >> (8 * j + 2 * qd)) & 3ull) << (2 * j);
             vis[i] = mine;
         } else {
             const uint32_t all_t = (p.T == 32) ? 0xFFFFFFFFu : ((1u << p.T) - 1u);
-            vis[i] = (has_draft && lrow[i] < rows) ? anc32[lrow[i] / p.G] : all_t;
+            vis[i] = (has_draft && lrow[i] < rows) ? anc32[div_g(lrow[i])] : all_t;
         }
     }
 
     const int L = p.seq_lens[s];
     const int nb = min((L + p.B - 1) / p.B, p.NBmax);
     const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-    const int j0 = (int)((long long)split * n_sel / p.splits);
-    const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
+    const int j0 = slice_begin(split, n_sel);
+    const int j1 = slice_begin(split + 1, n_sel);
     const int off = has_draft ? 1 : 0;
     const int n_total = (j1 - j0) * upb + off;
 
@@ -509,11 +519,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
         for (int c = 0; c < 64; ++c) sc[c] = __uint_as_float(sr[c >> 5][c & 31]);
         if (is_draft || nvalid < kUnit) {
+            unsigned long long allowed = nvalid >= 64 ? ~0ull : ((1ull << nvalid) - 1ull);
+            if (is_draft) allowed &= row_vis;
+            const uint32_t a_lo = (uint32_t)allowed, a_hi = (uint32_t)(allowed >> 32);
 #pragma unroll
-            for (int c = 0; c < 64; ++c) {
-                bool ok = c < nvalid;
-                if (is_draft) ok = ok && ((row_vis >> c) & 1ull);
-                if (!ok) sc[c] = -INFINITY;
+            for (int c = 0; c < 32; ++c) {
+                if (!((a_lo >> c) & 1u)) sc[c] = -INFINITY;
+                if (!((a_hi >> c) & 1u)) sc[32 + c] = -INFINITY;
             }
         }
         float mx4[4];
@@ -760,7 +772,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int row = lrow[i];
         if (row >= rows) continue;
         if (p.splits == 1) {
-            const int ii = row / p.G, g = row - ii * p.G;
+            const int ii = div_g(row), g = row - ii * p.G;
             const size_t orow = ((size_t)s * p.T + i0 + ii) * p.Hq + h * p.G + g;
             const float inv = 1.f / lsum;
             uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + wg * 32 + qd;
