@@ -139,12 +139,14 @@ __global__ void __launch_bounds__(kThreads, 1)
     // First block of split k's slice of a list of n blocks.  With 65-128 rows the draft tokens' unit of the last split
     // costs about as much as three ordinary units (masking 64 columns per thread, a first pass through that code), so
     // there the list is cut as if it were that much longer and the last slice comes out shorter.
+    // (Up to 64 rows: 32-bit products -- k <= 148 splits, n <= 32768 blocks -- because a 64-bit division here costs every
+    // CTA of a short launch 0.3 us before its first load; the 128-row instantiation measured faster with the 64-bit form.)
     auto slice_begin = [&](int k, int n) {
         if constexpr (NH == 4) {
             const int w_draft = (3 + upb - 1) / upb;
             return min(n, (int)((long long)k * (n + w_draft) / p.splits));
         } else {
-            return (int)((long long)k * n / p.splits);
+            return (int)((uint32_t)k * (uint32_t)n / (uint32_t)p.splits);
         }
     };
     const float inv_g = 1.f / (float)p.G;
@@ -193,7 +195,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (p.sel_idx && j0_spec + lane < p.max_sel)
                 blk_spec = p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j0_spec + lane];
             const int L = p.seq_lens[s];
-            const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+            const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
             const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
             const int j0 = slice_begin(split, n_sel);
             const int j1 = slice_begin(split + 1, n_sel);
@@ -249,7 +251,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (lane == 0) {
                 const int L = p.seq_lens[s];
                 grid_dependency_wait();
-                const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+                const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
                 const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
                 const int j0 = slice_begin(split, n_sel);
                 const int j1 = slice_begin(split + 1, n_sel);
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
 
     const int L = p.seq_lens[s];
-    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
+    const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
     const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
     const int j0 = slice_begin(split, n_sel);
     const int j1 = slice_begin(split + 1, n_sel);
