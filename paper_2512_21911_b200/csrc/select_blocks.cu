@@ -80,13 +80,13 @@ __device__ __forceinline__ uint32_t cluster_map_shared(uint32_t addr, uint32_t r
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_shared_cluster_v4(uint32_t addr, uint4 v)
+// 16-byte store into another CTA's shared memory that reports its bytes to an mbarrier there when it has landed: the
+// receiver needs no fence and no separate arrival from the sender
+__device__ __forceinline__ void st_async_cluster_v4(uint32_t addr, uint4 v, uint32_t remote_bar)
 {
-    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(remote_bar)
+                 : "memory");
 }
 __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t parity, uint32_t limit = (1u << 19))
 {
@@ -105,8 +105,8 @@ __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t
 }
 
 // Cluster of CL CTAs per (sequence, KV head).  Every CTA scores a slice of the blocks and writes the
-// keys straight into CTA 0's shared memory (distributed shared memory), then signals an mbarrier there
-// and exits; CTA 0 selects.  The only cluster-wide barrier is split (arrive early, wait late) so that
+// keys straight into CTA 0's shared memory (distributed shared memory) with stores that count their bytes
+// on an mbarrier there, and exits; CTA 0 waits for the expected number of bytes and selects.  The only cluster-wide barrier is split (arrive early, wait late) so that
 // its latency hides behind the loads.
 // kBf16: the representatives are stored in bfloat16 (storage variant); scores are fp32 either way.
 template <bool kBf16>
@@ -125,14 +125,14 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     __shared__ uint32_t cand_n;
     __shared__ uint32_t pass_bin[3];               // boundary bin of a radix pass: index, keys still to take in it, its size
     __shared__ uint32_t warp_sel[kWarps], warp_eq[kWarps];
-    __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: one arrival per CTA of the cluster
+    __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: the bytes of all keys (one arrival: CTA 0 itself)
 
     SEL_STAMP(0);
     // While the kernel that precedes this one in the stream drains: pull this warp's first batch of
     // representative rows and the query row towards L2 (a prefetch consumes no data, so it is safe even if
     // that kernel is still writing them), set up the barrier, zero the histograms.
     if (tid == 0) {
-        svk::mbar_init(svk::smem_u32(&keys_ready), CL);
+        svk::mbar_init(svk::smem_u32(&keys_ready), 1);
         svk::mbar_fence_init();
     }
     for (int i = tid; i < 4 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
@@ -195,6 +195,14 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     SEL_STAMP(12);
 
     const uint32_t keys0 = cluster_map_shared(svk::smem_u32(keys_all), 0);
+    const uint32_t ready0 = cluster_map_shared(svk::smem_u32(&keys_ready), 0);
+    if (rank == 0 && tid == 0) {
+        // what the cluster is about to send: one 16-byte store per four keys of every CTA's slice
+        uint32_t quads = 0;
+        if (!keep_all)
+            for (int r = 0; r < CL; ++r) quads += (uint32_t)(max(0, min(p.chunk, nb - r * p.chunk)) + 3) >> 2;
+        svk::mbar_arrive_expect_tx(svk::smem_u32(&keys_ready), 16u * quads);
+    }
     if (need_scores) {
         const float4 qv = reinterpret_cast<const float4 *>(qbar)[lane];
         for (; b < b1; b += kWarps * kRowsPerIter) {
@@ -210,22 +218,18 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                 if (p.out_scores && lane == 0 && bb < b1) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = d;
             }
             // rows b .. b+3 are 4 consecutive keys: one 16-byte store into CTA 0 (entries past nb are never read)
-            if (lane == 0 && !keep_all) st_shared_cluster_v4(keys0 + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]));
+            if (lane == 0 && !keep_all) st_async_cluster_v4(keys0 + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]), ready0);
             if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter, b1);
         }
     }
     SEL_STAMP(13);
-    __syncthreads();   // the release (cluster scope) of the arrive below covers the stores this barrier ordered before it
-    SEL_STAMP(4);
-    if (tid == 0) mbar_arrive_cluster(cluster_map_shared(svk::smem_u32(&keys_ready), 0));
     if (rank != 0) return;
+    SEL_STAMP(4);
 
     int32_t *out = p.out_idx + ((size_t)s * p.Hkv + h) * p.max_sel;
     if (keep_all) {
         for (int bb = tid; bb < nb; bb += kThreads) out[bb] = bb;
         if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = nb;
-        // the other CTAs still signal the barrier in this CTA's shared memory: wait for them before exiting
-        mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0);
         return;
     }
     if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) return;   // gave up: leave the output untouched
