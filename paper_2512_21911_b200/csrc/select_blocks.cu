@@ -125,6 +125,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     __shared__ uint32_t cand_n;
     __shared__ uint32_t pass_bin[3];               // boundary bin of a radix pass: index, keys still to take in it, its size
     __shared__ uint32_t warp_sel[kWarps], warp_eq[kWarps];
+    __shared__ uint32_t key_min, key_max;          // smallest / largest evictable key (fast path)
     __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: the bytes of all keys (one arrival: CTA 0 itself)
 
     SEL_STAMP(0);
@@ -132,6 +133,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     // representative rows and the query row towards L2 (a prefetch consumes no data, so it is safe even if
     // that kernel is still writing them), set up the barrier, zero the histograms.
     if (tid == 0) {
+        key_min = 0xFFFFFFFFu, key_max = 0u, cand_n = 0;
         svk::mbar_init(svk::smem_u32(&keys_ready), 1);
         svk::mbar_fence_init();
     }
@@ -255,11 +257,12 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         }
         kmin = __reduce_min_sync(0xffffffffu, kmin);
         kmax = __reduce_max_sync(0xffffffffu, kmax);
-        if (lane == 0) warp_sel[warp] = kmin, warp_eq[warp] = kmax;
-        if (tid == 0) cand_n = 0;
+        if (lane == 0) {
+            atomicMin(&key_min, kmin);
+            atomicMax(&key_max, kmax);
+        }
         __syncthreads();
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) kmin = min(kmin, warp_sel[w]), kmax = max(kmax, warp_eq[w]);
+        kmin = key_min, kmax = key_max;
         const float xmin = key_score(kmin), xmax = key_score(kmax);
         const float scale = 65535.f / (xmax - xmin);
         const uint32_t R = (uint32_t)(N - forced);   // evictable blocks to keep: 0 <= R < number of evictable blocks
@@ -312,7 +315,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                 need = pass_bin[1];
                 in_bin = pass_bin[2];
                 settled = need == in_bin || in_bin <= (uint32_t)kFastCap;
-                __syncthreads();   // pass_bin is rewritten by the next level
+                if (!settled) __syncthreads();   // block-uniform; pass_bin is rewritten by the next level
             }
             if (settled) {   // block-uniform
                 const bool rank_them = need < in_bin;   // otherwise every key at the boundary prefix is kept
@@ -361,7 +364,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                         }
                         if (sel[c]) out[base + before + __popc(ballot & ((1u << lane) - 1u))] = c * kThreads + tid;
                         base += total;
-                        __syncthreads();
+                        if ((c + 1) * kThreads < nb) __syncthreads();   // block-uniform; warp_sel is rewritten by the next round
                     }
                 }
                 if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
