@@ -403,7 +403,7 @@ def run_gpu(args):
                      "peak_kind": f"of {peak_kind}",
                      # dram__bytes_read.sum + dram__bytes_write.sum of verify_attn_tc_kernel<1> from the ncu capture
                      # summarised in profiles/cfg1_step_tcgen05_4layers.md (same shapes, per launch)
-                     "traffic": 16952832 if (w.n_layers, w.budget_blocks) == (32, 64) else None,
+                     "traffic": 16931840 if (w.n_layers, w.budget_blocks) == (32, 64) else None,
                      "kernel": "sv_verify_attn (split-KV attention + split merge), one launch per layer",
                      "bytes_per_launch": attn_bytes, "us_per_launch": us_attn},
         "kv_gathered_gbs": gathered / (us_attn * 1e-6) / 1e9,
