@@ -180,6 +180,9 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     float qsum = 0.f;
     if (tid < 128)
         for (int g = 0; g < G; ++g) qsum += __bfloat162float(q0[(size_t)g * 128 + tid]);
+    // CTA 0's barrier is initialised (every CTA arrived before its first global request); the wait costs a few hundred
+    // cycles even then, so it sits here, behind the loads it can overlap with
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 
     const int nb = min((L + p.B - 1) / p.B, p.NBmax);
     const int forced = min(nb, p.n_sink + p.n_local);
@@ -193,16 +196,14 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     if (tid < 128) qbar[tid] = qsum / (float)G;
     __syncthreads();
     SEL_STAMP(3);
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // CTA 0's barrier is initialised
     SEL_STAMP(12);
 
     const uint32_t keys0 = cluster_map_shared(svk::smem_u32(keys_all), 0);
     const uint32_t ready0 = cluster_map_shared(svk::smem_u32(&keys_ready), 0);
     if (rank == 0 && tid == 0) {
-        // what the cluster is about to send: one 16-byte store per four keys of every CTA's slice
-        uint32_t quads = 0;
-        if (!keep_all)
-            for (int r = 0; r < CL; ++r) quads += (uint32_t)(max(0, min(p.chunk, nb - r * p.chunk)) + 3) >> 2;
+        // what the cluster is about to send: one 16-byte store per four keys of every CTA's slice; the slices are
+        // multiples of four blocks long and only the last one in use can be ragged, so that is ceil(nb / 4) stores
+        const uint32_t quads = keep_all ? 0u : (uint32_t)(nb + 3) >> 2;
         svk::mbar_arrive_expect_tx(svk::smem_u32(&keys_ready), 16u * quads);
     }
     if (need_scores) {
