@@ -16,8 +16,9 @@
 namespace {
 
 constexpr int kOverlapThreads = 256;
-constexpr int kGlobalThreads = 1024;
+constexpr int kGlobalThreads = 512;   // block barriers dominate this kernel: 1024 threads 32.7 us per cold call, 512 24.6, 256 26.6
 constexpr int kGlobalWarps = kGlobalThreads / 32;
+constexpr int kMaxParts = 128;          // parts of the ordered compaction (heads x warps per head)
 constexpr int kMaxGlobalKeys = 49152;   // (head, block) pairs of one sequence held in shared memory (192 KB)
 
 // One CTA per (sequence, KV head): bitmap of every token's set, then all pairs.
@@ -91,7 +92,8 @@ __global__ void __launch_bounds__(kGlobalThreads) select_global_kernel(const flo
     extern __shared__ uint32_t keys[];   // [Hkv][NBmax]
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_tot[kGlobalWarps];
-    __shared__ uint32_t s_prefix, s_need;
+    __shared__ uint32_t s_prefix, s_need, s_and, s_or;
+    __shared__ int part_gt[kMaxParts], part_eq[kMaxParts];   // per part: blocks kept for sure / ties; later: start position / ties before
     const int s = blockIdx.x, tid = threadIdx.x;
     svk::grid_dependency_wait();   // the scores come from the kernel just before
     svk::grid_launch_dependents();
@@ -114,22 +116,42 @@ __global__ void __launch_bounds__(kGlobalThreads) select_global_kernel(const flo
         if (b < nb) k = (b < n_sink || b >= nb - n_local) ? 0xFFFFFFFFu : order_key(scores[((size_t)s * Hkv + h) * NBmax + b]);
         keys[e] = k;
     }
-    // K-th largest key among the evictable blocks: 4 passes of 8 bits, most significant first
+    // K-th largest key among the evictable blocks: passes of up to 8 bits, most significant first.  The keys of one
+    // sequence share their leading bits (same sign, neighbouring exponents), so the digits start at the highest bit in
+    // which any two evictable keys differ: the first pass then spreads the keys over the bins instead of piling
+    // them into a few (shared-memory atomics on one address serialise).
+    uint32_t k_and = 0xFFFFFFFFu, k_or = 0u;
+    for (int e = tid; e < n; e += kGlobalThreads) {
+        const uint32_t k = keys[e];
+        if (k != 0u && k != 0xFFFFFFFFu) k_and &= k, k_or |= k;
+    }
+    k_and = __reduce_and_sync(0xffffffffu, k_and);
+    k_or = __reduce_or_sync(0xffffffffu, k_or);
     if (tid == 0) {
         s_prefix = 0u;
         s_need = (uint32_t)max(0, N * Hkv - forced_per_head * Hkv);
+        s_and = 0xFFFFFFFFu, s_or = 0u;
+    }
+    __syncthreads();
+    if ((tid & 31) == 0) {
+        atomicAnd(&s_and, k_and);
+        atomicOr(&s_or, k_or);
     }
     __syncthreads();
     const bool take_none = s_need == 0u;
-    uint32_t mask = 0u;
-    for (int pass = 3; pass >= 0 && !take_none; --pass) {
+    const uint32_t diff = s_and ^ s_or;               // 0: every evictable key is the same (or there is none)
+    int top = diff ? 32 - __clz(diff) : 0;           // bits [0, top) still undecided
+    uint32_t mask = top >= 32 ? 0u : ~((1u << top) - 1u);
+    if (tid == 0) s_prefix = s_or & mask;             // the common leading bits
+    __syncthreads();
+    while (top > 0 && !take_none) {
+        const int w = min(8, top), shift = top - w;
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
         const uint32_t prefix = s_prefix;
-        const int shift = 8 * pass;
         for (int e = tid; e < n; e += kGlobalThreads) {
             const uint32_t k = keys[e];
-            if (k != 0u && k != 0xFFFFFFFFu && (k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+            if (k != 0u && k != 0xFFFFFFFFu && (k & mask) == prefix) atomicAdd(&hist[(k >> shift) & ((1u << w) - 1u)], 1u);
         }
         __syncthreads();
         if (tid < 32) {
@@ -162,11 +184,89 @@ __global__ void __launch_bounds__(kGlobalThreads) select_global_kernel(const flo
                 s_prefix = prefix | ((uint32_t)d << shift);
             }
         }
-        mask |= 255u << shift;
+        mask |= ((1u << w) - 1u) << shift;
+        top = shift;
         __syncthreads();
     }
     const uint32_t thr = take_none ? 0xFFFFFFFFu : s_prefix;   // keys above thr are taken, equal keys in (head, block) order
     const int need_eq = take_none ? 0 : (int)s_need;
+    const int lane = tid & 31, warp = tid >> 5;
+    if (Hkv <= kMaxParts) {
+        // Ordered compaction without block-wide scans: every head's blocks are cut into parts (a multiple of 32 blocks,
+        // one warp each, in (head, block) order); pass A counts per part, one warp turns the counts into start
+        // positions, pass B writes.
+        const int wph = max(1, kGlobalWarps / Hkv);                         // parts per head
+        const int part_len = (((nb + wph - 1) / wph) + 31) & ~31;
+        const int n_parts = Hkv * wph;                                      // <= max(kGlobalWarps, kMaxParts)
+        for (int part = warp; part < n_parts; part += kGlobalWarps) {
+            const int h = part / wph, sub = part - h * wph;
+            const int b_end = min(nb, (sub + 1) * part_len);
+            int n_gt = 0, n_eq = 0;
+            for (int b = sub * part_len + lane; b - lane < b_end; b += 32) {
+                const uint32_t k = b < b_end ? keys[h * NBmax + b] : 0u;
+                n_gt += __popc(__ballot_sync(0xffffffffu, k == 0xFFFFFFFFu || (k > thr && k != 0u)));
+                n_eq += __popc(__ballot_sync(0xffffffffu, k == thr && k != 0xFFFFFFFFu && k != 0u));
+            }
+            if (lane == 0) part_gt[part] = n_gt, part_eq[part] = n_eq;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // serial over the parts in order (at most kMaxParts + kGlobalWarps of them), 32 at a time
+            int eq_before = 0, head_pos = 0, cur_head = 0;
+            for (int p0 = 0; p0 < n_parts; p0 += 32) {
+                const int part = p0 + lane;
+                const int g = part < n_parts ? part_gt[part] : 0, e = part < n_parts ? part_eq[part] : 0;
+                int e_inc = e;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, e_inc, o);
+                    if (lane >= o) e_inc += v;
+                }
+                const int my_eq_before = eq_before + e_inc - e;               // ties in earlier parts
+                const int take = g + max(0, min(e, need_eq - my_eq_before));  // blocks this part keeps
+                // start position inside the head: sum of `take` over the earlier parts of the same head
+                const int h = part < n_parts ? part / wph : -1;
+                int t_inc = take;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, t_inc, o);
+                    const int hv = __shfl_up_sync(0xffffffffu, h, o);
+                    if (lane >= o && hv == h) t_inc += v;   // parts of one head are contiguous: a segmented scan
+                }
+                int start = t_inc - take + (h == cur_head ? head_pos : 0);
+                if (part < n_parts) {
+                    part_eq[part] = my_eq_before;
+                    part_gt[part] = start;
+                    const bool last_of_head = part == n_parts - 1 || (part + 1) / wph != h;
+                    if (last_of_head) out_cnt[(size_t)s * Hkv + h] = min(start + take, max_sel);
+                }
+                // carry into the next 32 parts
+                eq_before += __shfl_sync(0xffffffffu, e_inc, 31);
+                const int last_h = __shfl_sync(0xffffffffu, h, 31), last_end = __shfl_sync(0xffffffffu, start + take, 31);
+                cur_head = last_h, head_pos = last_end;
+            }
+        }
+        __syncthreads();
+        for (int part = warp; part < n_parts; part += kGlobalWarps) {
+            const int h = part / wph, sub = part - h * wph;
+            const int b_end = min(nb, (sub + 1) * part_len);
+            int pos = part_gt[part], eq_rank = part_eq[part];
+            for (int b = sub * part_len + lane; b - lane < b_end; b += 32) {
+                const uint32_t k = b < b_end ? keys[h * NBmax + b] : 0u;
+                const bool eq = k == thr && k != 0xFFFFFFFFu && k != 0u;
+                const uint32_t eq_ball = __ballot_sync(0xffffffffu, eq);
+                const int my_rank = eq_rank + __popc(eq_ball & ((1u << lane) - 1u));
+                const bool take = k == 0xFFFFFFFFu || (k > thr && k != 0u) || (eq && my_rank < need_eq);
+                const uint32_t take_ball = __ballot_sync(0xffffffffu, take);
+                const int my_pos = pos + __popc(take_ball & ((1u << lane) - 1u));
+                if (take && my_pos < max_sel) out_idx[((size_t)s * Hkv + h) * max_sel + my_pos] = b;
+                pos += __popc(take_ball);
+                eq_rank += __popc(eq_ball);
+            }
+        }
+        return;
+    }
+    // more heads than the part tables hold: block-wide scans, head by head
     int eq_seen = 0;
     for (int h = 0; h < Hkv; ++h) {
         int taken = 0;

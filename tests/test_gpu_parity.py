@@ -987,9 +987,12 @@ def test_select_fuzz_exact_scores(sv):
 def test_select_global_fuzz_exact_scores(sv):
     """The shared-budget variant on the same hand-made score distributions, bit-exact including ties across heads."""
     g = np.random.default_rng(78)
-    S, Hkv, Hq, T, B = 2, 4, 4, 2, 64
-    for trial in range(18):
-        NB = int(g.choice([40, 200, 512, 1000]))
+    S, T, B = 2, 2, 64
+    for trial in range(24):
+        # head counts that give 16, 5, 4 and 1 warps per head in the ordered compaction, more parts than warps, and
+        # more heads than its part tables hold (block-wide scans instead)
+        Hkv = Hq = [4, 1, 3, 24, 4, 136][trial % 6]
+        NB = int(g.choice([40, 200, 512, 1000])) if Hkv <= 24 else int(g.choice([40, 200]))
         lens = np.array([NB * B - int(g.integers(0, B)), max(B, int(g.integers(NB // 2, NB)) * B - 7)], np.int32)
         n_sink, n_local = int(g.integers(0, 2)), int(g.integers(0, 3))
         budget = np.array([int(g.integers(n_sink + n_local, NB)), int(g.integers(n_sink + n_local, NB + 3))], np.int32)
