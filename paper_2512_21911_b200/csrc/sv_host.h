@@ -58,7 +58,11 @@ inline sv_status check_kv(const sv_geom *g, const sv_kv *kv, bool need_v)
 inline void pdl_attribute(cudaLaunchAttribute *attr)
 {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;
+#ifdef SV_TRACE
+    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;   // development builds only
+#else
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+#endif
 }
 
 // SMs of the current device (148 when there is no device to ask).

@@ -741,7 +741,12 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
     else
         e = launch_attn<4, 2, 2>(tk, tv, p, grid, cs);   // 8 warps: 4 x 32 rows x 2 key halves
     if (e != cudaSuccess) return SV_ERR_CUDA;
-    if (splits > 1 && !getenv("SV_PROBE_SKIP_MERGE")) {
+#ifdef SV_TRACE
+    const bool skip_merge = getenv("SV_PROBE_SKIP_MERGE") != nullptr;   // development builds only: time the attention kernel alone
+#else
+    const bool skip_merge = false;
+#endif
+    if (splits > 1 && !skip_merge) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((rows * 32 + kMergeThreads - 1) / kMergeThreads, geom->n_kv_heads, geom->n_seq);
         cfg.blockDim = dim3(kMergeThreads);

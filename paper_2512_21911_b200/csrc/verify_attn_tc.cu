@@ -811,7 +811,11 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;
+#ifdef SV_TRACE
+    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;   // development builds only
+#else
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+#endif
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide>, tm_k, tm_v, p);
