@@ -220,6 +220,7 @@ def run_gpu(args):
 
     eng = make_engine([True] * w.n_layers)
     eng_reuse = make_engine([l % 2 == 0 for l in range(w.n_layers)])   # anchors on even layers (Eq. 9)
+    eng_chain = make_engine([l == 0 for l in range(w.n_layers)])        # only layer 0 retrieves, every other layer reuses
     # all layers' pools in one allocation, so that the tail-block refresh of the stack is one launch
     k_all = torch.empty((w.n_layers,) + layers[0]["k_pool"].shape, dtype=torch.bfloat16, device=dev)
     v_all = torch.empty_like(k_all)
@@ -228,9 +229,11 @@ def run_gpu(args):
         v_all[l].copy_(bf16_dev(c["v_pool"]))
     eng.set_kv_stack(k_all, v_all)
     eng_reuse.set_kv_stack(k_all, v_all)
+    eng_chain.set_kv_stack(k_all, v_all)
     for l in range(w.n_layers):
         eng.build_reps(l)
     eng_reuse.reps = eng.reps
+    eng_chain.reps = eng.reps
     # per-step inputs: pinned host copies (end-to-end timing) and device-resident copies (kernel timing)
     q_h = torch.stack([torch.from_numpy(c["q"].view(np.int16)).view(torch.bfloat16) for c in layers]).pin_memory()
     dk_h = torch.stack([torch.from_numpy(c["draft_k"].view(np.int16)).view(torch.bfloat16) for c in layers]).pin_memory()
@@ -295,6 +298,7 @@ def run_gpu(args):
                               "kernels_per_step": eng.kernels_per_step(refresh_tail=True)}))
         return
     g_reuse = capture(lambda: eng_reuse.verify_step(q, dk, dv, out, refresh_tail=True))
+    g_chain = capture(lambda: eng_chain.verify_step(q, dk, dv, out, refresh_tail=True))
     g_attn = capture(lambda: [sv.sv_verify_attn(eng.geom, q[l], eng.kv[l], dk[l], dv[l], None, eng.sel_idx, eng.sel_cnt,
                                                 out[l], workspace=eng.workspace, status_word=eng.status)
                               for l in range(w.n_layers)])
@@ -307,6 +311,7 @@ def run_gpu(args):
     ms_step = time_replays(g_step, args.steps, max(args.warmup, 3), sampler=sampler)
     side = max(10, min(args.steps, 200))
     ms_reuse = time_replays(g_reuse, side, 3)
+    ms_chain = time_replays(g_chain, side, 3)
     ms_attn = time_replays(g_attn, side, 3)
     ms_dense = time_replays(g_dense, max(5, side // 4), 3)
     ms_reps = time_replays(g_reps, max(5, side // 4), 3)
@@ -361,7 +366,8 @@ def run_gpu(args):
         return e0.elapsed_time(e1) / steps
 
     ms_e2e = time_e2e(side, 4)
-    assert int(eng.status.item()) == 0 and int(eng_reuse.status.item()) == 0, "a kernel gave up on a bounded wait"
+    assert int(eng.status.item()) == 0 and int(eng_reuse.status.item()) == 0 and int(eng_chain.status.item()) == 0, \
+        "a kernel gave up on a bounded wait"
 
     def allmax(x):
         if world == 1:
@@ -370,8 +376,8 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e, ms_reps = (aggregate_over_ranks(x, world, allmax)[0]
-                                                             for x in (ms_step, ms_reuse, ms_attn, ms_dense, ms_e2e, ms_reps))
+    ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps = (
+        aggregate_over_ranks(x, world, allmax)[0] for x in (ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps))
 
     # algorithmic bytes of one sv_verify_attn launch (K+V of the kept tokens and draft tokens, Q in, O out)
     S, T, Hq, Hkv, D, B, N = w.n_seq, w.n_draft, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, w.budget_blocks
@@ -410,6 +416,8 @@ def run_gpu(args):
         "pct_of_8tbs": 100.0 * gathered / (us_attn * 1e-6) / 8e12,
         "tokens_verified_per_s": S * T * world / (ms_step * 1e-3),
         "reuse_even_anchors": {"us_per_layer": ms_reuse * 1e3 / w.n_layers, "kernels_per_step": eng_reuse.kernels_per_step(True)},
+        "reuse_previous_layer": {"us_per_layer": ms_chain * 1e3 / w.n_layers, "kernels_per_step": eng_chain.kernels_per_step(True),
+                                 "note": "only layer 0 retrieves; every later layer attends over the previous layer's blocks"},
         "dense_verify": {"us_per_layer": us_dense, "gbs": dense_bytes / (us_dense * 1e-6) / 1e9,
                          "frac": dense_bytes / (us_dense * 1e-6) / 1e9 / peak, "bytes_per_launch": dense_bytes},
         "block_reps_rebuild": {"us_per_layer": ms_reps * 1e3 / w.n_layers, "bytes_per_launch": reps_bytes,
