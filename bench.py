@@ -526,6 +526,119 @@ def run_sweep(args):
         del pools
 
 
+def run_configs(args):
+    """--configs: timing lines for the two other full-size configurations (their parity is covered by the tests):
+    the 16-sequence batch with ragged prefixes (block 64, 2048-token budget, 5 draft tokens as a chain) and the
+    4 x 131072-token long-context case (GQA 8, block 128, 4096-token budget, 16-node draft tree).  K/V are seeded
+    device-side N(0, 1/128) tensors, lengths / page tables / the tree come from seeded host generators, the block
+    lists from sv_select_blocks.  Each configuration rotates over independent KV replicas so that at least 256 MiB
+    is gathered between two uses of a replica (HBM, not L2).  One JSON line per configuration."""
+    import torch
+
+    import paper_2512_21911_b200 as sv
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peaks()
+    stream = torch.cuda.Stream(device=dev)
+    D = 128
+    cases = [("cfg2", dict(S=16, Hq=32, Hkv=8, B=64, lens=(4096, 16384), budget_tokens=2048, T=5, tree=False, seed=1002)),
+             ("cfg3", dict(S=4, Hq=64, Hkv=8, B=128, lens=(131072, 131072), budget_tokens=4096, T=16, tree=True, seed=1003))]
+    for name, c in cases:
+        S, Hq, Hkv, B, T = c["S"], c["Hq"], c["Hkv"], c["B"], c["T"]
+        rng = np.random.default_rng(c["seed"])
+        lens = rng.integers(c["lens"][0], c["lens"][1] + 1, size=S).astype(np.int32)
+        nb = (lens + B - 1) // B
+        NB = int(nb.max())
+        n_pages = int(nb.sum())
+        N = c["budget_tokens"] // B
+        perm = rng.permutation(n_pages).astype(np.int32)
+        bt_h = np.zeros((S, NB), np.int32)
+        o = 0
+        for s_ in range(S):
+            bt_h[s_, :nb[s_]] = perm[o:o + nb[s_]]
+            o += nb[s_]
+        parent_h = None
+        if c["tree"]:
+            parent_h = np.full((S, T), -1, np.int32)
+            for s_ in range(S):
+                for i in range(1, T):
+                    parent_h[s_, i] = rng.integers(0, i)
+        gathered = int(sum(min(N, int(x)) for x in nb)) * Hkv * B * D * 2 * 2
+        n_rep = max(2, -(-(256 << 20) // gathered))
+        gen = torch.Generator(device=dev).manual_seed(c["seed"])
+
+        def rnd(shape):
+            return torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).mul_(D ** -0.5).to(torch.bfloat16)
+
+        pools = [(rnd((n_pages, Hkv, B, D)), rnd((n_pages, Hkv, B, D))) for _ in range(n_rep)]
+        bt = torch.from_numpy(bt_h).to(dev)
+        sl = torch.from_numpy(lens).to(dev)
+        bud = torch.full((S,), N, dtype=torch.int32, device=dev)
+        parent = None if parent_h is None else torch.from_numpy(parent_h).to(dev)
+        geom = sv.make_geom(S, Hq, Hkv, D, B, NB, T)
+        q, dk, dv = rnd((S, T, Hq, D)), rnd((S, T, Hkv, D)), rnd((S, T, Hkv, D))
+        out = torch.zeros_like(q)
+        kvs = [sv.make_kv(k, v, bt, sl) for k, v in pools]
+        reps = [torch.zeros((S, Hkv, NB, D), device=dev) for _ in pools]
+        for kv, r in zip(kvs, reps):
+            sv.sv_block_reps(geom, kv, r)
+        idx = torch.zeros((S, Hkv, N), dtype=torch.int32, device=dev)
+        cnt = torch.zeros((S, Hkv), dtype=torch.int32, device=dev)
+        ws = torch.zeros(max(16, sv.sv_workspace_bytes(geom, NB)), dtype=torch.uint8, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        sv.sv_select_blocks(geom, q, reps[0], sl, bud, 1, 1, idx, cnt)
+
+        def sel_all():
+            for r in reps:
+                sv.sv_select_blocks(geom, q, r, sl, bud, 1, 1, idx, cnt)
+
+        def attn_all():
+            for kv in kvs:
+                sv.sv_verify_attn(geom, q, kv, dk, dv, parent, idx, cnt, out, workspace=ws, status_word=status)
+
+        def both_all():
+            for kv, r in zip(kvs, reps):
+                sv.sv_select_blocks(geom, q, r, sl, bud, 1, 1, idx, cnt)
+                sv.sv_verify_attn(geom, q, kv, dk, dv, parent, idx, cnt, out, workspace=ws, status_word=status)
+
+        def dense_all():
+            for kv in kvs:
+                sv.sv_verify_attn(geom, q, kv, dk, dv, parent, None, None, out, workspace=ws, status_word=status)
+
+        def timed(fn, iters):
+            with torch.cuda.stream(stream):
+                fn(); fn()
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                for _ in range(3):
+                    g.replay()
+                e0.record(stream)
+                for _ in range(iters):
+                    g.replay()
+                e1.record(stream)
+                stream.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / iters / len(kvs)
+
+        us_sel, us_attn, us_both = timed(sel_all, 20), timed(attn_all, 20), timed(both_all, 20)
+        us_dense = timed(dense_all, 5)
+        assert int(status.item()) == 0, "a kernel gave up on a bounded wait"
+        dense_bytes = int(nb.sum()) * Hkv * B * D * 2 * 2
+        print(json.dumps({"config": name, "n_seq": S, "q_heads": Hq, "kv_heads": Hkv, "block": B, "n_draft": T,
+                          "tree": bool(c["tree"]), "context_min": int(lens.min()), "context_max": int(lens.max()),
+                          "budget_blocks": N, "splits": sv.sv_verify_attn_splits(geom, N), "replicas": n_rep,
+                          "gathered_kv_mib": round(gathered / 2 ** 20, 1),
+                          "select_us": round(us_sel, 2), "attn_us": round(us_attn, 2), "select_plus_attn_us": round(us_both, 2),
+                          "kv_gbs": round(gathered / us_attn / 1e3, 1),
+                          "frac_of_measured_peak": round(gathered / us_attn / 1e3 / peak, 3),
+                          "dense_attn_us": round(us_dense, 2), "dense_kv_mib": round(dense_bytes / 2 ** 20, 1),
+                          "dense_frac_of_measured_peak": round(dense_bytes / us_dense / 1e3 / peak, 3),
+                          "speedup_vs_dense": round(us_dense / us_both, 2)}), flush=True)
+        del pools, kvs, reps
+
+
 def run_variants(args):
     """--variants: the retrieval variants the paper discusses, timed beside the adopted strategy on one layer of
     the benchmark workload (seeded host-generated inputs, as in the main line).  Every timed call is preceded
@@ -631,11 +744,15 @@ def main():
                     help="profiling aid: time only the main step graph (no reuse / dense / attention-only / e2e passes)")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line: sparse vs dense latency over context x budget x draft length")
+    ap.add_argument("--configs", action="store_true",
+                    help="timing lines for the batched (16 ragged sequences) and long-context (4 x 128K, tree) configurations")
     ap.add_argument("--variants", action="store_true",
                     help="instead of the benchmark line: timings of the retrieval variants (shared budget, every token)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+    elif args.configs:
+        run_configs(args)
     elif args.variants:
         run_variants(args)
     elif args.impl == "reference":

@@ -628,11 +628,19 @@ bool use_tensor_memory_path()
 }
 
 // Blocks per CTA are minimised subject to one CTA per SM; then the fewest splits that achieve it.
-int choose_splits(const sv_geom *g, int n_blocks)
+// With at least one (sequence, KV head, row tile) per SM nothing needs splitting for occupancy, but long lists are
+// still cut into pieces of about 64 units when `balance` is set: the sequences of a batch differ in length, one CTA
+// per pair makes the longest of them the launch time, and with several CTAs per SM-slot the block scheduler evens
+// that out (16 ragged sequences of 4.8-15K tokens, dense: 138 -> 90 us).
+int choose_splits(const sv_geom *g, int n_blocks, bool balance = true)
 {
     const int pairs = g->n_seq * g->n_kv_heads * (use_tensor_memory_path() ? svh::row_tiles(g) : 1);
     const int per_pair = sm_count() / pairs;
-    if (per_pair <= 1 || n_blocks <= 1) return 1;
+    if (n_blocks <= 1) return 1;
+    if (per_pair <= 1) {
+        const int units = n_blocks * (g->block_size / 64);
+        return (balance && use_tensor_memory_path() && units >= 128) ? (units + 63) / 64 : 1;
+    }
     const int blocks_per_cta = (n_blocks + per_pair - 1) / per_pair;
     return (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
 }
@@ -668,19 +676,28 @@ extern "C" int32_t sv_verify_attn_splits(const sv_geom *geom, int32_t max_sel)
     return choose_splits(geom, max_sel);
 }
 
-extern "C" size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel)
+namespace {
+
+size_t workspace_bytes_for(const sv_geom *geom, int32_t max_sel, bool balance)
 {
-    if (svh::check_geom(geom) != SV_OK || max_sel < 1) return 0;
-    const size_t splits = (size_t)choose_splits(geom, max_sel);
+    const size_t splits = (size_t)choose_splits(geom, max_sel, balance);
     const size_t rows = (size_t)(geom->n_q_heads / geom->n_kv_heads) * geom->n_draft;
     return (size_t)geom->n_seq * geom->n_kv_heads * splits * rows * (128 + 2) * sizeof(float) + 256;
 }
 
-extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
-                                    const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
-                                    const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out,
-                                    float *lse, void *workspace, size_t workspace_bytes, int32_t *status_word,
-                                    void *stream)
+}  // namespace
+
+extern "C" size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel)
+{
+    if (svh::check_geom(geom) != SV_OK || max_sel < 1) return 0;
+    return workspace_bytes_for(geom, max_sel, true);
+}
+
+// `balance`: see choose_splits (the built-in-scratch entry point gives it up when the partials would not fit)
+static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                                  const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                                  const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
+                                  void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream, bool balance)
 {
     sv_status st = svh::check_geom(geom);
     if (st != SV_OK) return st;
@@ -696,11 +713,11 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
 
     const int G = geom->n_q_heads / geom->n_kv_heads;
     const int rows = G * geom->n_draft;
-    const int splits = choose_splits(geom, max_sel);
+    const int splits = choose_splits(geom, max_sel, balance);
     if (splits > 1) {
         if (!workspace) return SV_ERR_NULL;
         if (!svh::aligned(workspace, 16)) return SV_ERR_ALIGN;
-        if (workspace_bytes < sv_workspace_bytes(geom, max_sel)) return SV_ERR_WORKSPACE;
+        if (workspace_bytes < workspace_bytes_for(geom, max_sel, balance)) return SV_ERR_WORKSPACE;
     }
 
     CUtensorMap tk, tv;
@@ -765,6 +782,16 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
     return SV_OK;
 }
 
+extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                                    const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                                    const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out,
+                                    float *lse, void *workspace, size_t workspace_bytes, int32_t *status_word,
+                                    void *stream)
+{
+    return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
+                            workspace, workspace_bytes, status_word, stream, true);
+}
+
 // ---------------------------------------------------------------------- sv_verify_attn_noalloc
 //
 // Built-in scratch for callers that cannot allocate (see sv.h).  The array below is device memory that
@@ -807,9 +834,11 @@ extern "C" sv_status sv_verify_attn_noalloc(const sv_geom *geom, const void *q, 
     if (st != SV_OK) return st;
     const int32_t eff_sel = sel_idx ? max_sel : geom->max_blocks;
     if (eff_sel < 1) return SV_ERR_SHAPE;
-    if (sv_workspace_bytes(geom, eff_sel) > (size_t)SV_NOALLOC_SCRATCH_BYTES) return SV_ERR_SCRATCH_LIMIT;
+    // a batch that is only split to even out ragged lengths runs unsplit when those partials would not fit
+    const bool balance = workspace_bytes_for(geom, eff_sel, true) <= (size_t)SV_NOALLOC_SCRATCH_BYTES;
+    if (workspace_bytes_for(geom, eff_sel, balance) > (size_t)SV_NOALLOC_SCRATCH_BYTES) return SV_ERR_SCRATCH_LIMIT;
     void *scratch = noalloc_scratch_address();
     if (!scratch) return SV_ERR_CUDA;
-    return sv_verify_attn(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
-                          scratch, (size_t)SV_NOALLOC_SCRATCH_BYTES, status_word, stream);
+    return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
+                            scratch, (size_t)SV_NOALLOC_SCRATCH_BYTES, status_word, stream, balance);
 }

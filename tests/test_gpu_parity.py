@@ -361,6 +361,21 @@ def test_full_size_cfg2(sv):
     run_pipeline(sv, c, what="cfg2")
 
 
+def test_full_size_cfg2_dense_sampled(sv):
+    """Dense verification of the ragged 16-sequence batch: more (sequence, KV head) pairs than an SM each needs, lists
+    long enough that every pair is still cut into several CTAs to even out the lengths."""
+    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg2"]), sharp=True)
+    d = Dev(sv, c)
+    assert sv.sv_verify_attn_splits(d.geom, c["max_blocks"]) > 1
+    o, lse = gpu_attn(sv, d, None, None)
+    longest, shortest = int(np.argmax(c["seq_lens"])), int(np.argmin(c["seq_lens"]))
+    smp = [(longest, 4, 31), (longest, 0, 0), (shortest, 2, 13), (7, 3, 20), (15, 1, 5)]
+    o_ref, lse_ref = oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                              c["draft_k"], c["draft_v"], None, samples=smp)
+    check_attn(np.stack([o[s, i, h] for s, i, h in smp]), np.array([lse[s, i, h] for s, i, h in smp]), o_ref, lse_ref,
+               "cfg2 dense")
+
+
 def test_full_size_cfg3_sampled(sv):
     c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg3"]), sharp=True)
     _sampled_check(sv, c, 64, "cfg3")
