@@ -90,3 +90,31 @@ def test_noalloc_rejects_problems_beyond_the_built_in_scratch():
     assert e.value.status == 8 and "scratch" in str(e.value)
     torch.cuda.synchronize()
     assert (out == 3.0).all()
+
+
+def test_noalloc_runs_unsplit_where_only_the_balancing_split_would_not_fit():
+    """Dense verification of the ragged 16-sequence batch: the ordinary entry point cuts every (sequence, KV head) list
+    into several CTAs to even out the lengths, which needs more partials than the built-in scratch holds; every SM has
+    a pair anyway, so the no-alloc call runs the same problem without that split instead of refusing it."""
+    import paper_2512_21911_b200 as sv
+    w = si.WORKLOADS["cfg2"]
+    c, geom, t, kv, _, _ = _case(sv, w, True, layer=0)
+    nb = c["max_blocks"]
+    assert sv.sv_verify_attn_splits(geom, nb) > 1 and sv.sv_workspace_bytes(geom, nb) > sv.SV_NOALLOC_SCRATCH_BYTES
+    shape = (w.n_seq, w.n_draft, w.n_q_heads)
+    out_ref = torch.zeros(shape + (w.head_dim,), dtype=torch.bfloat16, device="cuda")
+    lse_ref = torch.zeros(shape, device="cuda")
+    ws = torch.empty(sv.sv_workspace_bytes(geom, nb), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sv.sv_verify_attn(geom, t["q"], kv, t["dk"], t["dv"], t["parent"], None, None, out_ref, lse=lse_ref, workspace=ws,
+                      status_word=status)
+    out = torch.full_like(out_ref, float("nan"))
+    lse = torch.full_like(lse_ref, float("nan"))
+    sv.sv_verify_attn_noalloc(geom, t["q"], kv, t["dk"], t["dv"], t["parent"], None, None, out, lse=lse, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o, o_ref = _host(out), _host(out_ref)
+    assert np.isfinite(o).all()
+    scale = max(1.0, float(np.abs(o_ref).max()))
+    assert np.abs(o - o_ref).max() <= 1e-2 * scale and np.abs(o - o_ref).mean() <= 1e-3 * scale
+    assert np.abs(lse.cpu().numpy() - lse_ref.cpu().numpy()).max() <= 1e-3
