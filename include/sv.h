@@ -213,7 +213,10 @@ SV_API sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv 
  * Same arguments and results as sv_verify_attn, minus workspace / workspace_bytes.  The call allocates
  * nothing on the device or through any allocating library routine.  Differences:
  *   - sizes: if sv_workspace_bytes(geom, max_sel) exceeds SV_NOALLOC_SCRATCH_BYTES the call launches
- *     nothing and returns SV_ERR_SCRATCH_LIMIT (use sv_verify_attn with your own workspace instead);
+ *     nothing and returns SV_ERR_SCRATCH_LIMIT (use sv_verify_attn with your own workspace instead).
+ *     One exception: a batch with at least one (sequence, KV head) pair per SM, whose long lists
+ *     sv_verify_attn cuts into several CTAs only to even out ragged sequence lengths, runs without that
+ *     cut (same results, no partials) when the partials of the cut would not fit;
  *   - set-up: the first call on each device looks up the device address of the built-in array (with
  *     that device current) and keeps it; make that first call outside any stream capture;
  *   - sharing: all calls on a device use the same array, and it keeps whatever the last call left in
