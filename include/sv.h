@@ -58,11 +58,32 @@ typedef enum {
     SV_ERR_WORKSPACE = 5,   /* workspace_bytes is smaller than sv_workspace_bytes() */
     SV_ERR_UNSUPPORTED = 6, /* head_dim != 128, block_size not 64/128, more than 64 draft tokens, more than 8 row tiles ... */
     SV_ERR_CUDA = 7,        /* a CUDA call or kernel launch failed */
-    SV_ERR_SCRATCH_LIMIT = 8 /* sv_verify_attn_noalloc: the problem needs more scratch than the built-in buffer holds */
+    SV_ERR_SCRATCH_LIMIT = 8, /* sv_verify_attn_noalloc: the problem needs more scratch than the built-in buffer holds */
+    SV_ERR_INDEX = 9        /* a device-side check found a block index, page id or list count outside its table
+                               (reported through a status word, see sv_status_word_check) */
 } sv_status;
 
 /* Static, human-readable text for a status code. */
 SV_API const char *sv_strerror(sv_status st);
+
+/*
+ * Device status word (the optional `status_word` argument of the attention entry points): a dev int32
+ * the caller zeroes once and reads back whenever it synchronises anyway.  Kernels OR bits into it and
+ * never clear it.  A non-zero word means the outputs written since it was last zero are invalid.
+ *   SV_STATUS_WAIT_MASK   a kernel gave up on one of its bounded waits (a copy or a tensor-core operation
+ *                         that never completed); the CTA drained and returned
+ *   SV_STATUS_INDEX       a block index in sel_idx or a page id in block_table lay outside its table; it was
+ *                         clamped into the table before any address was formed, so nothing out of range
+ *                         was read
+ *   SV_STATUS_NO_LIST     a count in sel_cnt was negative: sv_select_blocks writes -1 there when it had to
+ *                         give up on a list; the attention then covered the draft tokens only
+ * sv_status_word_check maps a word read back by the caller to a status: SV_OK, SV_ERR_INDEX
+ * (SV_STATUS_INDEX or SV_STATUS_NO_LIST set) or SV_ERR_CUDA (a wait gave up).  Host arithmetic only.
+ */
+#define SV_STATUS_WAIT_MASK 0x0FF
+#define SV_STATUS_INDEX 0x100
+#define SV_STATUS_NO_LIST 0x200
+SV_API sv_status sv_status_word_check(int32_t status_word_value);
 
 /* Geometry shared by all calls. */
 typedef struct {
@@ -103,6 +124,8 @@ SV_API int32_t sv_budget_blocks(int64_t L_seq, int64_t L0, double rho, int32_t b
  * Bytes of scratch that sv_verify_attn needs for this geometry when at most
  * max_sel blocks are kept per (sequence, KV head) (pass max_blocks for dense
  * attention).  Holds the per-split partial results of the split-KV kernel.
+ * 0 when the call needs none (one CTA per (sequence, KV head) writes the output
+ * itself; workspace may then be NULL) -- and for an invalid geometry.
  */
 SV_API size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel);
 
@@ -126,8 +149,9 @@ SV_API sv_status sv_block_reps(const sv_geom *geom, const sv_kv *kv, int32_t blo
  * accept_idx[s][0 .. n_accept[s]) are appended, in that order, at positions L_s, L_s + 1, ... of the paged
  * cache, seq_lens_out[s] = L_s + n_accept[s], and the representatives of the (at most two) blocks that
  * received tokens are recomputed exactly as sv_block_reps would.  The pages of blocks that are entered
- * must already be listed in block_table; tokens that would fall behind the last page of the table are
- * dropped (n_accept is clamped).  Replaces "append + sv_block_reps(SV_TAIL_BLOCK)" in a decoding loop.
+ * must already be listed in block_table; tokens that would fall behind the last page of the table, or into
+ * a block whose table entry is not a page of the pool (outside [0, n_pages): not assigned yet), are dropped
+ * (n_accept is clamped; nothing outside the pools is written).  Replaces "append + sv_block_reps(SV_TAIL_BLOCK)" in a decoding loop.
  *   k_pool/v_pool   dev bf16 [n_pages][Hkv][B][D], modified in place
  *   seq_lens        dev int32 [S] lengths before the commit; seq_lens_out dev int32 [S], a different buffer
  *   draft_k/draft_v dev bf16 [S][T][Hkv][D] of the step just verified
@@ -159,7 +183,9 @@ SV_API sv_status sv_kv_append(const sv_geom *geom, void *k_pool, void *v_pool, i
  *   seq_lens      dev int32 [S]
  *   budget_blocks dev int32 [S]: N, blocks to keep per KV head
  *   out_idx       dev int32 [S][Hkv][max_sel]: kept block indices, ascending; entries >= cnt untouched
- *   out_cnt       dev int32 [S][Hkv]
+ *   out_cnt       dev int32 [S][Hkv]; -1 marks a list the kernel could not produce (its bounded wait for the
+ *                 scores gave up): sv_verify_attn then attends over the draft tokens only and sets
+ *                 SV_STATUS_NO_LIST in its status word
  *   out_scores    dev fp32 [S][Hkv][NBmax] or NULL (diagnostic copy of the scores)
  * NBmax <= 32768.
  */
@@ -190,8 +216,9 @@ SV_API sv_status sv_select_blocks(const sv_geom *geom, const void *q, const floa
  *   workspace       dev scratch of at least sv_workspace_bytes(geom, max_sel)
  *                   bytes, 16-byte aligned; contents are overwritten.  Calls
  *                   that may overlap on the GPU need distinct workspaces.
- *   status_word     dev int32 or NULL: set non-zero if a kernel gave up on a
- *                   bounded wait (the output is then invalid)
+ *   status_word     dev int32 or NULL: bits are set if a kernel gave up on a bounded
+ *                   wait or had to clamp an index (see "Device status word" above;
+ *                   the output is then invalid)
  */
 SV_API sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
                          const void *draft_v, const int32_t *parent, const int32_t *sel_idx,

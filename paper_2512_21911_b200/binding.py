@@ -18,10 +18,13 @@ LIB_PATH = os.path.join(_HERE, "libsv.so")
 SV_OK = 0
 SV_TAIL_BLOCK = -1   # sv_block_reps(block_begin=SV_TAIL_BLOCK): refresh only each sequence's last block
 STATUS_NAMES = {0: "SV_OK", 1: "SV_ERR_NULL", 2: "SV_ERR_SHAPE", 3: "SV_ERR_ALIGN", 4: "SV_ERR_BUDGET",
-                5: "SV_ERR_WORKSPACE", 6: "SV_ERR_UNSUPPORTED", 7: "SV_ERR_CUDA", 8: "SV_ERR_SCRATCH_LIMIT"}
+                5: "SV_ERR_WORKSPACE", 6: "SV_ERR_UNSUPPORTED", 7: "SV_ERR_CUDA", 8: "SV_ERR_SCRATCH_LIMIT",
+                9: "SV_ERR_INDEX"}
+# bits of the device status word (see sv.h)
+SV_STATUS_WAIT_MASK, SV_STATUS_INDEX, SV_STATUS_NO_LIST = 0x0FF, 0x100, 0x200
 SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
-EXPORTS = ("sv_strerror", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
+EXPORTS = ("sv_strerror", "sv_status_word_check", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
            "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
            "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global", "sv_accept",
            "sv_block_reps_bf16", "sv_select_blocks_bf16reps")
@@ -54,6 +57,8 @@ def _load() -> ctypes.CDLL:
     gp, kp = ctypes.POINTER(sv_geom), ctypes.POINTER(sv_kv)
     lib.sv_strerror.restype = ctypes.c_char_p
     lib.sv_strerror.argtypes = [ctypes.c_int]
+    lib.sv_status_word_check.restype = ctypes.c_int
+    lib.sv_status_word_check.argtypes = [i32]
     lib.sv_budget_blocks.restype = i32
     lib.sv_budget_blocks.argtypes = [i64, i64, f64, i32, i32, i32]
     lib.sv_workspace_bytes.restype = sz
@@ -124,6 +129,11 @@ def make_kv(k_pool: torch.Tensor, v_pool: Optional[torch.Tensor], block_table: t
     return sv_kv(_ptr(k_pool, torch.bfloat16, "k_pool"), _ptr(v_pool, torch.bfloat16, "v_pool"),
                  _ptr(block_table, torch.int32, "block_table"), _ptr(seq_lens, torch.int32, "seq_lens"),
                  int(k_pool.shape[0]))
+
+
+def sv_status_word_check(value: int) -> int:
+    """Status code for a device status word the caller has read back (0 = SV_OK)."""
+    return int(_lib.sv_status_word_check(int(value)))
 
 
 def sv_budget_blocks(L_seq: int, L0: int, rho: float, block_size: int, n_sink: int = 0, n_local: int = 0) -> int:

@@ -1,11 +1,17 @@
-// Shared between the two attention kernels (mma.sync path and tcgen05 path): launch parameters.
+// Launch parameters of the attention kernel and the split merge, shared by the two files that hold them.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "sv.h"
+
 namespace svk {
+
+// Bits of the optional device status word (the values documented in sv.h).
+constexpr int kStatusIndex = SV_STATUS_INDEX;   // a block index or page id outside its table was clamped
+constexpr int kStatusNoList = SV_STATUS_NO_LIST;  // a selection count was negative (block selection gave up on that list)
 
 struct AttnParams {
     const __nv_bfloat16 *q;
@@ -23,7 +29,8 @@ struct AttnParams {
     int32_t *status;
     int T, Hq, Hkv, G, B, NBmax, max_sel, splits;
     float scale_log2;
-    int Tt, tiles;   // tcgen05 kernel: draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
+    int Tt, tiles;   // draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
+    int n_pages;     // pages in each pool: page ids from the block table are clamped to it
 };
 
 // tcgen05 / TMEM attention kernel (verify_attn_tc.cu): rows = G*T <= 128 packed as one M=128 tile.

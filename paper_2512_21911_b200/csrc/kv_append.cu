@@ -6,7 +6,8 @@
 // One CTA per (KV head, sequence).  At most 64 tokens are appended per sequence, so at most two blocks are
 // touched: the rows are copied with 128-bit loads/stores (K and V), then the one or two affected block
 // means are recomputed from the pool exactly as sv_block_reps does (fp32 sums in a fixed order), which keeps
-// them bit-identical to a full rebuild.  Traffic: n*512 bytes copied + at most 2*B*256 bytes re-read per
+// them bit-identical to a full rebuild.  Page ids are checked against the pool size before anything is
+// written: a table entry that is not a page of the pool ends the table (the rows are dropped).  Traffic: n*512 bytes copied + at most 2*B*256 bytes re-read per
 // (sequence, KV head): latency-bound, not bandwidth-bound.
 #include <cuda_bf16.h>
 
@@ -27,14 +28,20 @@ __global__ void __launch_bounds__(kThreads) kv_append_kernel(uint4 *__restrict__
                                                              const int32_t *__restrict__ accept_idx,
                                                              const int32_t *__restrict__ n_accept, int max_accept,
                                                              int32_t *__restrict__ seq_lens_out, float *__restrict__ reps,
-                                                             int T, int Hkv, int NBmax)
+                                                             int T, int Hkv, int NBmax, int n_pages)
 {
     const int h = blockIdx.x, s = blockIdx.y;
     svk::grid_dependency_wait();
     svk::grid_launch_dependents();
     const int L = seq_lens[s];
     int n = min(max(n_accept[s], 0), max_accept);
-    n = min(n, NBmax * B - L);                       // never past the last page of the table
+    n = L < 0 ? 0 : max(0, min(n, NBmax * B - L));   // never past the last page of the table (nothing if L is already there)
+    // A block whose table entry is not a page of the pool (not assigned yet: -1, or stale) ends the table: no row
+    // enters it.  n <= 64 <= B, so the rows touch at most the blocks L / B and L / B + 1.
+    for (int b = L / B; n > 0 && b <= (L + n - 1) / B; ++b) {
+        const int page = block_table[(size_t)s * NBmax + b];
+        if (page < 0 || page >= n_pages) n = max(0, min(n, b * B - L));
+    }
     const int Ln = L + n;
     if (h == 0 && threadIdx.x == 0) seq_lens_out[s] = Ln;
     if (n <= 0) return;
@@ -122,9 +129,9 @@ extern "C" sv_status sv_kv_append(const sv_geom *geom, void *k_pool, void *v_poo
         geom->block_size == 64
             ? cudaLaunchKernelEx(&cfg, kv_append_kernel<64>, kp, vp, block_table, seq_lens, dk, dv, accept_idx, n_accept,
                                  (int)max_accept, seq_lens_out, reps, (int)geom->n_draft, (int)geom->n_kv_heads,
-                                 (int)geom->max_blocks)
+                                 (int)geom->max_blocks, (int)n_pages)
             : cudaLaunchKernelEx(&cfg, kv_append_kernel<128>, kp, vp, block_table, seq_lens, dk, dv, accept_idx, n_accept,
                                  (int)max_accept, seq_lens_out, reps, (int)geom->n_draft, (int)geom->n_kv_heads,
-                                 (int)geom->max_blocks);
+                                 (int)geom->max_blocks, (int)n_pages);
     return e == cudaSuccess ? svh::launch_status() : SV_ERR_CUDA;
 }

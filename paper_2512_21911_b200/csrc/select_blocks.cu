@@ -2,13 +2,17 @@
 // first draft token's query, then the top-N blocks with the first/last few kept (Section 3.1), in one
 // launch.  reuse_prev copies the previous layer's set (Section 3.3, Eq. 9).
 //
-// One thread-block cluster per (sequence, KV head).  Each CTA of the cluster scores a contiguous
-// slice of the blocks (a GEMV over fp32 representatives: one warp per block row, 128-bit loads,
-// several rows in flight per warp) into its own shared memory as order-preserving 32-bit keys.  After a
-// cluster barrier CTA 0 pulls the slices through distributed shared memory and runs an exact
-// radix select (4 passes of 8 bits) for the N-th largest key, then compacts the kept block indices in
-// ascending order with a block-wide scan; equal keys are taken smallest index first.  No global
-// scratch, no spin-waits (hardware cluster barriers only).
+// One thread-block cluster (up to 8 CTAs) per (sequence, KV head).  Each CTA of the cluster scores a
+// contiguous slice of the blocks (a GEMV over the representatives: one warp per block row, 128-bit loads,
+// several rows in flight per warp), turns the scores into order-preserving 32-bit keys and pushes them
+// straight into CTA 0's shared memory with st.async stores that count their bytes on an mbarrier there;
+// the senders then exit.  CTA 0 waits (bounded) for the expected byte count and selects exactly: the
+// scores are mapped linearly onto 16-bit codes, a 256-bin histogram of the upper byte (and, for a crowded
+// bin, of the lower byte) finds the boundary, the few keys left at the boundary are ranked by their exact
+// keys (ties: smaller block index), and an ascending ballot compaction writes the list.  More than 2048
+// blocks, equal scores everywhere or a still crowded boundary take the general radix select on the key
+// bits (8-bit digits from the highest differing bit).  No global scratch.  If the bounded wait for the
+// keys ever gives up, the count of that (sequence, KV head) is written as -1 (see sv.h).
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
@@ -18,26 +22,6 @@
 #include "sv_ptx.cuh"
 
 namespace cg = cooperative_groups;
-
-#ifdef SV_TRACE
-// Development aid (never compiled into the library): cycle stamps of cluster 0.
-__device__ long long g_sv_trace_sel[8 * 32];
-extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_sel()
-{
-    long long *p = nullptr;
-    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace_sel);
-    return p;
-}
-#define SEL_STAMP(slot)                                                                              \
-    do {                                                                                             \
-        if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 8)                \
-            g_sv_trace_sel[blockIdx.x * 32 + (slot)] = clock64();                                    \
-    } while (0)
-#else
-#define SEL_STAMP(slot) \
-    do {                \
-    } while (0)
-#endif
 
 namespace {
 
@@ -128,7 +112,6 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     __shared__ uint32_t key_min, key_max;          // smallest / largest evictable key (fast path)
     __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: the bytes of all keys (one arrival: CTA 0 itself)
 
-    SEL_STAMP(0);
     // While the kernel that precedes this one in the stream drains: pull this warp's first batch of
     // representative rows and the query row towards L2 (a prefetch consumes no data, so it is safe even if
     // that kernel is still writing them), set up the barrier, zero the histograms.
@@ -138,9 +121,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         svk::mbar_fence_init();
     }
     for (int i = tid; i < 4 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
-    SEL_STAMP(10);
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // before any global request is in flight
-    SEL_STAMP(11);
     const int b0 = rank * p.chunk;
     constexpr int kRowBytes = kBf16 ? 256 : 512, kLaneBytes = kRowBytes / 32;
     const char *rbase = static_cast<const char *>(p.reps) + ((size_t)s * p.Hkv + h) * p.NBmax * kRowBytes;
@@ -162,10 +143,8 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     const int G = p.Hq / p.Hkv;
     const __nv_bfloat16 *q0 = p.q + ((size_t)s * p.T * p.Hq + (size_t)h * G) * 128;
     if (tid < G * 2) svk::prefetch_l2(q0 + tid * 64);
-    SEL_STAMP(1);
     svk::grid_dependency_wait();
     svk::grid_launch_dependents();
-    SEL_STAMP(2);
 
     // every load below is issued before the first use
     const int L = p.seq_lens[s];
@@ -195,8 +174,6 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     // retrieval query: mean of the first draft token's query over the GQA group
     if (tid < 128) qbar[tid] = qsum / (float)G;
     __syncthreads();
-    SEL_STAMP(3);
-    SEL_STAMP(12);
 
     const uint32_t keys0 = cluster_map_shared(svk::smem_u32(keys_all), 0);
     const uint32_t ready0 = cluster_map_shared(svk::smem_u32(&keys_ready), 0);
@@ -225,9 +202,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
             if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter, b1);
         }
     }
-    SEL_STAMP(13);
     if (rank != 0) return;
-    SEL_STAMP(4);
 
     int32_t *out = p.out_idx + ((size_t)s * p.Hkv + h) * p.max_sel;
     if (keep_all) {
@@ -235,8 +210,11 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = nb;
         return;
     }
-    if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) return;   // gave up: leave the output untouched
-    SEL_STAMP(5);
+    if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) {
+        // gave up: mark the list invalid (sv_verify_attn then attends over the draft tokens only and reports it)
+        if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = -1;
+        return;
+    }
 
     // ---- fast path (up to 2048 blocks = 4 keys per thread, scores not all equal) -----------------------------------
     // The scores of one (sequence, KV head) are mapped linearly onto 0..65535 (monotone in the score, so the
@@ -347,7 +325,6 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                         }
                     }
                 }
-                SEL_STAMP(7);
                 // ascending compaction
                 uint32_t base = 0;
 #pragma unroll
@@ -369,7 +346,6 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                     }
                 }
                 if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
-                SEL_STAMP(8);
                 return true;
             }
             // fall through: the fast path used hist[0] and hist[1]; clear them for the radix passes
@@ -460,12 +436,10 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         mask |= dmask << shift;
         remaining = rem_in_bin;
         lo = shift;
-        SEL_STAMP(14 + pass);
         if (remaining == bin_count) break;   // the whole boundary bin is kept: lower bits cannot matter
     }
     // evictable keys whose decided bits exceed the prefix are kept; of those equal to it, the first `remaining`
     // in index order (all of them after an early stop, none when only the forced blocks fit the budget)
-    SEL_STAMP(7);
     const uint32_t thr = prefix;
     const uint32_t take_eq = remaining;
 
@@ -504,7 +478,6 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         __syncthreads();
     }
     if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
-    SEL_STAMP(8);
 }
 
 __global__ void copy_selection_kernel(const int32_t *__restrict__ prev_idx, const int32_t *__restrict__ prev_cnt,

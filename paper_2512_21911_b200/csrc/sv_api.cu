@@ -15,8 +15,16 @@ extern "C" const char *sv_strerror(sv_status st)
         case SV_ERR_UNSUPPORTED: return "unsupported geometry";
         case SV_ERR_CUDA: return "CUDA call or kernel launch failed";
         case SV_ERR_SCRATCH_LIMIT: return "the problem needs more scratch than the built-in buffer of sv_verify_attn_noalloc holds";
+        case SV_ERR_INDEX: return "a block index, page id or list count was outside its table (device status word)";
     }
     return "unknown status";
+}
+
+extern "C" sv_status sv_status_word_check(int32_t v)
+{
+    if (v & SV_STATUS_WAIT_MASK) return SV_ERR_CUDA;
+    if (v & (SV_STATUS_INDEX | SV_STATUS_NO_LIST)) return SV_ERR_INDEX;
+    return v ? SV_ERR_CUDA : SV_OK;
 }
 
 extern "C" int32_t sv_budget_blocks(int64_t L_seq, int64_t L0, double rho, int32_t block_size, int32_t n_sink,

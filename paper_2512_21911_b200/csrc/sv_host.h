@@ -2,7 +2,8 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdlib.h>
+
+#include <atomic>
 
 #include "sv.h"
 
@@ -58,26 +59,53 @@ inline sv_status check_kv(const sv_geom *g, const sv_kv *kv, bool need_v)
 inline void pdl_attribute(cudaLaunchAttribute *attr)
 {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-#ifdef SV_TRACE
-    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;   // development builds only
-#else
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-#endif
 }
+
+// Per-device state.  One process may drive several GPUs, and function attributes and SM counts belong to
+// a device, so both are kept per device index (devices beyond the table are handled uncached).
+constexpr int kMaxDevices = 64;
+
+inline int current_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        dev = 0;
+    }
+    return dev;
+}
+
+// Runs `configure` (a callable returning cudaError_t, e.g. a cudaFuncSetAttribute call) once per device
+// for the call site that owns this object.
+struct OncePerDevice {
+    std::atomic<uint64_t> done{0};
+    template <class F>
+    cudaError_t run(F configure)
+    {
+        const int dev = current_device();
+        const bool cached = dev >= 0 && dev < kMaxDevices;
+        if (cached && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return cudaSuccess;
+        const cudaError_t e = configure();
+        if (e == cudaSuccess && cached) done.fetch_or(1ull << dev, std::memory_order_release);
+        return e;
+    }
+};
 
 // SMs of the current device (148 when there is no device to ask).
 inline int sm_count()
 {
-    static const int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
-            cudaGetLastError();
-            v = 148;
-        }
-        return v;
-    }();
-    return n;
+    static std::atomic<int> count[kMaxDevices];
+    const int dev = current_device();
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    int v = cached ? count[dev].load(std::memory_order_relaxed) : 0;
+    if (v > 0) return v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+        cudaGetLastError();
+        return 148;
+    }
+    if (cached) count[dev].store(v, std::memory_order_relaxed);
+    return v;
 }
 
 inline sv_status launch_status()

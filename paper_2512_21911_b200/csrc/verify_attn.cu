@@ -1,502 +1,32 @@
 // sv_verify_attn: attention of all draft tokens of a sequence over the kept KV blocks plus the draft
-// tokens' own K/V (Fig. 1), split-KV with a log-sum-exp merge.
+// tokens' own K/V (Fig. 1), split-KV with a log-sum-exp merge.  This file holds the host side of the
+// entry points (argument checks, tensor maps over the paged pools, the split rule, the launches) and the
+// merge kernel; the attention kernel itself (tcgen05 tensor cores, TMEM accumulators, TMA gather) is in
+// verify_attn_tc.cu.
 //
-// Grid (split, KV head, sequence).  A CTA owns a contiguous slice of the ascending block list of its
-// (sequence, KV head) and the G*T query rows of that KV head (GQA group x draft tokens packed as the
-// M dimension of the tensor-core tiles).  One producer warp walks the block list and gathers 64-token
-// K and V tiles from the paged pools with TMA (2-D tiled loads, 128-byte swizzle, completion on
-// mbarriers, L2 evict-first) into a ring of 32 KB stages (it belongs to a warpgroup that gives its
-// registers to the others with setmaxnreg); eight consumer warps take stages in turn
-// (warp groups of WM warps, each warp MT 16-row tiles), compute S = QK^T and O += PV with bf16
-// mma.sync, fp32 online softmax, and are merged across warp groups in shared memory at the end.  With
-// one split the CTA writes bf16 output directly; otherwise fp32 partials (m, l, o) go to the workspace
-// and a small merge kernel combines them.  The kernel is bound by HBM bandwidth (512 bytes of K/V per
-// cached token and KV head); tensor cores only keep the arithmetic (4*rows*128 flop per token) off
-// the critical path.
+// Grid (split [x row tile], KV head, sequence).  A CTA owns a contiguous slice of the ascending block list
+// of its (sequence, KV head) and the G*T query rows of that KV head (GQA group x draft tokens packed as the
+// M dimension of the tensor-core tiles).  With one split the CTA writes bf16 output directly; otherwise
+// fp32 partials (m, l, o) go to the workspace and the merge kernel below combines them.  The path is bound
+// by HBM bandwidth (512 bytes of K/V per cached token and KV head).
 //
-// The partially filled last block is loaded whole (the page exists) and masked: its key columns
-// beyond the sequence length get -inf and its value rows are zeroed in shared memory.  The draft
-// tokens' K/V (at most 32 rows) are staged by the CTA of the last split with ordinary loads and
-// masked with per-row ancestor bit masks (tree) or j <= i (chain).
-//
-// All waits are bounded: a wait that gives up sets *status_word and the CTA drains without hanging.
+// All device-side waits are bounded: a wait that gives up sets *status_word and the CTA drains without
+// hanging.  Block indices and page ids are clamped into their tables before any address is formed; a
+// clamp that fires also sets a bit of *status_word.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include <cstdlib>
 #include <mutex>
 
 #include "attn_common.cuh"
 #include "sv_host.h"
 #include "sv_ptx.cuh"
 
-#ifdef SV_TRACE
-// Development aid (never compiled into the library): per-CTA cycle stamps of the attention kernel.
-__device__ long long g_sv_trace[256 * 16];
-extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer()
-{
-    long long *p = nullptr;
-    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace);
-    return p;
-}
-#define SV_STAMP(slot)                                                                      \
-    do {                                                                                    \
-        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);    \
-        if (cta_ < 256) g_sv_trace[cta_ * 16 + (slot)] = clock64();                         \
-    } while (0)
-#else
-#define SV_STAMP(slot) \
-    do {               \
-    } while (0)
-#endif
-
 namespace {
 
 using namespace svk;
 
-constexpr int kMathWarps = 8;                      // warps 0..7: two warpgroups that get the registers
-constexpr int kMathThreads = kMathWarps * 32;
-constexpr int kThreads = kMathThreads + 128;       // + one producer warpgroup (one warp of it works)
-constexpr int kUnit = 64;                          // keys per pipeline stage
-constexpr int kStageBytes = 4 * kUnit * 128;       // K lo/hi + V lo/hi halves, 8 KB each
-constexpr int kDraftRows = 32;
-constexpr int kDraftBytes = 4 * kDraftRows * 128;
-constexpr int kSmemLimit = 232448;                 // 227 KB per CTA
-constexpr int kMiscBytes = 1024;
-
-
-// Warp layout: WM x KS consumer warps.  Warp (wm, ks) owns MT 16-row tiles of the query rows and the
-// keys [ks*64/KS, (ks+1)*64/KS) of every 64-key stage, so all warps work on a stage as soon as it lands
-// and every warp consumes every stage in order.
-template <int WM, int MT, int KS>
-struct Cfg {
-    static constexpr int kRowsPad = WM * MT * 16;
-    static constexpr int kKeysPerWarp = kUnit / KS;
-    static constexpr int kConsumerWarps = WM * KS;
-    static constexpr int kConsumerThreads = kConsumerWarps * 32;
-    static constexpr int kQBytes = kRowsPad * 256;
-    static constexpr int kMaxStages = (kSmemLimit - 1024 - kQBytes - kDraftBytes - kMiscBytes) / kStageBytes;
-    static constexpr int kStages = kMaxStages > 6 ? 6 : kMaxStages;
-    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kQBytes + kDraftBytes + kMiscBytes;
-    static_assert(kConsumerWarps <= kMathWarps, "too many consumer warps");
-    static_assert(kStages >= 3, "pipeline too shallow");
-    static_assert(kKeysPerWarp == 16 || kKeysPerWarp == 32, "a warp takes 16 or 32 keys of a stage");
-    // the cross-warp merge at the end reuses the ring and, behind it, the Q tile
-    static_assert(KS * kRowsPad * (128 + 2) * 4 <= kStages * kStageBytes + kQBytes, "merge area does not fit");
-};
-
-// NK keys (16 or 32) starting at key0 of a tile: S = Q K^T, masked online softmax, O += P V.
-// HALF = bytes between the dim 0-63 and dim 64-127 halves of the tile (rows * 128).
-template <int MT, int NK, uint32_t HALF, bool DRAFT>
-__device__ __forceinline__ void process_keys(uint32_t kbase, uint32_t vbase, uint32_t qbase, uint32_t q_half_stride,
-                                             int row_base, const uint32_t (&qf)[8][4], float (&o)[MT][16][4],
-                                             float (&m)[MT][2], float (&l)[MT][2], float scale_log2, int key0,
-                                             int nvalid, const uint32_t (&vis)[MT][2], int lane)
-{
-    float sacc[MT][NK / 8][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < NK / 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) sacc[mt][nt][e] = 0.f;
-
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-        uint32_t qa[MT][4];
-        if constexpr (MT == 1) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) qa[0][e] = qf[ks][e];
-        } else {
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                const uint32_t row = row_base + mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-                const uint32_t chunk = ks * 2 + (lane >> 4);
-                ldsm_x4(qa[mt], qbase + (chunk >> 3) * q_half_stride + swz128(row, chunk & 7));
-            }
-        }
-#pragma unroll
-        for (int np = 0; np < NK / 16; ++np) {
-            const uint32_t key = key0 + np * 16 + (lane >> 4) * 8 + (lane & 7);
-            const uint32_t chunk = ks * 2 + ((lane >> 3) & 1);
-            uint32_t kb[4];
-            ldsm_x4(kb, kbase + (chunk >> 3) * HALF + swz128(key, chunk & 7));
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                mma_bf16_16816(sacc[mt][2 * np], qa[mt], kb[0], kb[1]);
-                mma_bf16_16816(sacc[mt][2 * np + 1], qa[mt], kb[2], kb[3]);
-            }
-        }
-    }
-
-    if (DRAFT || nvalid < key0 + NK) {
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < NK / 8; ++nt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int col = key0 + nt * 8 + 2 * (lane & 3) + (e & 1);
-                    bool ok = col < nvalid;
-                    if (DRAFT) ok = ok && ((vis[mt][e >> 1] >> col) & 1u);
-                    if (!ok) sacc[mt][nt][e] = -INFINITY;
-                }
-    }
-
-    uint32_t pa[MT][NK / 16][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            float mx = -INFINITY;
-#pragma unroll
-            for (int nt = 0; nt < NK / 8; ++nt) mx = fmaxf(mx, fmaxf(sacc[mt][nt][2 * r], sacc[mt][nt][2 * r + 1]));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float m_new = fmaxf(m[mt][r], mx * scale_log2);
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-            const float corr = fast_exp2(m[mt][r] - m_use);
-            m[mt][r] = m_new;
-            float lsum = 0.f;
-#pragma unroll
-            for (int nt = 0; nt < NK / 8; ++nt) {
-                const float p0 = fast_exp2(fmaf(sacc[mt][nt][2 * r], scale_log2, -m_use));
-                const float p1 = fast_exp2(fmaf(sacc[mt][nt][2 * r + 1], scale_log2, -m_use));
-                sacc[mt][nt][2 * r] = p0;
-                sacc[mt][nt][2 * r + 1] = p1;
-                lsum += p0 + p1;
-            }
-            l[mt][r] = l[mt][r] * corr + lsum;
-            if (corr != 1.f) {   // the running maximum moved: rescale the accumulator rows of this thread
-#pragma unroll
-                for (int nt = 0; nt < 16; ++nt) {
-                    o[mt][nt][2 * r] *= corr;
-                    o[mt][nt][2 * r + 1] *= corr;
-                }
-            }
-        }
-#pragma unroll
-        for (int kk = 0; kk < NK / 16; ++kk) {
-            pa[mt][kk][0] = pack_bf16(sacc[mt][2 * kk][0], sacc[mt][2 * kk][1]);
-            pa[mt][kk][1] = pack_bf16(sacc[mt][2 * kk][2], sacc[mt][2 * kk][3]);
-            pa[mt][kk][2] = pack_bf16(sacc[mt][2 * kk + 1][0], sacc[mt][2 * kk + 1][1]);
-            pa[mt][kk][3] = pack_bf16(sacc[mt][2 * kk + 1][2], sacc[mt][2 * kk + 1][3]);
-        }
-    }
-
-#pragma unroll
-    for (int kk = 0; kk < NK / 16; ++kk) {
-        const uint32_t key = key0 + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-#pragma unroll
-        for (int dp = 0; dp < 8; ++dp) {
-            const uint32_t chunk = dp * 2 + (lane >> 4);
-            uint32_t vb[4];
-            ldsm_x4_trans(vb, vbase + (chunk >> 3) * HALF + swz128(key, chunk & 7));
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                mma_bf16_16816(o[mt][2 * dp], pa[mt][kk], vb[0], vb[1]);
-                mma_bf16_16816(o[mt][2 * dp + 1], pa[mt][kk], vb[2], vb[3]);
-            }
-        }
-    }
-}
-
-template <int WM, int MT, int KS>
-__global__ void __launch_bounds__(kThreads, 1)
-    verify_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                       const AttnParams p)
-{
-    using C = Cfg<WM, MT, KS>;
-    constexpr int ROWS_PAD = C::kRowsPad, STAGES = C::kStages, KW = C::kKeysPerWarp;
-    constexpr int kConsumerWarps = C::kConsumerWarps, kConsumerThreads = C::kConsumerThreads;
-
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *smem = smem_raw + (smem0 - smem_u32(smem_raw));
-    const uint32_t stage_base = smem0;
-    const uint32_t q_base = stage_base + STAGES * kStageBytes;
-    const uint32_t draft_base = q_base + C::kQBytes;
-    uint8_t *misc = smem + STAGES * kStageBytes + C::kQBytes + kDraftBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(misc);                 // full[STAGES], empty[STAGES]
-    int *meta = reinterpret_cast<int *>(misc + 256);                     // valid keys of the unit in each stage
-    uint32_t *anc = reinterpret_cast<uint32_t *>(misc + 256 + 64);       // [32] visible-draft masks
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 256 + 64 + 128);
-    const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + STAGES);
-
-    const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int upb = p.B / kUnit;
-    const bool has_draft = split == p.splits - 1;
-    const int rows = p.G * p.T;
-
-    if (tid == 0) {
-        SV_STAMP(0);
-        for (int i = 0; i < STAGES; ++i) {
-            mbar_init(full_bar + 8 * i, 1);
-            mbar_init(empty_bar + 8 * i, kConsumerWarps);
-        }
-        *abort_flag = 0;
-        mbar_fence_init();
-    }
-    __syncthreads();
-    if (tid == 0) SV_STAMP(1);
-
-    if (warp >= kMathWarps) {
-        // -------------------------------------------------------------- producer warpgroup
-        reg_dealloc<40>();   // hand registers to the math warpgroups
-        if (warp != kMathWarps) return;
-        if (lane == 0) {
-            tma_prefetch_desc(&tm_k);
-            tma_prefetch_desc(&tm_v);
-        }
-        // The block list is written by the kernel that precedes this one in the stream.
-        grid_dependency_wait();
-        if (lane == 0) SV_STAMP(2);
-        const int L = p.seq_lens[s];
-        const int nb = min((L + p.B - 1) / p.B, p.NBmax);
-        const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-        const int j0 = (int)((long long)split * n_sel / p.splits);
-        const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
-        const uint64_t policy = policy_evict_first();
-        bool dead = false;
-        for (int base = j0; base < j1; base += 32) {
-            const int j = base + lane;
-            int row0 = 0, tok0 = 0;
-            if (j < j1) {
-                int blk = p.sel_idx ? p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j] : j;
-                blk = max(0, min(blk, p.NBmax - 1));
-                const int page = p.block_table[(size_t)s * p.NBmax + blk];
-                row0 = (page * p.Hkv + h) * p.B;
-                tok0 = blk * p.B;
-            }
-            const int n_here = min(32, j1 - base);
-            for (int i = 0; i < n_here; ++i) {
-                const int r0 = __shfl_sync(0xffffffffu, row0, i);
-                const int t0 = __shfl_sync(0xffffffffu, tok0, i);
-                if (lane == 0 && i == 0 && base == j0) SV_STAMP(3);
-                if (lane == 0 && !dead) {
-                    for (int uo = 0; uo < upb; ++uo) {
-                        const int u = (base - j0 + i) * upb + uo;
-                        const int stage = u % STAGES, it = u / STAGES;
-                        if (it > 0 && !mbar_wait_bounded(empty_bar + 8 * stage, (it - 1) & 1)) {
-                            dead = true;
-                            *abort_flag = 1;
-                            if (p.status) atomicOr(p.status, 1);
-                            break;
-                        }
-                        const int nvalid = max(0, min(kUnit, L - (t0 + uo * kUnit)));
-                        meta[stage] = nvalid;
-                        const uint32_t fb = full_bar + 8 * stage;
-                        if (nvalid > 0) {
-                            const uint32_t dst = stage_base + stage * kStageBytes;
-                            const int y = r0 + uo * kUnit;
-                            mbar_arrive_expect_tx(fb, kStageBytes);
-                            tma_load_2d(dst, &tm_k, 0, y, fb, policy);
-                            tma_load_2d(dst + 8192, &tm_k, 64, y, fb, policy);
-                            tma_load_2d(dst + 16384, &tm_v, 0, y, fb, policy);
-                            tma_load_2d(dst + 24576, &tm_v, 64, y, fb, policy);
-                            if (u == 0) SV_STAMP(4);
-                        } else {
-                            mbar_arrive(fb);
-                        }
-                    }
-                }
-            }
-        }
-        return;
-    }
-
-    // ------------------------------------------------------------------ math warpgroups
-    reg_alloc<232>();
-    grid_dependency_wait();
-    grid_launch_dependents();   // the next kernel may be scheduled; it waits for this grid before reading
-    // Stage Q (and, in the last split, the draft tokens' K/V) while the producer chases the block list.
-    // Q rows r = i*G + g  ->  q[s][i][h*G + g][:], zero padded to ROWS_PAD, stored swizzled
-    for (int idx = tid; idx < ROWS_PAD * 16; idx += kMathThreads) {
-        const int r = idx >> 4, c = idx & 15;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (r < rows) {
-            const int i = r / p.G, g = r - i * p.G;
-            v = __ldg(reinterpret_cast<const uint4 *>(p.q + (((size_t)s * p.T + i) * p.Hq + h * p.G + g) * 128) + c);
-        }
-        *reinterpret_cast<uint4 *>(smem + (q_base - smem0) + (c >> 3) * (ROWS_PAD * 128) + swz128(r, c & 7)) = v;
-    }
-    if (has_draft) {
-        for (int idx = tid; idx < 2 * kDraftRows * 16; idx += kMathThreads) {
-            const int which = idx / (kDraftRows * 16);   // 0: K, 1: V
-            const int r = (idx >> 4) % kDraftRows, c = idx & 15;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < p.T) {
-                const __nv_bfloat16 *src = (which ? p.draft_v : p.draft_k) + (((size_t)s * p.T + r) * p.Hkv + h) * 128;
-                v = __ldg(reinterpret_cast<const uint4 *>(src) + c);
-            }
-            *reinterpret_cast<uint4 *>(smem + (draft_base - smem0) + which * (2 * kDraftRows * 128) +
-                                       (c >> 3) * (kDraftRows * 128) + swz128(r, c & 7)) = v;
-        }
-        if (tid < kDraftRows) {
-            uint32_t mask = 0;
-            if (tid < p.T) {
-                if (p.parent) {
-                    int a = tid;
-                    for (int step = 0; step < p.T && a >= 0; ++step) {
-                        mask |= 1u << a;
-                        const int nxt = p.parent[(size_t)s * p.T + a];
-                        a = nxt < a ? nxt : -1;   // parents must precede their children
-                    }
-                } else {
-                    mask = (tid == 31) ? 0xFFFFFFFFu : ((1u << (tid + 1)) - 1u);
-                }
-            }
-            anc[tid] = mask;
-        }
-    }
-    named_bar_sync(2, kMathThreads);
-    if (tid == 0) SV_STAMP(5);
-    if (warp >= kConsumerWarps) return;   // math warps this shape does not use
-
-    const int wm = warp % WM, kq = warp / WM;
-    const int row_base = wm * MT * 16;
-    const int key0 = kq * KW;
-    uint32_t qf[8][4];
-    if constexpr (MT == 1) {
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t row = row_base + (lane & 7) + ((lane >> 3) & 1) * 8;
-            const uint32_t chunk = ks * 2 + (lane >> 4);
-            ldsm_x4(qf[ks], q_base + (chunk >> 3) * (ROWS_PAD * 128) + swz128(row, chunk & 7));
-        }
-    }
-    float o[MT][16][4], m[MT][2], l[MT][2];
-    uint32_t vis[MT][2];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-        for (int nt = 0; nt < 16; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) o[mt][nt][e] = 0.f;
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            m[mt][r] = -INFINITY;
-            l[mt][r] = 0.f;
-            vis[mt][r] = 0xFFFFFFFFu;
-        }
-    }
-
-    // the draft tokens first: their tile is already in shared memory (warps kq == 0 take all 32 keys)
-    if (has_draft && kq == 0) {
-        const uint32_t all = (p.T == 32) ? 0xFFFFFFFFu : ((1u << p.T) - 1u);
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int row = row_base + mt * 16 + (lane >> 2) + 8 * r;
-                vis[mt][r] = row < rows ? anc[row / p.G] : all;
-            }
-        process_keys<MT, kDraftRows, kDraftRows * 128, true>(draft_base, draft_base + 2 * kDraftRows * 128, q_base,
-                                                             ROWS_PAD * 128, row_base, qf, o, m, l, p.scale_log2, 0,
-                                                             p.T, vis, lane);
-    }
-
-    if (tid == 0) SV_STAMP(6);
-    const int L = p.seq_lens[s];
-    const int nb = min((L + p.B - 1) / p.B, p.NBmax);
-    const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-    const int j0 = (int)((long long)split * n_sel / p.splits);
-    const int j1 = (int)((long long)(split + 1) * n_sel / p.splits);
-    const int n_units = (j1 - j0) * upb;
-    bool dead = false;
-    for (int u = 0; u < n_units; ++u) {
-        const int stage = u % STAGES, it = u / STAGES;
-        if (!dead && (*abort_flag || !mbar_wait_bounded(full_bar + 8 * stage, it & 1))) {
-            dead = true;
-            *abort_flag = 1;
-            if (p.status && lane == 0) atomicOr(p.status, 2);
-        }
-        if (dead) continue;
-        if (tid == 0 && u == 0) SV_STAMP(7);
-        if (tid == 0 && u == n_units - 1) SV_STAMP(8);
-        const int nvalid = min(meta[stage], kUnit);
-        if (nvalid > key0) {
-            const uint32_t kb = stage_base + stage * kStageBytes, vb = kb + 16384;
-            if (nvalid < key0 + KW) {
-                // zero this warp's value rows past the end of the sequence (0 * junk must stay 0)
-                for (int idx = lane; idx < (key0 + KW - nvalid) * 16; idx += 32) {
-                    const int r = nvalid + (idx >> 4), c = idx & 15;
-                    *reinterpret_cast<uint4 *>(smem + (vb - smem0) + (c >> 3) * 8192 + swz128(r, c & 7)) =
-                        make_uint4(0u, 0u, 0u, 0u);
-                }
-                fence_proxy_async();   // order these generic writes before the next TMA fill of the stage
-                __syncwarp();
-            }
-            process_keys<MT, KW, kUnit * 128, false>(kb, vb, q_base, ROWS_PAD * 128, row_base, qf, o, m, l, p.scale_log2,
-                                                     key0, nvalid, vis, lane);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
-    }
-
-    // ------------------------------------------------------------------ merge the key splits of the CTA
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            l[mt][r] += __shfl_xor_sync(0xffffffffu, l[mt][r], 1);
-            l[mt][r] += __shfl_xor_sync(0xffffffffu, l[mt][r], 2);
-        }
-    if (tid == 0) SV_STAMP(9);
-    named_bar_sync(1, kConsumerThreads);   // every stage has been consumed: the ring is free
-    float *part_o = reinterpret_cast<float *>(smem);                 // [KS][ROWS_PAD][128]
-    float *part_m = part_o + KS * ROWS_PAD * 128;                    // [KS][ROWS_PAD]
-    float *part_l = part_m + KS * ROWS_PAD;
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const int row = row_base + mt * 16 + (lane >> 2) + 8 * r;
-            float *dst = part_o + ((size_t)kq * ROWS_PAD + row) * 128 + 2 * (lane & 3);
-#pragma unroll
-            for (int nt = 0; nt < 16; ++nt)
-                *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(o[mt][nt][2 * r], o[mt][nt][2 * r + 1]);
-            if ((lane & 3) == 0) {
-                part_m[kq * ROWS_PAD + row] = m[mt][r];
-                part_l[kq * ROWS_PAD + row] = l[mt][r];
-            }
-        }
-    named_bar_sync(1, kConsumerThreads);
-
-    const size_t sh = (size_t)s * p.Hkv + h;
-    for (int idx = tid; idx < rows * 32; idx += kConsumerThreads) {
-        const int row = idx >> 5, c4 = idx & 31;
-        float M = -INFINITY;
-#pragma unroll
-        for (int g = 0; g < KS; ++g) M = fmaxf(M, part_m[g * ROWS_PAD + row]);
-        const float M_use = (M == -INFINITY) ? 0.f : M;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float lsum = 0.f;
-#pragma unroll
-        for (int g = 0; g < KS; ++g) {
-            const float w = fast_exp2(part_m[g * ROWS_PAD + row] - M_use);
-            const float4 v = *reinterpret_cast<const float4 *>(part_o + ((size_t)g * ROWS_PAD + row) * 128 + c4 * 4);
-            acc.x += w * v.x, acc.y += w * v.y, acc.z += w * v.z, acc.w += w * v.w;
-            lsum += w * part_l[g * ROWS_PAD + row];
-        }
-        if (p.splits == 1) {
-            const int i = row / p.G, g = row - i * p.G;
-            const size_t orow = ((size_t)s * p.T + i) * p.Hq + h * p.G + g;
-            const float inv = 1.f / lsum;
-            uint2 pk;
-            pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-            pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *reinterpret_cast<uint2 *>(p.out + orow * 128 + c4 * 4) = pk;
-            if (p.lse && c4 == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
-        } else {
-            const size_t prow = (sh * p.splits + split) * rows + row;
-            *reinterpret_cast<float4 *>(p.ws_o + prow * 128 + c4 * 4) = acc;
-            if (c4 == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
-        }
-    }
-    if (tid == 0) SV_STAMP(10);
-}
+constexpr int kUnit = 64;   // keys per pipeline stage of the attention kernel (box rows of the tensor maps)
 
 // Small CTAs: the reads of one launch (all partials, ~2 MB for the 32K-context case) spread over every SM.
 constexpr int kMergeThreads = 64;
@@ -616,17 +146,6 @@ bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
 
 using svh::sm_count;
 
-// The tcgen05 kernel is the product path.  Setting SV_ATTN_IMPL=mma in the environment (read once)
-// selects the older mma.sync kernel, kept for A/B comparisons of the two tensor-core paths.
-bool use_tensor_memory_path()
-{
-    static const bool tc = [] {
-        const char *v = getenv("SV_ATTN_IMPL");
-        return !(v && v[0] == 'm');
-    }();
-    return tc;
-}
-
 // Blocks per CTA are minimised subject to one CTA per SM; then the fewest splits that achieve it.
 // With at least one (sequence, KV head, row tile) per SM nothing needs splitting for occupancy, but long lists are
 // still cut into pieces of about 64 units when `balance` is set: the sequences of a batch differ in length, one CTA
@@ -634,38 +153,15 @@ bool use_tensor_memory_path()
 // that out (16 ragged sequences of 4.8-15K tokens, dense: 138 -> 90 us).
 int choose_splits(const sv_geom *g, int n_blocks, bool balance = true)
 {
-    const int pairs = g->n_seq * g->n_kv_heads * (use_tensor_memory_path() ? svh::row_tiles(g) : 1);
+    const int pairs = g->n_seq * g->n_kv_heads * svh::row_tiles(g);
     const int per_pair = sm_count() / pairs;
     if (n_blocks <= 1) return 1;
     if (per_pair <= 1) {
         const int units = n_blocks * (g->block_size / 64);
-        return (balance && use_tensor_memory_path() && units >= 128) ? (units + 63) / 64 : 1;
+        return (balance && units >= 128) ? (units + 63) / 64 : 1;
     }
     const int blocks_per_cta = (n_blocks + per_pair - 1) / per_pair;
     return (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
-}
-
-template <int WM, int MT, int WT>
-cudaError_t launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p, dim3 grid, cudaStream_t cs)
-{
-    using C = Cfg<WM, MT, WT>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(verify_attn_kernel<WM, MT, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = C::kSmemBytes;
-    cfg.stream = cs;
-    cudaLaunchAttribute attr[1];
-    svh::pdl_attribute(attr);
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, verify_attn_kernel<WM, MT, WT>, tk, tv, p);
 }
 
 }  // namespace
@@ -681,6 +177,7 @@ namespace {
 size_t workspace_bytes_for(const sv_geom *geom, int32_t max_sel, bool balance)
 {
     const size_t splits = (size_t)choose_splits(geom, max_sel, balance);
+    if (splits <= 1) return 0;   // one CTA per (sequence, KV head) writes the output itself: no partials
     const size_t rows = (size_t)(geom->n_q_heads / geom->n_kv_heads) * geom->n_draft;
     return (size_t)geom->n_seq * geom->n_kv_heads * splits * rows * (128 + 2) * sizeof(float) + 256;
 }
@@ -742,31 +239,15 @@ static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_k
     p.T = geom->n_draft, p.Hq = geom->n_q_heads, p.Hkv = geom->n_kv_heads, p.G = G, p.B = geom->block_size;
     p.NBmax = geom->max_blocks, p.max_sel = max_sel, p.splits = splits;
     p.Tt = svh::tokens_per_tile(geom), p.tiles = svh::row_tiles(geom);
+    p.n_pages = kv->n_pages;
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;   // 1/sqrt(128)
     p.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     dim3 grid(splits, geom->n_kv_heads, geom->n_seq);
-    cudaError_t e;
-    if (!use_tensor_memory_path() && (rows > svh::kMaxRows || geom->n_draft > 32)) return SV_ERR_UNSUPPORTED;
-    if (use_tensor_memory_path()) grid.x = splits * p.tiles;   // one CTA per (row tile, split)
-    if (use_tensor_memory_path())
-        e = launch_attn_tc(tk, tv, p, grid, cs);          // tcgen05 + TMEM, rows padded to one M = 128 tile
-    else if (rows <= 16)
-        e = launch_attn<1, 1, 4>(tk, tv, p, grid, cs);   // 4 warps: 16 rows x 16 keys of each stage
-    else if (rows <= 32)
-        e = launch_attn<2, 1, 4>(tk, tv, p, grid, cs);   // 8 warps: 2 row tiles x 4 key quarters
-    else if (rows <= 64)
-        e = launch_attn<4, 1, 2>(tk, tv, p, grid, cs);   // 8 warps: 4 row tiles x 2 key halves
-    else
-        e = launch_attn<4, 2, 2>(tk, tv, p, grid, cs);   // 8 warps: 4 x 32 rows x 2 key halves
-    if (e != cudaSuccess) return SV_ERR_CUDA;
-#ifdef SV_TRACE
-    const bool skip_merge = getenv("SV_PROBE_SKIP_MERGE") != nullptr;   // development builds only: time the attention kernel alone
-#else
-    const bool skip_merge = false;
-#endif
-    if (splits > 1 && !skip_merge) {
+    grid.x = splits * p.tiles;   // one CTA per (row tile, split)
+    if (launch_attn_tc(tk, tv, p, grid, cs) != cudaSuccess) return SV_ERR_CUDA;
+    if (splits > 1) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((rows * 32 + kMergeThreads - 1) / kMergeThreads, geom->n_kv_heads, geom->n_seq);
         cfg.blockDim = dim3(kMergeThreads);

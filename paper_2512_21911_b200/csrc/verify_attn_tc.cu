@@ -1,6 +1,6 @@
 // Sparse verification attention on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
-// Same contract as the mma.sync kernel in verify_attn.cu: grid (split, KV head, sequence); a CTA owns
+// Grid (split [x row tile], KV head, sequence); a CTA owns
 // a contiguous slice of the ascending block list of its (sequence, KV head) and all G*T query rows of
 // that KV head, padded to one M = 128 tile.  Per 64-key unit (32 KB of K and V gathered by TMA):
 //
@@ -27,53 +27,14 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include <stdlib.h>
-
 #include "attn_common.cuh"
+#include "sv_host.h"
 #include "sv_ptx.cuh"
-
-#ifndef SV_TRACE_U0
-#define SV_TRACE_U0 0
-#endif
-#ifdef SV_TRACE
-// Development aid (never compiled into the library): cycle stamps of the first CTAs (units SV_TRACE_U0 .. + 23) and
-// the wall-clock start / end of every CTA.
-__device__ long long g_sv_trace_tc[32 * 128];
-__device__ long long g_sv_trace_cta[1024 * 2];
-extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_cta()
-{
-    long long *p = nullptr;
-    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace_cta);
-    return p;
-}
-extern "C" __attribute__((visibility("default"))) long long *sv_trace_buffer_tc()
-{
-    long long *p = nullptr;
-    cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_sv_trace_tc);
-    return p;
-}
-#define TC_STAMP(slot)                                                                     \
-    do {                                                                                   \
-        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);   \
-        if (cta_ < 32 && (slot) < 128) g_sv_trace_tc[cta_ * 128 + (slot)] = clock64();     \
-        if ((slot) == 0 || (slot) == 120) {                                                \
-            long long ns_;                                                                 \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_));                        \
-            if (cta_ < 32) g_sv_trace_tc[cta_ * 128 + ((slot) == 0 ? 121 : 122)] = ns_;    \
-            if (cta_ < 1024) g_sv_trace_cta[cta_ * 2 + ((slot) == 0 ? 0 : 1)] = ns_;       \
-        }                                                                                  \
-    } while (0)
-#else
-#define TC_STAMP(slot) \
-    do {               \
-    } while (0)
-#endif
 
 namespace svk {
 namespace {
 
 constexpr int kThreads = 384;
-constexpr int kTraceU0 = SV_TRACE_U0;
 constexpr int kUnit = 64;                        // keys per unit
 constexpr int kTile = kUnit * 128;               // bytes of one [64 rows][64 bf16] half tile (8 KB)
 constexpr int kStageBytes = 4 * kTile;           // K lo/hi + V lo/hi
@@ -151,7 +112,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     };
     const float inv_g = 1.f / (float)p.G;
     auto div_g = [&](int r) { return (int)(((float)r + 0.5f) * inv_g); };
-    if (tid == 0) TC_STAMP(0);
     // The TMA producer warp initialises the barriers and runs ahead; everybody else meets it at a named
     // barrier (the producer only arrives), with the TMEM allocation done by warp 9 on the way.
     if (warp == 8) {
@@ -174,7 +134,6 @@ __global__ void __launch_bounds__(kThreads, 1)
         tc_fence_after_sync();
     }
     const uint32_t tmem_base = warp == 8 ? 0u : *tmem_slot;
-    if (tid == 0) TC_STAMP(1);
 
     if (warp >= 8) {
         reg_dealloc<40>();   // hand registers to the softmax warpgroups
@@ -196,7 +155,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 blk_spec = p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j0_spec + lane];
             const int L = p.seq_lens[s];
             const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
-            const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
+            const int cnt_in = p.sel_idx ? p.sel_cnt[(size_t)s * p.Hkv + h] : nb;
+            // a negative count marks a list that block selection could not produce: attend over the draft tokens
+            // only, and say so
+            if (cnt_in < 0 && lane == 0 && p.status) atomicOr(p.status, kStatusNoList);
+            const int n_sel = p.sel_idx ? max(0, min(cnt_in, p.max_sel)) : nb;
             const int j0 = slice_begin(split, n_sel);
             const int j1 = slice_begin(split + 1, n_sel);
             const int off = has_draft ? 1 : 0;
@@ -208,8 +171,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                     int blk = j;
                     if (p.sel_idx)
                         blk = (base == j0 && j0 == j0_spec) ? blk_spec : p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j];
+                    // indices are clamped into their tables before any address is formed; a clamp that fires is reported
+                    const int blk_in = blk;
                     blk = max(0, min(blk, p.NBmax - 1));
-                    const int page = p.block_table[(size_t)s * p.NBmax + blk];
+                    const int page_in = p.block_table[(size_t)s * p.NBmax + blk];
+                    const int page = max(0, min(page_in, p.n_pages - 1));
+                    if ((blk != blk_in || page != page_in) && p.status) atomicOr(p.status, kStatusIndex);
                     row0 = (page * p.Hkv + h) * p.B;
                     tok0 = blk * p.B;
                 }
@@ -234,7 +201,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                             const int y = r0 + uo * kUnit;
                             // an empty unit (block 128, tail of at most 64 tokens) is still loaded:
                             // it keeps the unit sequence uniform and is fully masked downstream
-                            if (u >= kTraceU0 && u < kTraceU0 + 24) TC_STAMP(8 + u - kTraceU0);
                             mbar_arrive_expect_tx(fb, kStageBytes);
                             tma_load_2d(dst, &tm_k, 0, y, fb, policy);
                             tma_load_2d(dst + kTile, &tm_k, 64, y, fb, policy);
@@ -249,8 +215,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             // warp 9 issues every S = Q K^T and owns the TMEM allocation; warp 10 issues every Ou = P V.
             // Descriptors are built once; per instruction only the 14-bit address field moves.
             if (lane == 0) {
+                grid_dependency_wait();   // the lengths may come from the kernel just before (a cache commit)
                 const int L = p.seq_lens[s];
-                grid_dependency_wait();
                 const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
                 const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
                 const int j0 = slice_begin(split, n_sel);
@@ -284,7 +250,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                             tc_mma_bf16(d, d_hi | (dq_lo + qo), d_hi | (k_lo + ko), idesc_s, ks > 0);
                         }
                         tc_commit(bar(kSReady + g));
-                        if (u >= kTraceU0 && u < kTraceU0 + 24) TC_STAMP(32 + u - kTraceU0);
                     }
                     // free TMEM only after every softmax warp has finished reading it
                     if (!mbar_wait_bounded(bar(kTmemDone), 0) && p.status) atomicOr(p.status, 16);
@@ -313,7 +278,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                                         idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);   // the warpgroup's first unit starts O
                         tc_commit(bar(kOReady + g));
                         tc_commit(bar(kEmpty + stage));
-                        if (u >= kTraceU0 && u < kTraceU0 + 24) TC_STAMP(56 + u - kTraceU0);
                     }
                 }
             }
@@ -349,7 +313,6 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     }
     grid_dependency_wait();
-    if (tid == 0) TC_STAMP(3);
     {
         // real rows: all loads of a thread are in flight together (16-byte chunks: Q up to 128 rows x 16, draft K and
         // V up to 64 tokens x 16 each)
@@ -375,7 +338,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                 w[x] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
             }
         }
-        if (tid == 0) TC_STAMP(4);
         if (!kWide && has_draft && tid < 32) {
             uint32_t mask = 0;
             if (tid < p.T) {
@@ -426,12 +388,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
         }
     }
-    if (tid == 0) TC_STAMP(5);
     fence_proxy_async();   // the tensor cores read these tiles through the async proxy
     named_bar_sync(2, 256);
     if (lane == 0) mbar_arrive(bar(kStaged));
     if (has_draft && tid == 0) mbar_arrive(bar(kFull + 0));   // the draft unit fills stage 0 in place of a TMA load
-    if (tid == 0) TC_STAMP(2);
 
     const int wg = warp >> 2, quad = warp & 3;
     if (quad >= n_active) return;                                 // this warp's TMEM lanes hold padding only
@@ -501,7 +461,6 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (p.status && lane == 0) atomicOr(p.status, 2);
         }
         if (dead) break;
-        if (tid == 0 && k >= kTraceU0 / 2 && k < kTraceU0 / 2 + 12) TC_STAMP(80 + k - kTraceU0 / 2);
         tc_fence_after_sync();
         const bool is_draft = u < off;
         const int stage = u % kStages;
@@ -696,7 +655,6 @@ __global__ void __launch_bounds__(kThreads, 1)
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kPReady + wg));
-        if (tid == 0 && k >= kTraceU0 / 2 && k < kTraceU0 / 2 + 12) TC_STAMP(92 + k - kTraceU0 / 2);
     }
     if constexpr (NH == 4) {
         // back to the four-threads-per-row slots the read-out uses: slot i of this thread is row 8 i + lane / 4 of the warp
@@ -727,10 +685,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         ml_mine[(2 * i + 1) * 128 + t] = l[i];
     }
     tc_fence_before_sync();
-    if (tid == 0) TC_STAMP(104);
     named_bar_sync(1, n_sm);
     tc_fence_after_sync();
-    if (tid == 0) TC_STAMP(106);
     // a warpgroup without units never wrote its accumulator
     const bool have_mine = k > 0 && !dead, have_other = n_total >= (wg == 0 ? 2 : 1);
     const uint32_t t_o_other = tmem_base + t_lane + 128 + (wg ^ 1) * 128;
@@ -764,7 +720,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
         }
     }
-    if (tid == 0) TC_STAMP(105);
     tc_fence_before_sync();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar(kTmemDone));   // this warp reads TMEM no more
@@ -789,7 +744,6 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (wg == 0 && qd == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
         }
     }
-    if (tid == 0) TC_STAMP(120);
 }
 
 }  // namespace
@@ -798,24 +752,18 @@ template <int NH, bool kWide>
 static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                              cudaStream_t stream)
 {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static svh::OncePerDevice once;   // function attributes belong to a device
+    const cudaError_t ce = once.run([] {
+        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    });
+    if (ce != cudaSuccess) return ce;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-#ifdef SV_TRACE
-    attr[0].val.programmaticStreamSerializationAllowed = getenv("SV_PROBE_NO_PDL") ? 0 : 1;   // development builds only
-#else
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-#endif
+    svh::pdl_attribute(attr);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide>, tm_k, tm_v, p);

@@ -128,6 +128,16 @@ class SparseVerifier:
         if self._stack_kv is not None:
             self._stack_lens.copy_(self.seq_lens.repeat(self.n_layers))
 
+    def check_status(self) -> None:
+        """Read the device status word back (this synchronises with the stream) and raise if a kernel gave up
+        on a bounded wait, clamped a block index or page id, or met a list that block selection marked invalid
+        (count -1).  The outputs written since the word was last zero are then invalid."""
+        st = sv.sv_status_word_check(int(self.status.item()))
+        if st == sv.SV_OK and int(self.sel_cnt.min().item()) < 0:
+            st = 9   # SV_ERR_INDEX: a list marked invalid that no attention call has consumed yet
+        if st != sv.SV_OK:
+            raise sv.SvError(st, "SparseVerifier.check_status")
+
     def dense_step(self, q, draft_k, draft_v, out) -> None:
         for l in range(self.n_layers):
             self.dense_layer(l, q[l], draft_k[l], draft_v[l], out[l])

@@ -417,20 +417,152 @@ def test_stacked_tail_refresh_equals_per_layer(sv):
             np.testing.assert_allclose(full[l, s, :, :nb].cpu().numpy(), ref[s, :, :nb], rtol=1e-5, atol=1e-6)
 
 
-def test_mma_sync_attention_path_stays_green():
-    """The older bf16 mma.sync attention kernel is kept selectable (SV_ATTN_IMPL=mma, read once per
-    process) for A/B runs against the tcgen05 kernel; run the small parity cases through it in a child."""
-    import os
-    import subprocess
-    import sys
-    if os.environ.get("SV_ATTN_IMPL", "").startswith("m"):
-        pytest.skip("already running on the mma.sync path")
-    env = dict(os.environ, SV_ATTN_IMPL="mma")
-    r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-q", "-x", "-m", "gpu", "-k",
-                        "(pipeline_parity_small or more_splits or empty_prefix) and not t60 and not t40 and not g8_t24 and not g16_t64"],
-                       env=env, capture_output=True, text=True,   # the older kernel stops at 128 query rows / 32 draft tokens
-                       cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+def test_out_of_range_indices_are_clamped_and_reported(sv):
+    """Block indices outside the table (-1, NBmax + 5), a page id outside the pool and a list count of -1 never reach
+    an address: the kernel clamps them into their tables and says so in the status word.  Nothing faults; the same
+    call with the valid inputs afterwards is exact again."""
+    c = si.make_layer(si.make_geometry(SMALL["cfg1_small"]), sharp=True)
+    d = Dev(sv, c)
+    idx, cnt, _ = gpu_select(sv, d, c["n_sink"], c["n_local"], c["max_sel"])
+    idx_ref, cnt_ref, _ = oracle_select(c, c["n_sink"], c["n_local"], c["max_sel"])
+    w = d.w
+    ws = torch.empty(max(16, sv.sv_workspace_bytes(d.geom, c["max_sel"])), dtype=torch.uint8, device="cuda")
+
+    def run(idx_t, cnt_t, kv):
+        out = torch.full((w.n_seq, w.n_draft, w.n_q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((w.n_seq, w.n_draft, w.n_q_heads), float("nan"), device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        sv.sv_verify_attn(d.geom, d.q, kv, d.draft_k, d.draft_v, d.parent, idx_t, cnt_t, out, lse=lse, workspace=ws,
+                          status_word=status)
+        torch.cuda.synchronize()
+        return bf16_host(out), lse.cpu().numpy().astype(np.float64), int(status.item())
+
+    bad_idx = idx.clone()
+    bad_idx[0, 0, 1] = -1
+    bad_idx[0, 1, 2] = c["max_blocks"] + 5
+    o, lse, st = run(bad_idx, cnt, d.kv)
+    assert st == sv.SV_STATUS_INDEX and sv.sv_status_word_check(st) == 9 and np.isfinite(o).all()
+    bad_table = d.block_table.clone()
+    bad_table[0, int(idx_ref[0, 0, 3])] = c["n_pages"] + 1000          # a kept block whose page id lies outside the pool
+    bad_table[0, int(idx_ref[0, 0, 4])] = -3
+    o, lse, st = run(idx, cnt, sv.make_kv(d.k_pool, d.v_pool, bad_table, d.seq_lens))
+    assert st == sv.SV_STATUS_INDEX and np.isfinite(o).all()
+    # a list that block selection marked invalid: the draft tokens only, and the word says so
+    no_list = cnt.clone()
+    no_list[0, 1] = -1
+    o, lse, st = run(idx, no_list, d.kv)
+    assert st == sv.SV_STATUS_NO_LIST and sv.sv_status_word_check(st) == 9
+    cnt_exp = cnt_ref.copy()
+    cnt_exp[0, 1] = 0
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_exp)
+    check_attn(o, lse, o_ref, lse_ref, "count -1 = no cached blocks")
+    # the valid inputs again: clean word, exact result
+    o, lse, st = run(idx, cnt, d.kv)
+    assert st == 0 and sv.sv_status_word_check(st) == 0
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref)
+    check_attn(o, lse, o_ref, lse_ref, "after the clamped calls")
+
+
+def test_engine_reports_a_bad_status_word(sv):
+    w = SMALL["cfg1_small"]
+    geom = si.make_geometry(w)
+    eng = sv.SparseVerifier(n_seq=w.n_seq, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                            block_size=w.block_size, max_blocks=geom["max_blocks"], n_draft=w.n_draft, n_layers=1,
+                            block_table=torch.from_numpy(geom["block_table"]).cuda(),
+                            seq_lens=torch.from_numpy(geom["seq_lens"]).cuda(),
+                            budget_blocks=torch.from_numpy(geom["budget"]).cuda(), max_sel=geom["max_sel"])
+    eng.check_status()
+    eng.sel_cnt[0, 0] = -1
+    with pytest.raises(sv.SvError) as e:
+        eng.check_status()
+    assert e.value.status == 9
+    eng.sel_cnt[0, 0] = 0
+    eng.status.fill_(2)
+    with pytest.raises(sv.SvError) as e:
+        eng.check_status()
+    assert e.value.status == 7
+
+
+def test_commit_then_dense_verify_on_the_new_lengths(sv):
+    """sv_kv_append writes the new lengths; a dense sv_verify_attn launched right behind it on the same stream reads
+    them from that buffer.  Sequences cross a block boundary, so a role of the attention kernel that picked the old
+    length up too early would issue fewer tiles than the others expect."""
+    w = si.shrink(SMALL["cfg2_small"], n_draft=8)
+    c = si.make_layer(si.make_geometry(w), sharp=True)
+    S, Hkv, T, B = w.n_seq, w.n_kv_heads, w.n_draft, w.block_size
+    bt = np.concatenate([c["block_table"], np.zeros((S, 1), np.int32)], axis=1)
+    for s in range(S):
+        bt[s, c["n_blocks"][s]] = c["n_pages"] + s
+    g = np.random.default_rng(11)
+    fresh = si.f32_to_bf16_bits(g.standard_normal((S, Hkv, B, 128)).astype(np.float32))
+    k_pool, v_pool = np.concatenate([c["k_pool"], fresh]), np.concatenate([c["v_pool"], fresh[::-1].copy()])
+    lens = ((c["seq_lens"] // B) * B + B - 2).astype(np.int32)       # two slots left: every commit of >= 3 rows adds a block
+    lens = np.minimum(lens, c["n_blocks"] * B - 2).astype(np.int32)
+    n_acc = np.full(S, T, np.int32)
+    acc = np.tile(np.arange(T, dtype=np.int32), (S, 1))
+    NB = bt.shape[1]
+    geom = sv.make_geom(S, w.n_q_heads, Hkv, 128, B, NB, T)
+    kp, vp = bf16_dev(k_pool), bf16_dev(v_pool)
+    btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
+    q, dk, dv = bf16_dev(c["q"]), bf16_dev(c["draft_k"]), bf16_dev(c["draft_v"])
+    new_len = torch.zeros_like(sld)
+    out = torch.full((S, T, w.n_q_heads, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((S, T, w.n_q_heads), float("nan"), device="cuda")
+    ws = torch.empty(max(16, sv.sv_workspace_bytes(geom, NB)), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kv_new = sv.make_kv(kp, vp, btd, new_len)
+    for _ in range(3):      # repeated: the overlap of the two kernels varies from launch to launch
+        kp.copy_(bf16_dev(k_pool)); vp.copy_(bf16_dev(v_pool)); new_len.zero_()
+        sv.sv_kv_append(geom, kp, vp, btd, sld, dk, dv, torch.from_numpy(acc).cuda(), torch.from_numpy(n_acc).cuda(), new_len, None)
+        sv.sv_verify_attn(geom, q, kv_new, dk, dv, None, None, None, out, lse=lse, workspace=ws, status_word=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+    ko, vo = k_pool.copy(), v_pool.copy()
+    len_o = oracle.kv_append(ko, vo, bt, lens, c["draft_k"], c["draft_v"], acc, n_acc, None)
+    assert ((len_o + B - 1) // B > (lens + B - 1) // B).all()
+    np.testing.assert_array_equal(new_len.cpu().numpy(), len_o)
+    o_ref, lse_ref = oracle.dense_verify_attn(c["q"], ko, vo, bt, len_o, c["draft_k"], c["draft_v"], None)
+    check_attn(bf16_host(out), lse.cpu().numpy().astype(np.float64), o_ref, lse_ref, "dense verify right behind a commit")
+
+
+def test_kv_append_drops_rows_for_unassigned_pages(sv):
+    """A block-table entry that is not a page of the pool (-1: not assigned yet) ends the table: rows that would
+    enter that block are dropped, the length stops at the block boundary, and nothing outside the sequence's own
+    pages is written (every other page of the pools is a canary)."""
+    B, Hkv, T, S, NB = 64, 2, 8, 3, 4
+    n_pages = 16
+    g = np.random.default_rng(3)
+    k_pool = si.f32_to_bf16_bits(g.standard_normal((n_pages, Hkv, B, 128)).astype(np.float32))
+    v_pool = si.f32_to_bf16_bits(g.standard_normal((n_pages, Hkv, B, 128)).astype(np.float32))
+    bt = np.array([[2, -1, -1, -1], [5, 7, n_pages + 9, -1], [9, 11, 12, 13]], np.int32)
+    lens = np.array([B - 3, 2 * B - 5, 4 * B - 2], np.int32)     # 3, 5 and 2 slots left before an unusable block / the end
+    n_acc = np.full(S, T, np.int32)
+    acc = np.tile(np.arange(T, dtype=np.int32), (S, 1))
+    dk = si.f32_to_bf16_bits(g.standard_normal((S, T, Hkv, 128)).astype(np.float32))
+    dv = si.f32_to_bf16_bits(g.standard_normal((S, T, Hkv, 128)).astype(np.float32))
+    geom = sv.make_geom(S, 4, Hkv, 128, B, NB, T)
+    kp, vp = bf16_dev(k_pool), bf16_dev(v_pool)
+    new_len = torch.zeros(S, dtype=torch.int32, device="cuda")
+    reps = torch.full((S, Hkv, NB, 128), 7.0, device="cuda")
+    sv.sv_kv_append(geom, kp, vp, torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda(), bf16_dev(dk), bf16_dev(dv),
+                    torch.from_numpy(acc).cuda(), torch.from_numpy(n_acc).cuda(), new_len, reps)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(new_len.cpu().numpy(), [B, 2 * B, 4 * B])
+    k_exp, v_exp = k_pool.copy(), v_pool.copy()
+    for s, (page, n) in enumerate([(2, 3), (7, 5), (13, 2)]):
+        k_exp[page, :, B - n:] = dk[s, :n].transpose(1, 0, 2)
+        v_exp[page, :, B - n:] = dv[s, :n].transpose(1, 0, 2)
+    np.testing.assert_array_equal(kp.cpu().view(torch.int16).numpy().view(np.uint16), k_exp)
+    np.testing.assert_array_equal(vp.cpu().view(torch.int16).numpy().view(np.uint16), v_exp)
+    r = reps.cpu().numpy()
+    assert (r[0, :, 1:] == 7.0).all() and (r[1, :, 2:] == 7.0).all() and (r[2, :, :3] == 7.0).all()
+    np.testing.assert_allclose(r[0, :, 0], si.bf16_bits_to_f64(k_exp[2]).mean(axis=1), rtol=1e-5, atol=1e-6)
+    # a length already past the table: nothing is appended and the length is kept
+    lens2 = np.array([NB * B + 5, 0, 0], np.int32)
+    sv.sv_kv_append(geom, kp, vp, torch.from_numpy(bt).cuda(), torch.from_numpy(lens2).cuda(), bf16_dev(dk), bf16_dev(dv),
+                    torch.from_numpy(acc).cuda(), torch.from_numpy(np.array([4, 0, 0], np.int32)).cuda(), new_len, None)
+    torch.cuda.synchronize()
+    assert int(new_len[0].item()) == NB * B + 5
 
 
 @pytest.mark.parametrize("block", [64, 128])

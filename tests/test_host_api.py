@@ -33,9 +33,21 @@ def test_exports_every_declared_symbol(svb):
 
 
 def test_strerror_texts(svb):
-    texts = {svb._strerror(i) for i in range(8)}
-    assert len(texts) == 8 and "ok" in texts
-    assert svb._strerror(99) == "unknown status"
+    texts = {svb._strerror(i) for i in range(10)}
+    assert len(texts) == 10 and "ok" in texts and "unknown status" not in texts
+    assert "scratch" in svb._strerror(8) and "index" in svb._strerror(9)
+    assert set(svb.STATUS_NAMES) == set(range(10))
+    assert svb._strerror(10) == svb._strerror(99) == "unknown status"
+
+
+def test_status_word_check(svb):
+    assert svb.sv_status_word_check(0) == 0
+    for wait_bit in (1, 2, 4, 8, 16, 32):
+        assert svb.sv_status_word_check(wait_bit) == 7
+        assert svb.sv_status_word_check(wait_bit | svb.SV_STATUS_INDEX) == 7     # a give-up outranks a clamp
+    assert svb.sv_status_word_check(svb.SV_STATUS_INDEX) == 9
+    assert svb.sv_status_word_check(svb.SV_STATUS_NO_LIST) == 9
+    assert svb.sv_status_word_check(1 << 20) == 7                                # unknown bits are not "ok"
 
 
 def test_budget_matches_eq6_and_oracle(svb):

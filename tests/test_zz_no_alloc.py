@@ -2,7 +2,7 @@
 memory (a server whose HBM is fully reserved by its KV-cache pool, code running under another
 component's allocator).  It keeps the split-KV partials in a scratch array built into the library
 instead of a caller workspace.  Checked here, through the C ABI, against the ordinary entry point on
-the same inputs, twice in a row (the array is shared by all calls and keeps the previous call's
+the same inputs (and against the CPU oracle), twice in a row (the array is shared by all calls and keeps the previous call's
 contents, which must not matter).  This file sorts last on purpose: a run that stops at the first
 failure has then already run every other test.
 """
@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import sv_inputs as si
 
 pytestmark = pytest.mark.gpu
@@ -68,6 +69,39 @@ def test_noalloc_matches_workspace_entry_point_twice():
         rel = np.linalg.norm(o - o_ref, axis=-1) / np.linalg.norm(o_ref, axis=-1)
         assert rel.max() <= 1e-2
         assert np.abs(lse.cpu().numpy() - lse_ref.cpu().numpy()).max() <= 1e-3
+        # and against the oracle directly, on the lists the library selected
+        o_cpu, lse_cpu = oracle.verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"],
+                                            c["draft_v"], c["parent"], idx.cpu().numpy(), cnt.cpu().numpy())
+        scale = max(1.0, float(np.abs(o_cpu).max()))
+        assert np.abs(o - o_cpu).max() <= 1e-2 * scale and np.abs(o - o_cpu).mean() <= 1e-3 * scale
+        assert (np.linalg.norm(o - o_cpu, axis=-1) / np.linalg.norm(o_cpu, axis=-1)).max() <= 1e-2
+        assert np.abs(lse.cpu().numpy() - lse_cpu).max() <= 1e-3
+
+
+def test_noalloc_runs_a_large_batch_that_needs_no_partials():
+    """256 (sequence, KV head) pairs of 128 query rows: every SM has a pair and the lists are short, so one CTA per
+    pair writes the output itself.  No partials exist, so the size of the built-in scratch does not matter and the
+    call must run (counted as if it were split, the partials would be four times the scratch)."""
+    import paper_2512_21911_b200 as sv
+    w = si.shrink(si.WORKLOADS["cfg3"], n_seq=32, seq_len=(600, 1024), budget_blocks=5, planted=1)
+    c, geom, t, kv, idx, cnt = _case(sv, w, True, layer=0)
+    assert sv.sv_verify_attn_splits(geom, c["max_sel"]) == 1 and sv.sv_workspace_bytes(geom, c["max_sel"]) == 0
+    rows = (w.n_q_heads // w.n_kv_heads) * w.n_draft
+    assert w.n_seq * w.n_kv_heads * rows * 520 > sv.SV_NOALLOC_SCRATCH_BYTES
+    shape = (w.n_seq, w.n_draft, w.n_q_heads)
+    out = torch.full(shape + (w.head_dim,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full(shape, float("nan"), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sv.sv_verify_attn_noalloc(geom, t["q"], kv, t["dk"], t["dv"], t["parent"], idx, cnt, out, lse=lse, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    smp = [(s, i, hq) for s in (0, 17, 31) for i in (0, 7, 15) for hq in (0, 9, 63)]
+    o_cpu, lse_cpu = oracle.verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"], c["draft_k"],
+                                        c["draft_v"], c["parent"], idx.cpu().numpy(), cnt.cpu().numpy(), samples=smp)
+    o = _host(out)
+    for n, (s_, i, hq) in enumerate(smp):
+        assert np.linalg.norm(o[s_, i, hq] - o_cpu[n]) <= 1e-2 * np.linalg.norm(o_cpu[n])
+        assert abs(float(lse[s_, i, hq]) - lse_cpu[n]) <= 1e-3
 
 
 def test_noalloc_rejects_problems_beyond_the_built_in_scratch():
