@@ -16,8 +16,7 @@
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
-#include <type_traits>
-
+#include "select_core.cuh"
 #include "sv_host.h"
 #include "sv_ptx.cuh"
 
@@ -29,23 +28,8 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kRowsPerIter = 4;   // independent representative rows a warp has in flight
 
-// Histogram bin -> shared-memory slot: one pad word per 32 bins, so that a warp whose lane j reads bins
-// 8j .. 8j+7 (the scan below) touches 32 different banks with every load.
-constexpr int kHistSlots = 256 + 8;
-constexpr int kFastCap = 32;     // ... and at most this many keys left at the boundary after the histogram levels
-__device__ __forceinline__ uint32_t hist_slot(uint32_t bin) { return bin + (bin >> 5); }
-
-// inverse of order_key (defined below): the score a key was made from
-__device__ __forceinline__ float key_score(uint32_t k)
-{
-    return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
-}
-
-__device__ __forceinline__ uint32_t order_key(float x)
-{
-    const uint32_t u = __float_as_uint(x + 0.0f);   // -0 -> +0
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
+using svsel::kForcedKey;
+using svsel::order_key;
 
 struct SelectParams {
     const __nv_bfloat16 *q;   // [S][T][Hq][128]
@@ -57,36 +41,6 @@ struct SelectParams {
     float *out_scores;
     int T, Hq, Hkv, B, NBmax, n_sink, n_local, max_sel, chunk;
 };
-
-__device__ __forceinline__ uint32_t cluster_map_shared(uint32_t addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-// 16-byte store into another CTA's shared memory that reports its bytes to an mbarrier there when it has landed: the
-// receiver needs no fence and no separate arrival from the sender
-__device__ __forceinline__ void st_async_cluster_v4(uint32_t addr, uint4 v, uint32_t remote_bar)
-{
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
-                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(remote_bar)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t parity, uint32_t limit = (1u << 19))
-{
-    for (uint32_t i = 0; i < limit; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
 
 // Cluster of CL CTAs per (sequence, KV head).  Every CTA scores a slice of the blocks and writes the
 // keys straight into CTA 0's shared memory (distributed shared memory) with stores that count their bytes
@@ -104,23 +58,17 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
 
     extern __shared__ __align__(16) uint32_t keys_all[];         // [CL*chunk] keys of all blocks (used in CTA 0)
     __shared__ float qbar[128];
-    __shared__ uint32_t hist[4][kHistSlots];
-    __shared__ unsigned long long cand[kFastCap];   // (key, ~block index) of the keys at the boundary (fast path)
-    __shared__ uint32_t cand_n;
-    __shared__ uint32_t pass_bin[3];               // boundary bin of a radix pass: index, keys still to take in it, its size
-    __shared__ uint32_t warp_sel[kWarps], warp_eq[kWarps];
-    __shared__ uint32_t key_min, key_max;          // smallest / largest evictable key (fast path)
+    __shared__ svsel::Scratch scratch;
     __shared__ uint64_t keys_ready;                // mbarrier in CTA 0: the bytes of all keys (one arrival: CTA 0 itself)
 
     // While the kernel that precedes this one in the stream drains: pull this warp's first batch of
     // representative rows and the query row towards L2 (a prefetch consumes no data, so it is safe even if
     // that kernel is still writing them), set up the barrier, zero the histograms.
     if (tid == 0) {
-        key_min = 0xFFFFFFFFu, key_max = 0u, cand_n = 0;
         svk::mbar_init(svk::smem_u32(&keys_ready), 1);
         svk::mbar_fence_init();
     }
-    for (int i = tid; i < 4 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
+    scratch.init(tid, kThreads);
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // before any global request is in flight
     const int b0 = rank * p.chunk;
     constexpr int kRowBytes = kBf16 ? 256 : 512, kLaneBytes = kRowBytes / 32;
@@ -175,8 +123,8 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     if (tid < 128) qbar[tid] = qsum / (float)G;
     __syncthreads();
 
-    const uint32_t keys0 = cluster_map_shared(svk::smem_u32(keys_all), 0);
-    const uint32_t ready0 = cluster_map_shared(svk::smem_u32(&keys_ready), 0);
+    const uint32_t keys0 = svk::cluster_map_shared(svk::smem_u32(keys_all), 0);
+    const uint32_t ready0 = svk::cluster_map_shared(svk::smem_u32(&keys_ready), 0);
     if (rank == 0 && tid == 0) {
         // what the cluster is about to send: one 16-byte store per four keys of every CTA's slice; the slices are
         // multiples of four blocks long and only the last one in use can be ragged, so that is ceil(nb / 4) stores
@@ -194,11 +142,11 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
                 for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
                 const int bb = b + i;
                 const bool is_forced = bb < p.n_sink || bb >= nb - p.n_local;
-                kk[i] = is_forced ? 0xFFFFFFFFu : order_key(d);
+                kk[i] = is_forced ? kForcedKey : order_key(d);
                 if (p.out_scores && lane == 0 && bb < b1) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = d;
             }
             // rows b .. b+3 are 4 consecutive keys: one 16-byte store into CTA 0 (entries past nb are never read)
-            if (lane == 0 && !keep_all) st_async_cluster_v4(keys0 + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]), ready0);
+            if (lane == 0 && !keep_all) svk::st_async_cluster_v4(keys0 + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]), ready0);
             if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter, b1);
         }
     }
@@ -210,273 +158,14 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
         if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = nb;
         return;
     }
-    if (!mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) {
+    if (!svk::mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) {
         // gave up: mark the list invalid (sv_verify_attn then attends over the draft tokens only and reports it)
         if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = -1;
         return;
     }
 
-    // ---- fast path (up to 2048 blocks = 4 keys per thread, scores not all equal) -----------------------------------
-    // The scores of one (sequence, KV head) are mapped linearly onto 0..65535 (monotone in the score, so the
-    // order is kept; equal codes are possible, equal scores are not split).  One histogram pass over the upper
-    // 8 bits of the code finds the boundary bin: unlike the raw float bits, the codes spread over all 256 bins,
-    // so plain shared-memory atomics rarely collide and the boundary bin holds only a few keys.  Those few are
-    // ranked against one another by their exact keys (ties: smaller block index first), which settles the
-    // selection exactly.  A boundary bin with more than kFastCap keys (outliers stretching the range) falls
-    // through to the general radix select below.
-    // NC = keys per thread (1, 2 or 4); returns true when the selection has been written
-    const auto fast_select = [&](auto nc_tag) -> bool {
-        constexpr int NC = decltype(nc_tag)::value;
-        uint32_t kk[NC], kmin = 0xFFFFFFFFu, kmax = 0u;
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            const int bb = c * kThreads + tid;
-            kk[c] = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
-            if (kk[c] != 0xFFFFFFFFu) kmin = min(kmin, kk[c]), kmax = max(kmax, kk[c]);
-        }
-        kmin = __reduce_min_sync(0xffffffffu, kmin);
-        kmax = __reduce_max_sync(0xffffffffu, kmax);
-        if (lane == 0) {
-            atomicMin(&key_min, kmin);
-            atomicMax(&key_max, kmax);
-        }
-        __syncthreads();
-        kmin = key_min, kmax = key_max;
-        const float xmin = key_score(kmin), xmax = key_score(kmax);
-        const float scale = 65535.f / (xmax - xmin);
-        const uint32_t R = (uint32_t)(N - forced);   // evictable blocks to keep: 0 <= R < number of evictable blocks
-        if (kmin < kmax && scale > 0.f && scale < 3.0e38f) {   // block-uniform
-            uint32_t q[NC];   // 16-bit code of the score; 0x10000 = forced or absent
-#pragma unroll
-            for (int c = 0; c < NC; ++c)
-                q[c] = kk[c] == 0xFFFFFFFFu ? 0x10000u : min(65535u, (uint32_t)((key_score(kk[c]) - xmin) * scale));
-            // level 0: upper byte of the code over all evictable keys; level 1 (only when the boundary bin of
-            // level 0 is too crowded to rank directly): lower byte over the keys of that bin
-            uint32_t bound = 0x100u, need = R, in_bin = 0;   // boundary prefix of the code, keys to keep / present at it
-            int shift = 8;
-            bool settled = R == 0;   // nothing evictable is kept: every code is below the boundary 0x100
-#pragma unroll 1
-            for (int lvl = 0; lvl < 2 && !settled; ++lvl) {
-                shift = 8 - 8 * lvl;
-#pragma unroll
-                for (int c = 0; c < NC; ++c)
-                    if (q[c] < 0x10000u && (lvl == 0 || (q[c] >> 8) == bound))
-                        atomicAdd(&hist[lvl][hist_slot((q[c] >> shift) & 255u)], 1u);
-                __syncthreads();
-                if (warp == 0) {   // lane j owns bins 255-8j .. 248-8j (descending)
-                    uint32_t c8[8], tot = 0;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        c8[i] = hist[lvl][hist_slot(255 - 8 * lane - i)];
-                        tot += c8[i];
-                    }
-                    uint32_t incl = tot;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= o) incl += v;
-                    }
-                    uint32_t above = incl - tot;
-                    if (above < need && need <= incl) {   // exactly one lane
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            if (above < need && need <= above + c8[i]) {
-                                pass_bin[0] = 255 - 8 * lane - i;
-                                pass_bin[1] = need - above;
-                                pass_bin[2] = c8[i];
-                            }
-                            above += c8[i];
-                        }
-                    }
-                }
-                __syncthreads();
-                bound = lvl == 0 ? pass_bin[0] : ((bound << 8) | pass_bin[0]);
-                need = pass_bin[1];
-                in_bin = pass_bin[2];
-                settled = need == in_bin || in_bin <= (uint32_t)kFastCap;
-                if (!settled) __syncthreads();   // block-uniform; pass_bin is rewritten by the next level
-            }
-            if (settled) {   // block-uniform
-                const bool rank_them = need < in_bin;   // otherwise every key at the boundary prefix is kept
-                if (rank_them) {
-                    // the few keys at the boundary: order them exactly, by key, ties by smaller block index
-#pragma unroll
-                    for (int c = 0; c < NC; ++c)
-                        if ((q[c] >> shift) == bound) {
-                            const uint32_t bb = (uint32_t)(c * kThreads + tid);
-                            cand[atomicAdd(&cand_n, 1u)] = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
-                        }
-                    __syncthreads();
-                }
-                bool sel[NC];
-#pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    const uint32_t bb = (uint32_t)(c * kThreads + tid);
-                    const uint32_t pc = q[c] >> shift;   // forced / absent: 0x10000 >> shift is above every boundary
-                    sel[c] = bb < (uint32_t)nb && pc > bound;
-                    if (bb < (uint32_t)nb && pc == bound) {
-                        sel[c] = true;
-                        if (rank_them) {
-                            const unsigned long long mine = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
-                            uint32_t rk = 0;
-#pragma unroll 4
-                            for (uint32_t t = 0; t < in_bin; ++t) rk += cand[t] > mine ? 1u : 0u;
-                            sel[c] = rk < need;
-                        }
-                    }
-                }
-                // ascending compaction
-                uint32_t base = 0;
-#pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    if (c * kThreads < nb) {   // block-uniform
-                        const uint32_t ballot = __ballot_sync(0xffffffffu, sel[c]);
-                        if (lane == 0) warp_sel[warp] = __popc(ballot);
-                        __syncthreads();
-                        uint32_t before = 0, total = 0;
-#pragma unroll
-                        for (int w = 0; w < kWarps; ++w) {
-                            const uint32_t v = warp_sel[w];
-                            if (w < warp) before += v;
-                            total += v;
-                        }
-                        if (sel[c]) out[base + before + __popc(ballot & ((1u << lane) - 1u))] = c * kThreads + tid;
-                        base += total;
-                        if ((c + 1) * kThreads < nb) __syncthreads();   // block-uniform; warp_sel is rewritten by the next round
-                    }
-                }
-                if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
-                return true;
-            }
-            // fall through: the fast path used hist[0] and hist[1]; clear them for the radix passes
-            for (int i = tid; i < 2 * kHistSlots; i += kThreads) (&hist[0][0])[i] = 0;
-            __syncthreads();
-        }
-        return false;
-    };
-    if (nb <= kThreads) {
-        if (fast_select(std::integral_constant<int, 1>{})) return;
-    } else if (nb <= 2 * kThreads) {
-        if (fast_select(std::integral_constant<int, 2>{})) return;
-    } else if (nb <= 4 * kThreads) {
-        if (fast_select(std::integral_constant<int, 4>{})) return;
-    }
-
-    // Exact radix select of the boundary key among the evictable blocks (the forced ones carry 0xFFFFFFFF and
-    // are kept without taking part).  The keys of one (sequence, KV head) share their leading bits (same sign,
-    // neighbouring exponents), so the digits start at the highest bit in which any two keys differ: the first
-    // 8-bit pass then spreads the keys over the bins (shared-memory atomics rarely collide) and usually leaves a
-    // boundary bin of a few keys, so that the second pass ends the search.  Every warp scans the histogram itself
-    // (one block barrier per pass); the passes stop as soon as the boundary bin is taken whole.
-    uint32_t k_and = 0xFFFFFFFFu, k_or = 0u;
-    for (int c0 = 0; c0 < nb; c0 += kThreads) {
-        const int bb = c0 + tid;
-        const uint32_t k = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
-        if (k != 0xFFFFFFFFu) k_and &= k, k_or |= k;
-    }
-    k_and = __reduce_and_sync(0xffffffffu, k_and);
-    k_or = __reduce_or_sync(0xffffffffu, k_or);
-    if (lane == 0) warp_sel[warp] = k_and, warp_eq[warp] = k_or;
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) k_and &= warp_sel[w], k_or |= warp_eq[w];
-    __syncthreads();   // warp_sel / warp_eq are reused by the compaction
-    const uint32_t diff = k_and ^ k_or;
-    uint32_t remaining = (uint32_t)(N - forced);        // evictable blocks to keep (N < nb here, so fewer than there are)
-    int lo = diff ? 32 - __clz(diff) : 0;               // undecided low bits
-    uint32_t mask = lo == 32 ? 0u : ~((1u << lo) - 1u); // bits decided so far: the common leading bits
-    uint32_t prefix = k_and & mask;
-#pragma unroll 1
-    for (int pass = 0; pass < 4 && lo > 0 && remaining > 0; ++pass) {
-        const int width = min(8, lo), shift = lo - width;
-        const uint32_t dmask = (1u << width) - 1u;
-        for (int c0 = 0; c0 < nb; c0 += kThreads) {
-            const int bb = c0 + tid;
-            const uint32_t k = bb < nb ? keys_all[bb] : 0xFFFFFFFFu;
-            const bool cand = k != 0xFFFFFFFFu && (k & mask) == prefix;
-            // one shared-memory atomic per distinct digit per warp: keys of similar magnitude pile onto few bins
-            const uint32_t digit = cand ? ((k >> shift) & dmask) : 256u;
-            const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-            if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[pass][hist_slot(digit)], (uint32_t)__popc(peers));
-        }
-        __syncthreads();
-        // warp 0 scans the histogram (the other warps would only compete for issue slots) and publishes the
-        // boundary bin; lane j owns bins 255-8j .. 248-8j (descending)
-        if (warp == 0) {
-            uint32_t c[8], tot = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                c[i] = hist[pass][hist_slot(255 - 8 * lane - i)];
-                tot += c[i];
-            }
-            uint32_t incl = tot;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            const uint32_t excl = incl - tot;
-            if (excl < remaining && remaining <= incl) {   // exactly one lane
-                uint32_t above = excl;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (above < remaining && remaining <= above + c[i]) {
-                        pass_bin[0] = 255 - 8 * lane - i;
-                        pass_bin[1] = remaining - above;
-                        pass_bin[2] = c[i];
-                    }
-                    above += c[i];
-                }
-            }
-        }
-        __syncthreads();
-        const uint32_t bin = pass_bin[0], rem_in_bin = pass_bin[1], bin_count = pass_bin[2];
-        // (pass_bin is rewritten only after the next pass's barrier)
-        prefix |= bin << shift;
-        mask |= dmask << shift;
-        remaining = rem_in_bin;
-        lo = shift;
-        if (remaining == bin_count) break;   // the whole boundary bin is kept: lower bits cannot matter
-    }
-    // evictable keys whose decided bits exceed the prefix are kept; of those equal to it, the first `remaining`
-    // in index order (all of them after an early stop, none when only the forced blocks fit the budget)
-    const uint32_t thr = prefix;
-    const uint32_t take_eq = remaining;
-
-    // ascending compaction
-    uint32_t base_sel = 0, base_eq = 0;
-    for (int c0 = 0; c0 < nb; c0 += kThreads) {
-        const int bb = c0 + tid;
-        const uint32_t key = bb < nb ? keys_all[bb] : 0u;
-        const bool is_forced = bb < nb && key == 0xFFFFFFFFu;
-        const uint32_t k = key & mask;
-        const bool gt = is_forced || (bb < nb && k > thr);
-        const bool eq = bb < nb && !is_forced && k == thr;
-        const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
-        const uint32_t gt_ballot = __ballot_sync(0xffffffffu, gt);
-        if (lane == 0) {
-            warp_eq[warp] = __popc(eq_ballot);
-            warp_sel[warp] = __popc(gt_ballot);
-        }
-        __syncthreads();
-        uint32_t eq_before = base_eq, eq_total = 0, gt_before = 0, gt_total = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const uint32_t e = warp_eq[w], g = warp_sel[w];
-            if (w < warp) eq_before += e, gt_before += g;
-            eq_total += e, gt_total += g;
-        }
-        // kept ties are the first take_eq in index order
-        const uint32_t lt = (1u << lane) - 1u;
-        const uint32_t eq_rank = eq_before + __popc(eq_ballot & lt);
-        const bool sel = gt || (eq && eq_rank < take_eq);
-        // position = kept entries before this one = greater keys before + kept ties before
-        const uint32_t eq_kept_before = min(eq_rank, take_eq) - min(base_eq, take_eq);   // kept ties before, this chunk
-        if (sel) out[base_sel + gt_before + __popc(gt_ballot & lt) + eq_kept_before] = bb;
-        base_sel += gt_total + min(base_eq + eq_total, take_eq) - min(base_eq, take_eq);
-        base_eq += eq_total;
-        __syncthreads();
-    }
+    svsel::select_top<kThreads>(
+        keys_all, nb, N, forced, scratch, tid, [] { __syncthreads(); }, [&](int pos, int block) { out[pos] = block; });
     if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
 }
 
