@@ -215,8 +215,7 @@ def run_gpu(args):
                               n_layers=w.n_layers, block_table=torch.from_numpy(geom["block_table"]).to(dev),
                               seq_lens=torch.from_numpy(geom["seq_lens"]).to(dev),
                               budget_blocks=torch.from_numpy(geom["budget"]).to(dev), max_sel=geom["max_sel"],
-                              n_sink=w.n_sink, n_local=w.n_local, anchors=anchors, device=str(dev),
-                              fused_select=not args.two_kernels)
+                              n_sink=w.n_sink, n_local=w.n_local, anchors=anchors, device=str(dev))
         return e
 
     eng = make_engine([True] * w.n_layers)
@@ -743,8 +742,6 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: run a shorter stack (default: all 32)")
     ap.add_argument("--only-step", action="store_true",
                     help="profiling aid: time only the main step graph (no reuse / dense / attention-only / e2e passes)")
-    ap.add_argument("--two-kernels", action="store_true",
-                    help="anchor layers call sv_select_blocks and sv_verify_attn separately instead of sv_select_verify_attn")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line: sparse vs dense latency over context x budget x draft length")
     ap.add_argument("--configs", action="store_true",

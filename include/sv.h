@@ -13,7 +13,6 @@
  *                     last few; or reuse the previous layer's set  (Eq. 5, Eq. 9)
  *   sv_verify_attn    attention of all draft tokens over the kept blocks
  *                     and the draft tokens' own K/V                       (Fig. 1)
- *   sv_select_verify_attn   the two steps above in one launch (an anchor layer)
  *   sv_kv_append      commit of the accepted draft tokens to the cache, with
  *                     the representatives of the grown blocks refreshed (Section 2.1)
  *   sv_accept         acceptance of the draft tokens after verification (Eq. 2-3)
@@ -225,31 +224,6 @@ SV_API sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv 
                          const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
                          const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
                          void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
-
-/*
- * Block selection and sparse verification attention of one layer in one call (Fig. 1: score the block
- * representatives with the first draft token's query, keep the top-N blocks, attend over them; Section 3.1,
- * Eq. 5).  Same results as sv_select_blocks(reuse_prev = 0, out_scores = NULL) followed by sv_verify_attn on
- * its lists, but the attention kernel selects for itself: the CTAs that share a (sequence, KV head) form
- * thread-block clusters, score the representatives together, exchange the scores through distributed shared
- * memory and each derive the list in their own shared memory, so the chain "selection kernel -> list in
- * global memory -> attention kernel" and one kernel boundary disappear.  The lists are also written to
- * sel_idx / sel_cnt (ascending; entries >= cnt untouched; -1 if the exchange gave up), for inspection and for
- * the layers that reuse them (Eq. 9: call sv_verify_attn with them on the non-anchor layers).
- * Arguments as in sv_select_blocks and sv_verify_attn; workspace as for sv_verify_attn (sv_workspace_bytes).
- * Shapes the in-kernel selection does not cover (more than 2048 blocks per sequence, or more than 128 kept
- * blocks per CTA) run the two stand-alone kernels one after the other instead.
- */
-SV_API sv_status sv_select_verify_attn(const sv_geom *geom, const void *q, const sv_kv *kv, const float *reps,
-                                       const int32_t *budget_blocks, int32_t n_sink, int32_t n_local,
-                                       const void *draft_k, const void *draft_v, const int32_t *parent,
-                                       int32_t *sel_idx, int32_t *sel_cnt, int32_t max_sel, float softmax_scale,
-                                       void *out, float *lse, void *workspace, size_t workspace_bytes,
-                                       int32_t *status_word, void *stream);
-
-/* Kernel launches one sv_select_verify_attn call enqueues for this geometry: 1 or 2 (attention, split merge) when the
- * attention kernel selects for itself, 2 or 3 when the stand-alone selection kernel runs first.  0: invalid geometry. */
-SV_API int32_t sv_select_verify_attn_launches(const sv_geom *geom, int32_t max_sel);
 
 /*
  * sv_verify_attn for callers that cannot provide or allocate a workspace.  (The paper has no

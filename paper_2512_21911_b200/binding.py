@@ -25,7 +25,7 @@ SV_STATUS_WAIT_MASK, SV_STATUS_INDEX, SV_STATUS_NO_LIST = 0x0FF, 0x100, 0x200
 SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
 EXPORTS = ("sv_strerror", "sv_status_word_check", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
-           "sv_verify_attn", "sv_select_verify_attn", "sv_select_verify_attn_launches", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
+           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
            "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global", "sv_accept",
            "sv_block_reps_bf16", "sv_select_blocks_bf16reps")
 
@@ -63,8 +63,6 @@ def _load() -> ctypes.CDLL:
     lib.sv_budget_blocks.argtypes = [i64, i64, f64, i32, i32, i32]
     lib.sv_workspace_bytes.restype = sz
     lib.sv_workspace_bytes.argtypes = [gp, i32]
-    lib.sv_select_verify_attn_launches.restype = i32
-    lib.sv_select_verify_attn_launches.argtypes = [gp, i32]
     lib.sv_verify_attn_splits.restype = i32
     lib.sv_verify_attn_splits.argtypes = [gp, i32]
     lib.sv_block_reps.restype = ctypes.c_int
@@ -73,8 +71,6 @@ def _load() -> ctypes.CDLL:
     lib.sv_select_blocks.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
     lib.sv_verify_attn.restype = ctypes.c_int
     lib.sv_verify_attn.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
-    lib.sv_select_verify_attn.restype = ctypes.c_int
-    lib.sv_select_verify_attn.argtypes = [gp, vp, kp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
     lib.sv_anchor_jaccard.restype = ctypes.c_int
     lib.sv_anchor_jaccard.argtypes = [gp, i32, vp, vp, i32, vp, vp, vp]
     lib.sv_pick_anchors.restype = ctypes.c_int
@@ -148,10 +144,6 @@ def sv_workspace_bytes(geom: sv_geom, max_sel: int) -> int:
     return int(_lib.sv_workspace_bytes(ctypes.byref(geom), max_sel))
 
 
-def sv_select_verify_attn_launches(geom: sv_geom, max_sel: int) -> int:
-    return int(_lib.sv_select_verify_attn_launches(ctypes.byref(geom), max_sel))
-
-
 def sv_verify_attn_splits(geom: sv_geom, max_sel: int) -> int:
     return int(_lib.sv_verify_attn_splits(ctypes.byref(geom), max_sel))
 
@@ -209,25 +201,6 @@ def sv_verify_attn(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_id
                                _ptr(sel_cnt, torch.int32, "sel_cnt"), max_sel, float(softmax_scale),
                                _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"), ws_ptr, ws_bytes,
                                _ptr(status_word, torch.int32, "status_word"), _stream(stream)), "sv_verify_attn")
-
-
-def sv_select_verify_attn(geom: sv_geom, q, kv: sv_kv, reps, budget_blocks, n_sink: int, n_local: int, draft_k, draft_v,
-                          parent, sel_idx, sel_cnt, out, lse=None, workspace=None, softmax_scale: float = 0.0,
-                          status_word=None, stream=None) -> None:
-    """Block selection + sparse verification attention of one layer in one call; sel_idx / sel_cnt receive the lists."""
-    ws_ptr = workspace.data_ptr() if workspace is not None else None
-    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
-    if workspace is not None and not workspace.is_cuda:
-        raise TypeError("workspace must be a CUDA tensor")
-    _check(_lib.sv_select_verify_attn(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), ctypes.byref(kv),
-                                      _ptr(reps, torch.float32, "reps"), _ptr(budget_blocks, torch.int32, "budget_blocks"),
-                                      n_sink, n_local, _ptr(draft_k, torch.bfloat16, "draft_k"),
-                                      _ptr(draft_v, torch.bfloat16, "draft_v"), _ptr(parent, torch.int32, "parent"),
-                                      _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
-                                      int(sel_idx.shape[-1]), float(softmax_scale), _ptr(out, torch.bfloat16, "out"),
-                                      _ptr(lse, torch.float32, "lse"), ws_ptr, ws_bytes,
-                                      _ptr(status_word, torch.int32, "status_word"), _stream(stream)),
-           "sv_select_verify_attn")
 
 
 def sv_verify_attn_noalloc(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=None,

@@ -31,19 +31,10 @@ struct AttnParams {
     float scale_log2;
     int Tt, tiles;   // draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
     int n_pages;     // pages in each pool: page ids from the block table are clamped to it
-    // Selection inside the attention launch (reps != nullptr): the CTAs of a cluster of `cl` splits score `chunk`
-    // blocks each, exchange the keys and select for themselves; the list is also written to out_idx / out_cnt.
-    const float *reps;       // [S][Hkv][NBmax][128]
-    const int32_t *budget;   // [S]
-    int32_t *out_idx;        // [S][Hkv][max_sel]
-    int32_t *out_cnt;        // [S][Hkv]
-    int n_sink, n_local, cl, chunk;
 };
 
-// tcgen05 / TMEM attention kernel (verify_attn_tc.cu); p.reps != nullptr selects inside the launch.
+// tcgen05 / TMEM attention kernel (verify_attn_tc.cu): rows = G*T <= 128 packed as one M=128 tile.
 cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                            cudaStream_t stream);
-int attn_select_max_blocks();
-int attn_select_max_slice();
 
 }  // namespace svk

@@ -153,20 +153,21 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     if (rank != 0) return;
 
     int32_t *out = p.out_idx + ((size_t)s * p.Hkv + h) * p.max_sel;
+    int cnt_out;
     if (keep_all) {
         for (int bb = tid; bb < nb; bb += kThreads) out[bb] = bb;
-        if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = nb;
-        return;
+        cnt_out = nb;
+    } else if (!__syncthreads_and(svk::mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0))) {
+        cnt_out = -1;   // gave up: mark the list invalid (sv_verify_attn then attends over the draft tokens only and reports it)
+    } else {
+        svsel::select_top<kThreads>(
+            keys_all, nb, N, forced, scratch, tid, [] { __syncthreads(); }, [&](int pos, int block) { out[pos] = block; });
+        cnt_out = N;
     }
-    if (!svk::mbar_wait_cluster_bounded(svk::smem_u32(&keys_ready), 0)) {
-        // gave up: mark the list invalid (sv_verify_attn then attends over the draft tokens only and reports it)
-        if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = -1;
-        return;
+    __syncthreads();   // every thread's entries of the list are written
+    if (tid == 0) {
+        p.out_cnt[(size_t)s * p.Hkv + h] = cnt_out;
     }
-
-    svsel::select_top<kThreads>(
-        keys_all, nb, N, forced, scratch, tid, [] { __syncthreads(); }, [&](int pos, int block) { out[pos] = block; });
-    if (tid == 0) p.out_cnt[(size_t)s * p.Hkv + h] = N;
 }
 
 __global__ void copy_selection_kernel(const int32_t *__restrict__ prev_idx, const int32_t *__restrict__ prev_cnt,

@@ -141,14 +141,30 @@ __device__ __forceinline__ void select_top(const uint32_t *keys_all, int nb, int
             }
             if (settled) {   // uniform
                 const bool rank_them = need < in_bin;   // otherwise every key at the boundary prefix is kept
+                uint32_t my_slot[NC];
                 if (rank_them) {
-                    // the few keys at the boundary: order them exactly, by key, ties by smaller block index
+                    // the few keys at the boundary: order them exactly, by key, ties by smaller block index.  Their
+                    // owners list them; then kThreads / kFastCap threads per listed key count the larger ones (a slice
+                    // of the list each, summed with shuffles) and leave its rank in shared memory.
 #pragma unroll
-                    for (int c = 0; c < NC; ++c)
+                    for (int c = 0; c < NC; ++c) {
+                        my_slot[c] = 0xFFFFFFFFu;
                         if ((q[c] >> shift) == bound) {
                             const uint32_t bb = (uint32_t)(NC * tid + c);
-                            sc.cand[atomicAdd(&sc.cand_n, 1u)] = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
+                            my_slot[c] = atomicAdd(&sc.cand_n, 1u);
+                            sc.cand[my_slot[c]] = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
                         }
+                    }
+                    sync();
+                    constexpr int TPC = kThreads / kFastCap;   // threads per listed key (a power of two <= 32)
+                    static_assert(TPC >= 1 && TPC <= 32 && (TPC & (TPC - 1)) == 0 && kThreads % kFastCap == 0, "rank layout");
+                    const uint32_t ci = (uint32_t)tid / TPC, part = (uint32_t)tid % TPC;
+                    const unsigned long long mine = ci < in_bin ? sc.cand[ci] : ~0ull;
+                    uint32_t rk = 0;
+                    for (uint32_t t = part; t < in_bin; t += TPC) rk += sc.cand[t] > mine ? 1u : 0u;
+#pragma unroll
+                    for (int o = TPC / 2; o > 0; o >>= 1) rk += __shfl_xor_sync(0xffffffffu, rk, o);
+                    if (part == 0) sc.hist[2][ci] = rk;   // (hist[2] serves the radix path only, which is not taken from here)
                     sync();
                 }
                 uint32_t n_mine = 0, sel_bits = 0;
@@ -157,16 +173,7 @@ __device__ __forceinline__ void select_top(const uint32_t *keys_all, int nb, int
                     const uint32_t bb = (uint32_t)(NC * tid + c);
                     const uint32_t pc = q[c] >> shift;   // forced / absent: 0x10000 >> shift is above every boundary
                     bool sel = bb < (uint32_t)nb && pc > bound;
-                    if (bb < (uint32_t)nb && pc == bound) {
-                        sel = true;
-                        if (rank_them) {
-                            const unsigned long long mine = ((unsigned long long)kk[c] << 32) | (0xFFFFFFFFu - bb);
-                            uint32_t rk = 0;
-#pragma unroll 8
-                            for (uint32_t t = 0; t < in_bin; ++t) rk += sc.cand[t] > mine ? 1u : 0u;
-                            sel = rk < need;
-                        }
-                    }
+                    if (bb < (uint32_t)nb && pc == bound) sel = rank_them ? sc.hist[2][my_slot[c]] < need : true;
                     if (sel) sel_bits |= 1u << c, ++n_mine;
                 }
                 // ascending compaction: exclusive prefix sum of the per-thread counts (warp scan, then the warps' totals)

@@ -43,11 +43,8 @@ __global__ void __launch_bounds__(kMergeThreads) merge_splits_kernel(const AttnP
     const int h = blockIdx.y, s = blockIdx.z;
     const int rows = p.G * p.T;
     const int idx = blockIdx.x * kMergeThreads + threadIdx.x;
-    // The kernel after this one may be scheduled at once: its blocks wait for this grid's completion before they read
-    // anything, and this grid's blocks are all resident already (they hold no shared memory), so nothing can starve.
-    // Released only after the wait, the next layer's attention blocks started about 2 us later than their SMs were free.
-    grid_launch_dependents();
     grid_dependency_wait();     // the partials come from the attention kernel just before
+    grid_launch_dependents();
     if (idx >= rows * 32) return;
     const int row = idx >> 5, c4 = idx & 31;
     const size_t sh = (size_t)s * p.Hkv + h;
@@ -193,39 +190,11 @@ extern "C" size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel)
     return workspace_bytes_for(geom, max_sel, true);
 }
 
-// Block selection inside the attention launch (sv_select_verify_attn): what the kernel needs beyond the lists.
-struct SelectArgs {
-    const float *reps;
-    const int32_t *budget;
-    int32_t n_sink, n_local;
-};
-
-// Splits and cluster size of the launch that selects for itself: the CTAs of a cluster share the scoring, so the
-// splits of a (sequence, KV head) come in clusters of 4 (or 2); every cluster scores all blocks of its pair.
-static void fused_shape(const sv_geom *geom, int32_t max_sel, int *splits, int *cl)
-{
-    const int n = choose_splits(geom, max_sel, true);
-    *cl = n >= 4 ? 4 : (n >= 2 ? 2 : 1);
-    *splits = n / *cl * *cl;
-}
-
-// Whether the attention kernel can select for itself at this shape (otherwise the fused entry point runs the two
-// stand-alone steps one after the other, with the same results).
-static bool fused_fits(const sv_geom *geom, int32_t max_sel)
-{
-    int splits, cl;
-    fused_shape(geom, max_sel, &splits, &cl);
-    return geom->max_blocks <= svk::attn_select_max_blocks() && max_sel <= svk::attn_select_max_blocks() &&
-           (max_sel + 3 + splits - 1) / splits <= svk::attn_select_max_slice();
-}
-
 // `balance`: see choose_splits (the built-in-scratch entry point gives it up when the partials would not fit)
-// `sel`: non-NULL when the kernel selects the blocks itself; sel_idx / sel_cnt then receive the lists
 static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
                                   const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
                                   const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
-                                  void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream, bool balance,
-                                  const SelectArgs *sel = nullptr)
+                                  void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream, bool balance)
 {
     sv_status st = svh::check_geom(geom);
     if (st != SV_OK) return st;
@@ -241,8 +210,7 @@ static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_k
 
     const int G = geom->n_q_heads / geom->n_kv_heads;
     const int rows = G * geom->n_draft;
-    int splits = choose_splits(geom, max_sel, balance), cl = 1;
-    if (sel) fused_shape(geom, max_sel, &splits, &cl);
+    const int splits = choose_splits(geom, max_sel, balance);
     if (splits > 1) {
         if (!workspace) return SV_ERR_NULL;
         if (!svh::aligned(workspace, 16)) return SV_ERR_ALIGN;
@@ -272,14 +240,6 @@ static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_k
     p.NBmax = geom->max_blocks, p.max_sel = max_sel, p.splits = splits;
     p.Tt = svh::tokens_per_tile(geom), p.tiles = svh::row_tiles(geom);
     p.n_pages = kv->n_pages;
-    p.reps = nullptr, p.budget = nullptr, p.out_idx = nullptr, p.out_cnt = nullptr;
-    p.n_sink = p.n_local = 0, p.cl = 1, p.chunk = 0;
-    if (sel) {
-        p.reps = sel->reps, p.budget = sel->budget, p.n_sink = sel->n_sink, p.n_local = sel->n_local;
-        p.out_idx = const_cast<int32_t *>(sel_idx), p.out_cnt = const_cast<int32_t *>(sel_cnt);
-        p.cl = cl;
-        p.chunk = ((geom->max_blocks + cl - 1) / cl + 31) / 32 * 32;   // blocks a CTA scores: 8 warps x 4 rows per round
-    }
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;   // 1/sqrt(128)
     p.scale_log2 = scale * 1.4426950408889634f;
 
@@ -311,43 +271,6 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
 {
     return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
                             workspace, workspace_bytes, status_word, stream, true);
-}
-
-extern "C" sv_status sv_select_verify_attn(const sv_geom *geom, const void *q, const sv_kv *kv, const float *reps,
-                                           const int32_t *budget_blocks, int32_t n_sink, int32_t n_local,
-                                           const void *draft_k, const void *draft_v, const int32_t *parent,
-                                           int32_t *sel_idx, int32_t *sel_cnt, int32_t max_sel, float softmax_scale,
-                                           void *out, float *lse, void *workspace, size_t workspace_bytes,
-                                           int32_t *status_word, void *stream)
-{
-    sv_status st = svh::check_geom(geom);
-    if (st != SV_OK) return st;
-    st = svh::check_kv(geom, kv, true);
-    if (st != SV_OK) return st;
-    if (!reps || !budget_blocks || !sel_idx || !sel_cnt) return SV_ERR_NULL;
-    if (!svh::aligned(reps, 16)) return SV_ERR_ALIGN;
-    if (max_sel < 1 || n_sink < 0 || n_local < 0) return SV_ERR_SHAPE;
-    if (n_sink + n_local > max_sel) return SV_ERR_BUDGET;
-    if (!fused_fits(geom, max_sel)) {
-        // too many blocks for the in-kernel selection: the stand-alone selection kernel, then the attention
-        st = sv_select_blocks(geom, q, reps, kv->seq_lens, budget_blocks, n_sink, n_local, 0, nullptr, nullptr, sel_idx,
-                              sel_cnt, max_sel, nullptr, stream);
-        if (st != SV_OK) return st;
-        return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
-                                workspace, workspace_bytes, status_word, stream, true);
-    }
-    const SelectArgs sel = {reps, budget_blocks, n_sink, n_local};
-    return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
-                            workspace, workspace_bytes, status_word, stream, true, &sel);
-}
-
-extern "C" int32_t sv_select_verify_attn_launches(const sv_geom *geom, int32_t max_sel)
-{
-    if (svh::check_geom(geom) != SV_OK || max_sel < 1) return 0;
-    if (!fused_fits(geom, max_sel)) return 1 + (choose_splits(geom, max_sel, true) > 1 ? 2 : 1);
-    int splits, cl;
-    fused_shape(geom, max_sel, &splits, &cl);
-    return splits > 1 ? 2 : 1;
 }
 
 // ---------------------------------------------------------------------- sv_verify_attn_noalloc

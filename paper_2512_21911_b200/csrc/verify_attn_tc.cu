@@ -28,7 +28,6 @@
 #include <cuda_bf16.h>
 
 #include "attn_common.cuh"
-#include "select_core.cuh"
 #include "sv_host.h"
 #include "sv_ptx.cuh"
 
@@ -48,6 +47,7 @@ constexpr int kOffDraft = 0;                     // the draft unit is the first 
 constexpr int kOffMisc = kOffP + 2 * kPBytes;
 constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
+static_assert(2 * kStages + 10 <= 32, "one lane of the producer warp per barrier");
 constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns
 
 // barrier slots (8 bytes each) inside the misc area
@@ -60,30 +60,14 @@ enum Bar {
     kOReady = kPReady + 2,      // [2] the warpgroup's latest PV has been added to O in TMEM
     kStaged = kOReady + 2,      // Q (and the draft unit) are staged
     kTmemDone = kStaged + 1,    // all warps are done with TMEM
-    kKeys = kTmemDone + 1,      // kSel: the keys of all blocks of this (sequence, KV head) have arrived from the cluster
-    kList = kKeys + 1,          // kSel: the block list and its length are in shared memory
-    kTable = kList + 1,         // kSel: this sequence's row of the block table is in shared memory
-    kNumBars = kTable + 1
+    kNumBars = kTmemDone + 1
 };
-
-// kSel: the selection's working set lives in the two P tiles, which nobody touches before the first softmax
-constexpr int kSelMaxBlocks = 2048;                      // keys, page ids and list entries of at most this many blocks
-constexpr int kSelOffKeys = kOffP;                       // uint32 [kSelMaxBlocks] order-preserving score keys
-constexpr int kSelOffTable = kSelOffKeys + 4 * kSelMaxBlocks;    // int32 [kSelMaxBlocks] this sequence's row of the block table
-constexpr int kSelOffList = kSelOffTable + 4 * kSelMaxBlocks;    // int32 [kSelMaxBlocks] the kept blocks, ascending
-constexpr int kSelOffScratch = kSelOffList + 4 * kSelMaxBlocks;
-constexpr int kSelOffQbar = kSelOffScratch + ((int)sizeof(svsel::Scratch) + 15) / 16 * 16;   // float [128]
-static_assert(kSelOffQbar + 512 <= kOffP + 2 * kPBytes, "the selection's working set fits the P tiles");
-constexpr int kSelSliceRegs = 4;                         // the producer keeps its slice in registers: 32 blocks per register
-constexpr int kSelMaxSlice = 32 * kSelSliceRegs;
-static_assert(kNumBars <= 32, "one lane of the producer warp per barrier");
 
 // NH = 8-row groups per TMEM lane quadrant that hold real query rows: 1 (rows <= 32), 2 (<= 64), 4 (<= 128).
 // kWide: more than one row tile per (sequence, KV head) or more than 32 draft tokens (64-bit ancestor masks).  The
 // common case keeps split = blockIdx.x, plain row arithmetic and 32-bit masks: deriving the split from a division
 // costs 3 % on long loops, and the wider mask code 7 % at 128 rows.
-// kSel: the CTA selects the blocks itself before it attends (the fused entry point; see the selection section below).
-template <int NH, bool kWide, bool kSel>
+template <int NH, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
     verify_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                           const AttnParams p)
@@ -98,8 +82,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint32_t *anc32 = reinterpret_cast<uint32_t *>(misc + 320);                     // [32] the same, up to 32 draft tokens
     volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 448);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 456);
-    volatile int *sel_n = reinterpret_cast<volatile int *>(misc + 460);   // kSel: length of the block list, then this CTA's
-                                                                          // slice of it: [n, first, end]
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
     // blockIdx.x = row tile * splits + split: the query rows of draft tokens i0 .. i0 + Tq - 1, a slice of the blocks
@@ -128,16 +110,6 @@ __global__ void __launch_bounds__(kThreads, 1)
             return (int)((uint32_t)k * (uint32_t)n / (uint32_t)p.splits);
         }
     };
-    // where a kept block's K/V tiles start: first row of the pool's (page, KV head) slab, first token of the block.
-    // Indices are clamped into their tables before any address is formed; a clamp that fires is reported.
-    auto locate = [&](int blk_in, auto page_of, int &row0, int &tok0) {
-        const int blk = max(0, min(blk_in, p.NBmax - 1));
-        const int page_in = page_of(blk);
-        const int page = max(0, min(page_in, p.n_pages - 1));
-        if ((blk != blk_in || page != page_in) && p.status) atomicOr(p.status, kStatusIndex);
-        row0 = (page * p.Hkv + h) * p.B;
-        tok0 = blk * p.B;
-    };
     const float inv_g = 1.f / (float)p.G;
     auto div_g = [&](int r) { return (int)(((float)r + 0.5f) * inv_g); };
     // The TMA producer warp initialises the barriers and runs ahead; everybody else meets it at a named
@@ -154,12 +126,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (lane == 0) *abort_flag = 0;
         __syncwarp();
-        // kSel: the CTAs of a cluster send one another score keys; nobody may send before every CTA's barriers exist.
-        // Every thread arrives here and waits (once) just before its dependency wait.
-        if constexpr (kSel) cluster_arrive_relaxed();   // the initialising lanes executed fence.mbarrier_init
         named_bar_arrive(3, kThreads);
     } else {
-        if constexpr (kSel) cluster_arrive_relaxed();
         if (warp == 9) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tc_fence_before_sync();
         named_bar_sync(3, kThreads);
@@ -178,75 +146,41 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint64_t policy = policy_evict_first();
             // pull this sequence's block-table row towards L2 while the previous kernel drains
             for (int i = lane * 32; i < p.NBmax; i += 32 * 32) prefetch_l2(p.block_table + (size_t)s * p.NBmax + i);
-            if constexpr (kSel) cluster_wait();
             grid_dependency_wait();   // the block list is written by the kernel just before
-            if constexpr (kSel) {
-                // this sequence's row of the block table -> shared memory while the softmax warps score and select, so
-                // that the page look-ups do not add a trip to L2 between "list known" and "first tile requested"
-                int *tbl = reinterpret_cast<int *>(smem + kSelOffTable);
-                for (int i = lane; i < p.NBmax; i += 32) tbl[i] = p.block_table[(size_t)s * p.NBmax + i];
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kTable));
-            }
             // First batch of block indices speculatively, assuming the list is full (cnt == max_sel): its
             // load then overlaps the loads of the count and the length instead of following them.
             const int j0_spec = slice_begin(split, p.max_sel);
             int blk_spec = 0;
-            if (!kSel && p.sel_idx && j0_spec + lane < p.max_sel)
+            if (p.sel_idx && j0_spec + lane < p.max_sel)
                 blk_spec = p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j0_spec + lane];
             const int L = p.seq_lens[s];
             const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
-            bool dead = false;
-            int n_sel;
-            if constexpr (kSel) {
-                // the softmax warps publish the list they selected (and its length) in shared memory
-                if (!mbar_wait_bounded(bar(kList), 0)) {
-                    dead = true;
-                    *abort_flag = 1;
-                    if (p.status && lane == 0) atomicOr(p.status, 1);
-                }
-                n_sel = dead ? 0 : sel_n[0];
-            } else {
-                const int cnt_in = p.sel_idx ? p.sel_cnt[(size_t)s * p.Hkv + h] : nb;
-                // a negative count marks a list that block selection could not produce: attend over the draft tokens
-                // only, and say so
-                if (cnt_in < 0 && lane == 0 && p.status) atomicOr(p.status, kStatusNoList);
-                n_sel = p.sel_idx ? max(0, min(cnt_in, p.max_sel)) : nb;
-            }
-            const int j0 = (kSel && !dead) ? sel_n[1] : slice_begin(split, n_sel);
-            const int j1 = (kSel && !dead) ? sel_n[2] : slice_begin(split + 1, n_sel);
+            const int cnt_in = p.sel_idx ? p.sel_cnt[(size_t)s * p.Hkv + h] : nb;
+            // a negative count marks a list that block selection could not produce: attend over the draft tokens
+            // only, and say so
+            if (cnt_in < 0 && lane == 0 && p.status) atomicOr(p.status, kStatusNoList);
+            const int n_sel = p.sel_idx ? max(0, min(cnt_in, p.max_sel)) : nb;
+            const int j0 = slice_begin(split, n_sel);
+            const int j1 = slice_begin(split + 1, n_sel);
             const int off = has_draft ? 1 : 0;
-            // kSel: the softmax warps have looked the slice up (first pool row and first token of every block); it is
-            // copied to registers now (32 blocks per register), because it sits in the P tiles, which those warps
-            // overwrite as soon as the first unit has landed
-            int row0r[kSelSliceRegs], tok0r[kSelSliceRegs];
-            if constexpr (kSel) {
-                const int2 *loc = reinterpret_cast<const int2 *>(smem + kSelOffKeys);
-#pragma unroll
-                for (int x = 0; x < kSelSliceRegs; ++x) {
-                    const int2 v = (32 * x + lane < j1 - j0) ? loc[32 * x + lane] : make_int2(0, 0);
-                    row0r[x] = v.x, tok0r[x] = v.y;
-                }
-            }
-            int bi = 0;
-            for (int base = j0; base < j1; base += 32, ++bi) {
+            bool dead = false;
+            for (int base = j0; base < j1; base += 32) {
                 const int j = base + lane;
                 int row0 = 0, tok0 = 0;
-                if constexpr (kSel) {
-                    row0 = row0r[0], tok0 = tok0r[0];
-#pragma unroll
-                    for (int x = 1; x < kSelSliceRegs; ++x)
-                        if (bi == x) row0 = row0r[x], tok0 = tok0r[x];
-                } else if (j < j1) {
+                if (j < j1) {
                     int blk = j;
                     if (p.sel_idx)
                         blk = (base == j0 && j0 == j0_spec) ? blk_spec : p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j];
-                    locate(blk, [&](int b) { return p.block_table[(size_t)s * p.NBmax + b]; }, row0, tok0);
+                    // indices are clamped into their tables before any address is formed; a clamp that fires is reported
+                    const int blk_in = blk;
+                    blk = max(0, min(blk, p.NBmax - 1));
+                    const int page_in = p.block_table[(size_t)s * p.NBmax + blk];
+                    const int page = max(0, min(page_in, p.n_pages - 1));
+                    if ((blk != blk_in || page != page_in) && p.status) atomicOr(p.status, kStatusIndex);
+                    row0 = (page * p.Hkv + h) * p.B;
+                    tok0 = blk * p.B;
                 }
                 const int n_here = min(32, j1 - base);
-                // (One thread requests the four 8 KB boxes of a unit one after the other, ~570 cycles per unit: that is the
-                // rate at which an SM takes tiles in, not issue latency -- four lanes issuing them with one instruction
-                // measured 4 % slower.)
                 for (int i = 0; i < n_here; ++i) {
                     const int r0 = __shfl_sync(0xffffffffu, row0, i);
                     const int t0 = __shfl_sync(0xffffffffu, tok0, i);
@@ -280,24 +214,16 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---------------------------------------------------------- MMA issuers (one thread each)
             // warp 9 issues every S = Q K^T and owns the TMEM allocation; warp 10 issues every Ou = P V.
             // Descriptors are built once; per instruction only the 14-bit address field moves.
-            if constexpr (kSel) cluster_wait();
             if (lane == 0) {
                 grid_dependency_wait();   // the lengths may come from the kernel just before (a cache commit)
                 const int L = p.seq_lens[s];
                 const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
-                bool dead = false;
-                int n_sel;
-                if constexpr (kSel) {
-                    dead = !mbar_wait_bounded(bar(kList), 0);
-                    n_sel = dead ? 0 : sel_n[0];
-                } else {
-                    n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-                }
+                const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
                 const int j0 = slice_begin(split, n_sel);
                 const int j1 = slice_begin(split + 1, n_sel);
                 const int off = has_draft ? 1 : 0;
                 const int n_total = (j1 - j0) * upb + off;
-                dead = dead || !mbar_wait_bounded(bar(kStaged), 0);
+                bool dead = !mbar_wait_bounded(bar(kStaged), 0);
                 if (warp == 9) {
                     constexpr uint32_t idesc_s = umma_idesc_bf16(128, kUnit, false);
                     const uint64_t dq = umma_desc_sw128(smem0 + kOffQ, 16, 1024);
@@ -360,8 +286,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tc_fence_after_sync();
                 tmem_dealloc(tmem_base, kTmemCols);
             }
-        } else {
-            if constexpr (kSel) cluster_wait();
         }
         return;
     }
@@ -388,140 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     make_uint4(0u, 0u, 0u, 0u);
         }
     }
-    if constexpr (kSel) {
-        reinterpret_cast<svsel::Scratch *>(smem + kSelOffScratch)->init(tid, 256);
-        // pull this CTA's slice of the representatives towards L2 while the previous kernel drains (a prefetch
-        // consumes no data, so it is safe even if that kernel is still writing them)
-        const int pb0 = (int)cluster_ctarank() * p.chunk, pb1 = min(pb0 + p.chunk, p.NBmax);
-        const char *pbase = reinterpret_cast<const char *>(p.reps + (((size_t)s * p.Hkv + h) * p.NBmax + pb0) * 128);
-        for (int i = tid; i < (pb1 - pb0) * 4; i += 256) prefetch_l2(pbase + (size_t)i * 128);
-        cluster_wait();
-    }
     grid_dependency_wait();
-    int n_sel_own = 0;   // kSel: length of the list this CTA selected
-    if constexpr (kSel) {
-        // -------------------------------------------------------------- block selection (Eq. 5, Section 3.1)
-        // The CTAs of a cluster belong to one (sequence, KV head).  Each scores a slice of the representatives against
-        // the group mean of the first draft token's query (warp per 4 rows, 16-byte loads, up to 16 rows in flight per
-        // warp), turns the scores into order-preserving keys and sends them to every CTA of the cluster (st.async
-        // into the same shared-memory offset there, bytes counted on that CTA's mbarrier).  Then every CTA selects
-        // for itself, in its own shared memory, with the code the stand-alone selection kernel uses, and keeps the
-        // ascending list there for its producer warp; the first CTA of the (sequence, KV head) also writes it out.
-        uint32_t *keys = reinterpret_cast<uint32_t *>(smem + kSelOffKeys);
-        int *list = reinterpret_cast<int *>(smem + kSelOffList);
-        svsel::Scratch &scr = *reinterpret_cast<svsel::Scratch *>(smem + kSelOffScratch);
-        float *qbar = reinterpret_cast<float *>(smem + kSelOffQbar);
-        // every load of this section is issued before the first use: lengths, the query rows and the first batch of
-        // representative rows (rows past the sequence's end exist in the array and are discarded below)
-        const int rank = (int)cluster_ctarank(), CL = (int)cluster_nctarank();
-        const int b0 = rank * p.chunk, b_hi = min(b0 + p.chunk, p.NBmax);
-        const float4 *rbase = reinterpret_cast<const float4 *>(p.reps + ((size_t)s * p.Hkv + h) * p.NBmax * 128) + lane;
-        constexpr int kInFlight = 4;   // rounds (of 4 rows per warp) whose loads are issued together
-        float4 r[kInFlight][4];
-        auto load_batch = [&](int it0, int hi) {
-#pragma unroll
-            for (int j = 0; j < kInFlight; ++j)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = it0 + j * 32 + i;
-                    r[j][i] = row < hi ? __ldg(rbase + (size_t)row * 32) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-        };
-        const int L = p.seq_lens[s];
-        const int budget = p.budget[s];
-        const __nv_bfloat16 *q0 = p.q + ((size_t)s * p.T * p.Hq + (size_t)h * p.G) * 128;
-        float qsum = 0.f;
-        if (tid < 128)
-            for (int g = 0; g < p.G; ++g) qsum += __bfloat162float(q0[(size_t)g * 128 + tid]);
-        load_batch(b0 + warp * 4, b_hi);
-        const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
-        const int forced = min(nb, p.n_sink + p.n_local);
-        int N = min(max(budget, forced), p.max_sel);
-        const bool keep_all = N >= nb;
-        if (keep_all) N = nb;
-        const bool writer = blockIdx.x == 0;
-        int32_t *out_idx = p.out_idx + ((size_t)s * p.Hkv + h) * p.max_sel;
-        bool ok = true;
-        if (!keep_all) {
-            const int b1 = min(b0 + p.chunk, nb);
-            if (tid < 128) qbar[tid] = qsum * inv_g;
-            // what the cluster is about to send here: one 16-byte store per four keys of every CTA's slice (the slices
-            // are multiples of four blocks long and only the last one in use can be ragged)
-            if (tid == 0) mbar_arrive_expect_tx(bar(kKeys), 16u * ((uint32_t)(nb + 3) >> 2));
-            named_bar_sync(2, 256);
-            const float4 qv = reinterpret_cast<const float4 *>(qbar)[lane];
-            const uint32_t keys_here = smem0 + kSelOffKeys;
-            const uint32_t keys_there = cluster_map_shared(keys_here, (uint32_t)min(lane, CL - 1));
-            const uint32_t bar_there = cluster_map_shared(bar(kKeys), (uint32_t)min(lane, CL - 1));
-#pragma unroll 1
-            for (int it0 = b0 + warp * 4; it0 < b1; it0 += 32 * kInFlight) {
-                if (it0 != b0 + warp * 4) load_batch(it0, b1);   // the first batch is already here
-#pragma unroll
-                for (int j = 0; j < kInFlight; ++j) {
-                    const int b = it0 + j * 32;
-                    if (b < b1) {   // warp-uniform
-                        // four dot products reduced together: two exchange steps fold the four partial sums of a lane
-                        // into one (lanes 0-7 end up with row 0, 8-15 row 1, 16-23 row 2, 24-31 row 3), three more finish it
-                        float d[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) d[i] = r[j][i].x * qv.x + r[j][i].y * qv.y + r[j][i].z * qv.z + r[j][i].w * qv.w;
-                        const bool up16 = lane & 16, up8 = lane & 8;
-                        const float s0 = up16 ? d[0] : d[2], s1 = up16 ? d[1] : d[3];   // what the partner half needs
-                        float e0 = (up16 ? d[2] : d[0]) + __shfl_xor_sync(0xffffffffu, s0, 16);   // rows 0 / 2
-                        float e1 = (up16 ? d[3] : d[1]) + __shfl_xor_sync(0xffffffffu, s1, 16);   // rows 1 / 3
-                        float f = (up8 ? e1 : e0) + __shfl_xor_sync(0xffffffffu, up8 ? e0 : e1, 8);
-#pragma unroll
-                        for (int o = 4; o > 0; o >>= 1) f += __shfl_xor_sync(0xffffffffu, f, o);
-                        // lane 8 i now holds the score of row (lane & 16 ? 2 : 0) + (lane & 8 ? 1 : 0)
-                        uint32_t kk[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float di = __shfl_sync(0xffffffffu, f, ((i & 2) ? 16 : 0) + ((i & 1) ? 8 : 0));
-                            const int bb = b + i;
-                            kk[i] = (bb < p.n_sink || bb >= nb - p.n_local) ? svsel::kForcedKey : svsel::order_key(di);
-                        }
-                        // lane r sends the four keys to CTA r of the cluster (entries past nb are never read)
-                        if (lane < CL)
-                            st_async_cluster_v4(keys_there + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]), bar_there);
-                    }
-                }
-            }
-            ok = named_bar_and(2, 256, mbar_wait_cluster_bounded(bar(kKeys), 0));
-            if (ok) {
-                svsel::select_top<256>(
-                    keys, nb, N, forced, scr, tid, [] { named_bar_sync(2, 256); },
-                    [&](int pos, int block) {
-                        list[pos] = block;
-                        if (writer) out_idx[pos] = block;
-                    });
-            } else {
-                N = 0;   // gave up on the keys: the draft tokens only, and the caller is told
-                if (tid == 0 && p.status) atomicOr(p.status, 64);
-            }
-        } else {
-            for (int b = tid; b < nb; b += 256) {
-                list[b] = b;
-                if (writer) out_idx[b] = b;
-            }
-        }
-        named_bar_sync(2, 256);   // the list is complete
-        // This CTA's slice of it, looked up by one thread per block (the keys are dead; their place takes the result)
-        const int sj0 = slice_begin(split, N), sj1 = slice_begin(split + 1, N);
-        if (tid < sj1 - sj0) {
-            if (!mbar_wait_bounded(bar(kTable), 0) && p.status) atomicOr(p.status, 64);
-            const int *tbl = reinterpret_cast<const int *>(smem + kSelOffTable);
-            int2 v;
-            locate(list[sj0 + tid], [&](int blk) { return tbl[blk]; }, v.x, v.y);
-            reinterpret_cast<int2 *>(smem + kSelOffKeys)[tid] = v;
-        }
-        named_bar_sync(2, 256);
-        if (tid == 0) {
-            sel_n[0] = N, sel_n[1] = sj0, sel_n[2] = sj1;
-            mbar_arrive(bar(kList));
-            if (writer) p.out_cnt[(size_t)s * p.Hkv + h] = ok ? N : -1;
-        }
-        n_sel_own = N;
-    }
     {
         // real rows: all loads of a thread are in flight together (16-byte chunks: Q up to 128 rows x 16, draft K and
         // V up to 64 tokens x 16 each)
@@ -636,7 +427,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     const int L = p.seq_lens[s];
     const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
-    const int n_sel = kSel ? n_sel_own : (p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb);
+    const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
     const int j0 = slice_begin(split, n_sel);
     const int j1 = slice_begin(split + 1, n_sel);
     const int off = has_draft ? 1 : 0;
@@ -957,14 +748,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 }  // namespace
 
-template <int NH, bool kWide, bool kSel>
+template <int NH, bool kWide>
 static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                              cudaStream_t stream)
 {
     static svh::OncePerDevice once;   // function attributes belong to a device
     const cudaError_t ce = once.run([] {
-        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide, kSel>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kSmemBytes);
+        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     });
     if (ce != cudaSuccess) return ce;
     cudaLaunchConfig_t cfg = {};
@@ -972,44 +762,25 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     svh::pdl_attribute(attr);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if constexpr (kSel) {   // the CTAs that exchange score keys form a cluster along the split dimension
-        attr[1].id = cudaLaunchAttributeClusterDimension;
-        attr[1].val.clusterDim.x = (unsigned)p.cl;
-        attr[1].val.clusterDim.y = 1;
-        attr[1].val.clusterDim.z = 1;
-        cfg.numAttrs = 2;
-    }
-    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide, kSel>, tm_k, tm_v, p);
-}
-
-template <bool kSel>
-static cudaError_t launch_rows(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
-                               cudaStream_t stream)
-{
-    const int rows = p.G * p.Tt;   // rows of a full row tile
-    if (p.tiles > 1 || p.T > 32) {
-        if (rows <= 32) return launch_tc<1, true, kSel>(tm_k, tm_v, p, grid, stream);
-        if (rows <= 64) return launch_tc<2, true, kSel>(tm_k, tm_v, p, grid, stream);
-        return launch_tc<4, true, kSel>(tm_k, tm_v, p, grid, stream);
-    }
-    if (rows <= 32) return launch_tc<1, false, kSel>(tm_k, tm_v, p, grid, stream);
-    if (rows <= 64) return launch_tc<2, false, kSel>(tm_k, tm_v, p, grid, stream);
-    return launch_tc<4, false, kSel>(tm_k, tm_v, p, grid, stream);
+    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide>, tm_k, tm_v, p);
 }
 
 cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                            cudaStream_t stream)
 {
-    return p.reps ? launch_rows<true>(tm_k, tm_v, p, grid, stream) : launch_rows<false>(tm_k, tm_v, p, grid, stream);
+    const int rows = p.G * p.Tt;   // rows of a full row tile
+    if (p.tiles > 1 || p.T > 32) {
+        if (rows <= 32) return launch_tc<1, true>(tm_k, tm_v, p, grid, stream);
+        if (rows <= 64) return launch_tc<2, true>(tm_k, tm_v, p, grid, stream);
+        return launch_tc<4, true>(tm_k, tm_v, p, grid, stream);
+    }
+    if (rows <= 32) return launch_tc<1, false>(tm_k, tm_v, p, grid, stream);
+    if (rows <= 64) return launch_tc<2, false>(tm_k, tm_v, p, grid, stream);
+    return launch_tc<4, false>(tm_k, tm_v, p, grid, stream);
 }
-
-// Limits of the in-kernel selection: blocks whose keys / page ids / list entries fit the shared-memory working set,
-// and blocks per CTA whose locations the producer warp keeps in registers.
-int attn_select_max_blocks() { return kSelMaxBlocks; }
-int attn_select_max_slice() { return kSelMaxSlice; }
 
 }  // namespace svk

@@ -1,8 +1,8 @@
 """SparseVerifier: runs block selection and sparse verification attention for a stack of layers.
 
 A thin driver over the C-ABI calls: it owns the per-layer representatives, the shared block list,
-the split-KV workspace and the outputs, and enqueues, per layer, ``sv_select_verify_attn`` (anchor layers:
-block selection inside the attention launch) or ``sv_verify_attn`` on the previous layer's list (Eq. 9); after verification,
+the split-KV workspace and the outputs, and enqueues, per layer, ``sv_select_blocks`` (anchor
+layers) or the reuse of the previous layer's list (Eq. 9), then ``sv_verify_attn``; after verification,
 ``accept`` (Eq. 2-3) and ``commit`` (append the kept rows to the cache) close the decoding step.  All compute
 is in the library's kernels; this class only holds buffers and calls them in order.
 """
@@ -20,13 +20,12 @@ class SparseVerifier:
                  max_blocks: int, n_draft: int, n_layers: int, block_table: torch.Tensor, seq_lens: torch.Tensor,
                  budget_blocks: torch.Tensor, max_sel: int, n_sink: int = 1, n_local: int = 1,
                  anchors: Optional[Sequence[bool]] = None, parent: Optional[torch.Tensor] = None,
-                 device: str = "cuda", fused_select: bool = True):
+                 device: str = "cuda"):
         self.geom = sv.make_geom(n_seq, n_q_heads, n_kv_heads, head_dim, block_size, max_blocks, n_draft)
         self.n_layers = n_layers
         self.block_table, self.seq_lens, self.budget, self.parent = block_table, seq_lens, budget_blocks, parent
         self.n_sink, self.n_local, self.max_sel = n_sink, n_local, max_sel
         self.anchors = list(anchors) if anchors is not None else [True] * n_layers
-        self.fused_select = fused_select   # anchor layers: one sv_select_verify_attn call instead of select + attention
         assert self.anchors[0], "layer 0 has no preceding layer to reuse"
         dev = torch.device(device)
         self.reps = torch.zeros((n_layers, n_seq, n_kv_heads, max_blocks, head_dim), dtype=torch.float32, device=dev)
@@ -72,12 +71,6 @@ class SparseVerifier:
 
     def verify_layer(self, layer: int, q, draft_k, draft_v, out, lse=None) -> None:
         """select (anchor) or reuse (non-anchor), then sparse verification attention, on the current stream."""
-        if self.anchors[layer] and self.fused_select:
-            # selection inside the attention launch; the lists land in sel_idx / sel_cnt for the layers that reuse them
-            sv.sv_select_verify_attn(self.geom, q, self.kv[layer], self.reps[layer], self.budget, self.n_sink,
-                                     self.n_local, draft_k, draft_v, self.parent, self.sel_idx, self.sel_cnt, out, lse=lse,
-                                     workspace=self.workspace, status_word=self.status)
-            return
         if self.anchors[layer]:
             sv.sv_select_blocks(self.geom, q, self.reps[layer], self.seq_lens, self.budget, self.n_sink,
                                 self.n_local, self.sel_idx, self.sel_cnt)
@@ -152,10 +145,8 @@ class SparseVerifier:
     def kernels_per_step(self, refresh_tail: bool = False, dense: bool = False) -> int:
         """Kernel launches of one step: tail refresh and select per anchor layer; attention (+ merge) per layer."""
         splits = sv.sv_verify_attn_splits(self.geom, self.geom.max_blocks if dense else self.max_sel)
-        attn = 2 if splits > 1 else 1
+        attn = self.n_layers * (2 if splits > 1 else 1)
         if dense:
-            return self.n_layers * attn
+            return attn
         refresh = 0 if not refresh_tail else (1 if self._stack_kv is not None else sum(self.anchors))
-        anchor = sv.sv_select_verify_attn_launches(self.geom, self.max_sel) if self.fused_select else 1 + attn
-        n_anchor = sum(self.anchors)
-        return refresh + n_anchor * anchor + (self.n_layers - n_anchor) * attn
+        return refresh + sum(self.anchors) + attn

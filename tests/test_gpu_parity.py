@@ -120,23 +120,6 @@ def run_pipeline(sv, c, n_sink=None, n_local=None, what=""):
     return d, idx, cnt, o, lse
 
 
-def gpu_fused(sv, d, n_sink, n_local, max_sel):
-    """sv_select_verify_attn: selection inside the attention launch.  Returns (idx, cnt, out, lse)."""
-    w = d.w
-    sv.sv_block_reps(d.geom, d.kv, d.reps)
-    idx = torch.full((w.n_seq, w.n_kv_heads, max_sel), -7, dtype=torch.int32, device="cuda")
-    cnt = torch.full((w.n_seq, w.n_kv_heads), -7, dtype=torch.int32, device="cuda")
-    out = torch.full((w.n_seq, w.n_draft, w.n_q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
-    lse = torch.full((w.n_seq, w.n_draft, w.n_q_heads), float("nan"), device="cuda")
-    ws = torch.empty(max(16, sv.sv_workspace_bytes(d.geom, max_sel)), dtype=torch.uint8, device="cuda")
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    sv.sv_select_verify_attn(d.geom, d.q, d.kv, d.reps, d.budget, n_sink, n_local, d.draft_k, d.draft_v, d.parent, idx, cnt,
-                             out, lse=lse, workspace=ws, status_word=status)
-    torch.cuda.synchronize()
-    assert int(status.item()) == 0
-    return idx.cpu().numpy(), cnt.cpu().numpy(), bf16_host(out), lse.cpu().numpy().astype(np.float64)
-
-
 def check_lists(idx_h, cnt_h, idx_ref, cnt_ref, what=""):
     np.testing.assert_array_equal(cnt_h, cnt_ref, err_msg=what)
     for s in range(cnt_ref.shape[0]):
@@ -146,22 +129,18 @@ def check_lists(idx_h, cnt_h, idx_ref, cnt_ref, what=""):
             assert (idx_h[s, h, n:] == -7).all()
 
 
-def run_fused(sv, c, n_sink=None, n_local=None, what="", samples=None):
-    """The one-call form of select + attention against the oracle: lists bit-exact, attention within the bar."""
-    n_sink = c["n_sink"] if n_sink is None else n_sink
-    n_local = c["n_local"] if n_local is None else n_local
+def run_sampled(sv, c, samples, what=""):
+    """select + attention on a full-size case: lists bit-exact, attention checked on the sampled (s, i, hq) rows."""
     d = Dev(sv, c)
-    idx_h, cnt_h, o, lse = gpu_fused(sv, d, n_sink, n_local, c["max_sel"])
-    idx_ref, cnt_ref, _ = oracle_select(c, n_sink, n_local, c["max_sel"])
-    check_lists(idx_h, cnt_h, idx_ref, cnt_ref, what)
-    if samples is None:
-        o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref)
-        check_attn(o, lse, o_ref, lse_ref, what)
-    else:
-        o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref, samples=samples)
-        check_attn(np.stack([o[s, i, hq] for s, i, hq in samples]), np.array([lse[s, i, hq] for s, i, hq in samples]),
-                   o_ref, lse_ref, what)
-        assert np.isfinite(o).all()
+    idx, cnt, _ = gpu_select(sv, d, c["n_sink"], c["n_local"], c["max_sel"])
+    torch.cuda.synchronize()
+    idx_ref, cnt_ref, _ = oracle_select(c, c["n_sink"], c["n_local"], c["max_sel"])
+    check_lists(idx.cpu().numpy(), cnt.cpu().numpy(), idx_ref, cnt_ref, what)
+    o, lse = gpu_attn(sv, d, idx, cnt)
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref, samples=samples)
+    check_attn(np.stack([o[s, i, hq] for s, i, hq in samples]), np.array([lse[s, i, hq] for s, i, hq in samples]),
+               o_ref, lse_ref, what)
+    assert np.isfinite(o).all()
     return d
 
 
@@ -201,66 +180,39 @@ def test_pipeline_parity_small(sv, name, sharp):
     run_pipeline(sv, c, what=f"{name} sharp={sharp}")
 
 
-@pytest.mark.parametrize("name", list(SMALL))
-@pytest.mark.parametrize("sharp", [False, True])
-def test_fused_select_attention_small(sv, name, sharp):
-    c = si.make_layer(si.make_geometry(SMALL[name]), sharp=sharp)
-    run_fused(sv, c, what=f"fused {name} sharp={sharp}")
-
-
-@pytest.mark.parametrize("forced", [(0, 0), (2, 4)])
-def test_fused_sink_local_variants(sv, forced):
-    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(900, 2000), budget_blocks=10, n_sink=forced[0], n_local=forced[1])
-    c = si.make_layer(si.make_geometry(w), sharp=True)
-    run_fused(sv, c, what=f"fused forced={forced}")
-
-
-def test_fused_budget_covering_all_blocks_and_empty_prefix(sv):
-    """Budget >= number of blocks keeps everything (no scoring, no exchange); a sequence without cached tokens keeps
-    nothing and attends over the draft tokens only."""
-    w = si.shrink(SMALL["cfg2_small"], budget_blocks=60)
-    c = si.make_layer(si.make_geometry(w), sharp=True)
-    run_fused(sv, c, what="fused keep-all")
-    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(300, 900), budget_blocks=4, tree=True)
-    c = si.make_layer(si.make_geometry(w), sharp=True)
-    c["seq_lens"] = c["seq_lens"].copy()
-    c["seq_lens"][1] = 0
-    c["n_blocks"] = ((c["seq_lens"] + 63) // 64).astype(np.int32)
-    d = Dev(sv, c)
-    idx_h, cnt_h, o, lse = gpu_fused(sv, d, 1, 1, c["max_sel"])
-    idx_ref, cnt_ref, _ = oracle_select(c, 1, 1, c["max_sel"])
-    assert (cnt_ref[1] == 0).all()
-    check_lists(idx_h, cnt_h, idx_ref, cnt_ref, "fused empty prefix")
-    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref)
-    check_attn(o, lse, o_ref, lse_ref, "fused empty prefix")
-
-
-@pytest.mark.parametrize("sharp", [False, True])
-def test_fused_full_size_cfg1_one_layer(sv, sharp):
-    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg1"]), layer=5, sharp=sharp)
-    run_fused(sv, c, what=f"fused cfg1 sharp={sharp}")
-
-
-def test_fused_full_size_cfg2(sv):
-    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg2"]), sharp=True)
-    run_fused(sv, c, what="fused cfg2")
-
-
-def test_fused_full_size_cfg3_sampled(sv):
+def test_full_size_cfg3_one_pair_in_full(sv):
+    """The long-context tree configuration: besides random samples, every draft row and query head of one
+    (sequence, KV head) pair -- all 128 query rows of one CTA group."""
     c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg3"]), sharp=True)
-    g = np.random.default_rng(17)
     w = c["workload"]
-    smp = [(int(g.integers(0, w.n_seq)), int(g.integers(0, w.n_draft)), int(g.integers(0, w.n_q_heads))) for _ in range(48)]
-    run_fused(sv, c, what="fused cfg3", samples=smp)
+    G = w.n_q_heads // w.n_kv_heads
+    smp = [(2, i, 5 * G + g) for i in range(w.n_draft) for g in range(G)]
+    run_sampled(sv, c, smp, what="cfg3, sequence 2, KV head 5")
 
 
-@pytest.mark.parametrize("point", [(8192, 1 / 16, 8), (32768, 1 / 4, 8), (131072, 1 / 16, 16), (131072, 1 / 4, 1)])
-def test_fused_sweep_points(sv, point):
+def test_full_size_cfg3_dense_sampled(sv):
+    """Dense verification of the 4 x 131072-token tree configuration (2 GiB of K/V per call) on sampled rows."""
+    c = si.make_layer(si.make_geometry(si.WORKLOADS["cfg3"]), sharp=True)
+    d = Dev(sv, c)
+    o, lse = gpu_attn(sv, d, None, None)
+    g = np.random.default_rng(23)
+    w = c["workload"]
+    smp = [(int(g.integers(0, w.n_seq)), int(g.integers(0, w.n_draft)), int(g.integers(0, w.n_q_heads))) for _ in range(32)]
+    o_ref, lse_ref = oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                              c["draft_k"], c["draft_v"], c["parent"], samples=smp)
+    check_attn(np.stack([o[s, i, h] for s, i, h in smp]), np.array([lse[s, i, h] for s, i, h in smp]), o_ref, lse_ref,
+               "cfg3 dense")
+
+
+@pytest.mark.parametrize("point", [(8192, 1 / 16, 8), (8192, 1 / 4, 16), (32768, 1 / 16, 4), (32768, 1 / 4, 8),
+                                   (131072, 1 / 16, 16), (131072, 1 / 32, 8), (131072, 1 / 4, 1)])
+def test_more_sweep_points(sv, point):
+    """Further points of the context x budget x draft-length sweep: every context, the 1/16 budget, 8 draft tokens."""
     c = si.make_layer(si.make_geometry(si.sweep_workload(*point)), sharp=True)
     g = np.random.default_rng(19)
     w = c["workload"]
     smp = [(0, int(g.integers(0, w.n_draft)), int(g.integers(0, w.n_q_heads))) for _ in range(32)]
-    run_fused(sv, c, what=f"fused sweep {point}", samples=smp)
+    run_sampled(sv, c, smp, what=f"sweep {point}")
 
 
 @pytest.mark.parametrize("forced", [(0, 0), (2, 4)])
@@ -420,8 +372,7 @@ def test_layer_stack_with_reuse_matches_oracle(sv):
         rel = np.linalg.norm(o - o_ref, axis=-1) / np.linalg.norm(o_ref, axis=-1)
         assert rel.max() <= 1e-2, (l, rel.max())
     np.testing.assert_array_equal(eng.sel_idx.cpu().numpy(), ref_sel[2][0])
-    attn = 2 if sv.sv_verify_attn_splits(eng.geom, geom["max_sel"]) > 1 else 1
-    assert eng.kernels_per_step() == 2 * sv.sv_select_verify_attn_launches(eng.geom, geom["max_sel"]) + 2 * attn
+    assert eng.kernels_per_step() == 2 + 4 * (2 if sv.sv_verify_attn_splits(eng.geom, geom["max_sel"]) > 1 else 1)
 
 
 # ------------------------------------------------------------------ full-size configurations
