@@ -38,6 +38,24 @@ METRIC = "sparse_verify_attn_us_per_layer"
 UNIT = "us/layer"
 
 
+def ncu_dram_bytes(kernel, **shape):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` at this shape, from the table of ncu captures
+    kept under profiles/ (one line per capture: kernel, key=value pairs, bytes); None when no capture matches."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_bytes_per_launch.txt")
+    if not os.path.exists(path):
+        return None
+    want = {k: str(v) for k, v in shape.items()}
+    with open(path) as f:
+        for line in f:
+            parts = line.split()
+            if len(parts) < 3 or parts[0].startswith("#") or parts[0] != kernel:
+                continue
+            kv = dict(x.split("=", 1) for x in parts[1:-1] if "=" in x)
+            if kv == want:
+                return int(parts[-1])
+    return None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -91,14 +109,20 @@ def run_reference(args):
         nh //= 2
     for _ in range(args.warmup):
         oracle_layer_seconds(case, nh)
-    times = [oracle_layer_seconds(case, nh) for _ in range(args.steps)]
+    walls = []
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        times.append(oracle_layer_seconds(case, nh))
+        walls.append(time.perf_counter() - t0)
     sec_per_layer = sum(times) / len(times)
     us = sec_per_layer * 1e6
-    sample = (f"one layer per step: block selection of the layer + sparse attention of the query heads of {nh} of "
-              f"{w.n_kv_heads} KV heads, scaled to the layer")
+    sample = (f"a step of this arm is a bounded sample, not the whole stack: one layer's block selection + sparse attention "
+              f"of the query heads of {nh} of {w.n_kv_heads} KV heads; `value` scales the attention part to the layer, "
+              f"`ms_per_step` is the wall time of the sample as measured")
     line = {
         "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": sec_per_layer * 1e3 * w.n_layers, "higher_is_better": False,
+        "warmup": args.warmup, "ms_per_step": sum(walls) / len(walls) * 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w, geom),
         "cpu_baseline": {"value": us, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
@@ -290,7 +314,27 @@ def run_gpu(args):
         def __exit__(self, *a):
             return False
 
+    # one uncaptured pass with an NVTX range per stage, for timelines taken with a profiler (graph replays show as one node)
+    nvtx = torch.cuda.nvtx
+    with torch.cuda.stream(stream):
+        nvtx.range_push("sv step (annotated, untimed)")
+        nvtx.range_push("sv_block_reps tail refresh, all layers")
+        eng.refresh_tail_all()
+        nvtx.range_pop()
+        for l in range(w.n_layers):
+            nvtx.range_push(f"layer {l}: sv_select_blocks")
+            sv.sv_select_blocks(eng.geom, q[l], eng.reps[l], eng.seq_lens, eng.budget, eng.n_sink, eng.n_local, eng.sel_idx,
+                                eng.sel_cnt)
+            nvtx.range_pop()
+            nvtx.range_push(f"layer {l}: sv_verify_attn")
+            sv.sv_verify_attn(eng.geom, q[l], eng.kv[l], dk[l], dv[l], None, eng.sel_idx, eng.sel_cnt, out[l],
+                              workspace=eng.workspace, status_word=eng.status)
+            nvtx.range_pop()
+        nvtx.range_pop()
+        stream.synchronize()
+    nvtx.range_push("capture")
     g_step = capture(lambda: eng.verify_step(q, dk, dv, out, refresh_tail=True))
+    nvtx.range_pop()
     if args.only_step:
         ms = time_replays(g_step, args.steps, args.warmup)
         if rank == 0:
@@ -308,7 +352,9 @@ def run_gpu(args):
     g_reps = capture(lambda: [sv.sv_block_reps(eng.geom, eng.kv[l], reps_scratch) for l in range(w.n_layers)])
 
     sampler = ClockSampler(local)
+    nvtx.range_push("timed: step graph replays")
     ms_step = time_replays(g_step, args.steps, max(args.warmup, 3), sampler=sampler)
+    nvtx.range_pop()
     side = max(10, min(args.steps, 200))
     ms_reuse = time_replays(g_reuse, side, 3)
     ms_chain = time_replays(g_chain, side, 3)
@@ -365,7 +411,29 @@ def run_gpu(args):
         barrier()
         return e0.elapsed_time(e1) / steps
 
-    ms_e2e = time_e2e(side, 4)
+    ms_e2e_pipelined = time_e2e(side, 4)
+
+    def time_e2e_serial(steps, warmup):
+        """Copy in, run the step, copy out, one step after the other on one stream: the next step's queries depend on
+        what this step accepts, so a decoding loop cannot overlap the copies of neighbouring steps."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            for i in range(warmup + steps):
+                if i == warmup:
+                    stream.synchronize()
+                    barrier()
+                    e0.record(stream)
+                q.copy_(q_h, non_blocking=True)
+                dk.copy_(dk_h, non_blocking=True)
+                dv.copy_(dv_h, non_blocking=True)
+                g_step.replay()
+                out_h.copy_(out, non_blocking=True)
+            e1.record(stream)
+            stream.synchronize()
+        barrier()
+        return e0.elapsed_time(e1) / steps
+
+    ms_e2e = time_e2e_serial(side, 4)
     assert int(eng.status.item()) == 0 and int(eng_reuse.status.item()) == 0 and int(eng_chain.status.item()) == 0, \
         "a kernel gave up on a bounded wait"
 
@@ -376,8 +444,9 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps = (
-        aggregate_over_ranks(x, world, allmax)[0] for x in (ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps))
+    ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps, ms_e2e_pipelined = (
+        aggregate_over_ranks(x, world, allmax)[0]
+        for x in (ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps, ms_e2e_pipelined))
 
     # algorithmic bytes of one sv_verify_attn launch (K+V of the kept tokens and draft tokens, Q in, O out)
     S, T, Hq, Hkv, D, B, N = w.n_seq, w.n_draft, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, w.budget_blocks
@@ -400,16 +469,20 @@ def run_gpu(args):
         "clocks": sampler.summary(),
         "e2e": {"value": ms_e2e * 1e3 / (w.n_layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
-                "note": "per step: Q and draft K/V of all layers copied from pinned host memory, outputs copied back "
-                        "(copies of neighbouring steps overlap the kernels: two buffer sets, three streams); "
-                        "the KV cache is device-resident state"},
+                "note": "per step, one after the other on one stream: Q and draft K/V of all layers copied from pinned host "
+                        "memory, the step, the outputs copied back (a decoding loop cannot overlap neighbouring steps: the "
+                        "next queries depend on this step's acceptance); the KV cache is device-resident state",
+                "pipelined_value": ms_e2e_pipelined * 1e3 / (w.n_layers * world),
+                "pipelined_note": "the same copies with two buffer sets and three streams, so that the copies of steps "
+                                  "i+1 / i-1 run under the kernels of step i (an upper bound no real loop reaches)"},
         "gpu_launches": args.steps * eng.kernels_per_step(refresh_tail=True),
         "kernels_per_step": eng.kernels_per_step(refresh_tail=True),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}",
-                     # dram__bytes_read.sum + dram__bytes_write.sum of verify_attn_tc_kernel<1> from the ncu capture
-                     # summarised in profiles/cfg1_step_tcgen05_4layers.md (same shapes, per launch)
-                     "traffic": 16931840 if (w.n_layers, w.budget_blocks) == (32, 64) else None,
+                     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this shape, if one
+                     # is on record (profiles/ncu_dram_bytes_per_launch.txt)
+                     "traffic": ncu_dram_bytes("verify_attn_tc_kernel", S=S, Hq=Hq, Hkv=Hkv, B=B, context=int(geom["seq_lens"][0]),
+                                               kept_blocks=N, T=T),
                      "kernel": "sv_verify_attn (split-KV attention + split merge), one launch per layer",
                      "bytes_per_launch": attn_bytes, "us_per_launch": us_attn},
         "kv_gathered_gbs": gathered / (us_attn * 1e-6) / 1e9,
@@ -428,7 +501,19 @@ def run_gpu(args):
         "min_score_gap_over_delta": min_ratio,
     }
 
+    # the paper's own context for this configuration (no latency is published; Table 2 gives attention sparsity only)
+    s_a = 1.0 - min(N * B, int(geom["seq_lens"][0])) / float(geom["seq_lens"][0])
+    line["paper_context"] = {
+        "attention_sparsity_s_a": s_a, "implied_reduction_of_the_quadratic_term": 1.0 / (1.0 - s_a),
+        "table2_s_a": {"L0=4K": [0.34, 0.39, 0.41, 0.41, 0.45], "L0=2K": [0.60, 0.63, 0.64, 0.56, 0.66],
+                       "L0=1K": [0.75, 0.77, 0.77, 0.72, 0.78]},
+        "note": "Table 2: GovReport / 2WikiMQA / HotpotQA / LCC / RepoBench-P, Llama-3.1-8B-Instruct + EAGLE-3 drafts, 60-token "
+                "trees, rho = 0.1, 8 x H800-80G, precision not stated; Table 1: sparse attention costs 4B(1-s_a)T^2 d of the "
+                "4BT^2 d term.  The paper reports no latency or speed-up for this path"}
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import ctypes
+
         import oracle
         oracle_layer_seconds(layers[0], 1)
         n_layers_sample = w.n_layers
@@ -438,6 +523,44 @@ def run_gpu(args):
                                 "kind": "oracle",
                                 "sample": f"{n_layers_sample} of {w.n_layers} layers, each in full (block selection + sparse "
                                           f"attention of all heads), {time.perf_counter() - t0:.1f} s of wall time"}
+        # parity of this run's output beside the timing (layer 0 in full), and how far sparse is from dense (information:
+        # the paper bounds no approximation error)
+        c0 = layers[0]
+        idx_ref, cnt_ref, _ = oracle.select_blocks(c0["q"], c0["k_pool"], c0["block_table"], c0["seq_lens"], c0["budget"],
+                                                   w.n_sink, w.n_local, c0["max_sel"])
+        o_ref, _ = oracle.verify_attn(c0["q"], c0["k_pool"], c0["v_pool"], c0["block_table"], c0["seq_lens"], c0["draft_k"],
+                                      c0["draft_v"], c0["parent"], idx_ref, cnt_ref)
+        t0 = time.perf_counter()
+        o_dense, _ = oracle.dense_verify_attn(c0["q"], c0["k_pool"], c0["v_pool"], c0["block_table"], c0["seq_lens"],
+                                              c0["draft_k"], c0["draft_v"], c0["parent"])
+        t_dense = time.perf_counter() - t0
+        with torch.cuda.stream(stream):
+            eng.verify_layer(0, q[0], dk[0], dv[0], out[0])
+            stream.synchronize()
+        o_gpu = si.bf16_bits_to_f64(out[0].cpu().view(torch.int16).numpy().view(np.uint16))
+        idx_ok = bool((eng.sel_cnt.cpu().numpy() == cnt_ref).all() and (eng.sel_idx.cpu().numpy() == idx_ref).all())
+        err = np.abs(o_gpu - o_ref)
+        rel = np.linalg.norm(o_gpu - o_ref, axis=-1) / np.linalg.norm(o_ref, axis=-1)
+        rel_sd = np.linalg.norm(o_ref - o_dense, axis=-1) / np.linalg.norm(o_dense, axis=-1)
+        line["parity"] = {"layer": 0, "block_lists_exact": idx_ok, "max_abs": float(err.max()), "mean_abs": float(err.mean()),
+                          "max_row_rel_l2": float(rel.max()), "bar": "lists exact; max-abs 1e-2, mean-abs 1e-3, row rel-L2 1e-2"}
+        line["sparse_vs_dense_oracle"] = {"max_row_rel_l2": float(rel_sd.max()), "mean_row_rel_l2": float(rel_sd.mean()),
+                                          "note": "information only: synthetic i.i.d. keys, no bound is claimed"}
+        line["cpu_baseline_dense"] = {"value": t_dense * 1e6, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                      "sample": "dense verification of layer 0 in full"}
+        # the same oracle on one thread (a quarter of a layer's KV heads, scaled)
+        try:
+            gomp = ctypes.CDLL("libgomp.so.1")
+            n_thr = oracle.num_threads()
+            gomp.omp_set_num_threads(1)
+            nh1 = max(1, w.n_kv_heads // 4)
+            t1 = oracle_layer_seconds(c0, nh1)
+            gomp.omp_set_num_threads(n_thr)
+            line["cpu_baseline_1thread"] = {"value": t1 * 1e6, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                            "sample": f"layer 0: block selection + sparse attention of {nh1} of {w.n_kv_heads} "
+                                                      f"KV heads, scaled to the layer"}
+        except OSError:
+            pass
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -542,7 +665,12 @@ def run_configs(args):
     stream = torch.cuda.Stream(device=dev)
     D = 128
     cases = [("cfg2", dict(S=16, Hq=32, Hkv=8, B=64, lens=(4096, 16384), budget_tokens=2048, T=5, tree=False, seed=1002)),
-             ("cfg3", dict(S=4, Hq=64, Hkv=8, B=128, lens=(131072, 131072), budget_tokens=4096, T=16, tree=True, seed=1003))]
+             ("cfg3", dict(S=4, Hq=64, Hkv=8, B=128, lens=(131072, 131072), budget_tokens=4096, T=16, tree=True, seed=1003)),
+             # the paper's own verification shape (Section 2.2, set-up of Section 4.1): a 60-token draft tree on
+             # Llama-3.1-8B geometry (240 query rows per KV head), budget from Eq. 6 with rho = 0.1 and L0 = 4K
+             ("tree60", dict(S=1, Hq=32, Hkv=8, B=64, lens=(32768, 32768), budget_tokens=None, T=60, tree=True, seed=1060))]
+    if args.only:
+        cases = [c for c in cases if c[0] in args.only.split(",")]
     for name, c in cases:
         S, Hq, Hkv, B, T = c["S"], c["Hq"], c["Hkv"], c["B"], c["T"]
         rng = np.random.default_rng(c["seed"])
@@ -550,7 +678,7 @@ def run_configs(args):
         nb = (lens + B - 1) // B
         NB = int(nb.max())
         n_pages = int(nb.sum())
-        N = c["budget_tokens"] // B
+        N = c["budget_tokens"] // B if c["budget_tokens"] else sv.sv_budget_blocks(int(lens.max()), 4096, 0.1, B, 1, 1)
         perm = rng.permutation(n_pages).astype(np.int32)
         bt_h = np.zeros((S, NB), np.int32)
         o = 0
@@ -622,20 +750,24 @@ def run_configs(args):
                 stream.synchronize()
             return e0.elapsed_time(e1) * 1e3 / iters / len(kvs)
 
-        us_sel, us_attn, us_both = timed(sel_all, 20), timed(attn_all, 20), timed(both_all, 20)
-        us_dense = timed(dense_all, 5)
+        iters = args.steps if args.only else 20
+        us_sel, us_attn, us_both = timed(sel_all, iters), timed(attn_all, iters), timed(both_all, iters)
+        us_dense = timed(dense_all, 5) if not args.only else None
         assert int(status.item()) == 0, "a kernel gave up on a bounded wait"
         dense_bytes = int(nb.sum()) * Hkv * B * D * 2 * 2
         print(json.dumps({"config": name, "n_seq": S, "q_heads": Hq, "kv_heads": Hkv, "block": B, "n_draft": T,
                           "tree": bool(c["tree"]), "context_min": int(lens.min()), "context_max": int(lens.max()),
-                          "budget_blocks": N, "splits": sv.sv_verify_attn_splits(geom, N), "replicas": n_rep,
+                          "budget_blocks": N, "query_rows_per_kv_head": (Hq // Hkv) * T,
+                          "splits": sv.sv_verify_attn_splits(geom, N), "replicas": n_rep,
+                          "attn_algorithmic_bytes": gathered + Hkv * S * T * D * 2 * 2 + 2 * S * T * Hq * D * 2,
                           "gathered_kv_mib": round(gathered / 2 ** 20, 1),
                           "select_us": round(us_sel, 2), "attn_us": round(us_attn, 2), "select_plus_attn_us": round(us_both, 2),
                           "kv_gbs": round(gathered / us_attn / 1e3, 1),
                           "frac_of_measured_peak": round(gathered / us_attn / 1e3 / peak, 3),
-                          "dense_attn_us": round(us_dense, 2), "dense_kv_mib": round(dense_bytes / 2 ** 20, 1),
-                          "dense_frac_of_measured_peak": round(dense_bytes / us_dense / 1e3 / peak, 3),
-                          "speedup_vs_dense": round(us_dense / us_both, 2)}), flush=True)
+                          "dense_attn_us": None if us_dense is None else round(us_dense, 2),
+                          "dense_kv_mib": round(dense_bytes / 2 ** 20, 1),
+                          "dense_frac_of_measured_peak": None if us_dense is None else round(dense_bytes / us_dense / 1e3 / peak, 3),
+                          "speedup_vs_dense": None if us_dense is None else round(us_dense / us_both, 2)}), flush=True)
         del pools, kvs, reps
 
 
@@ -746,6 +878,7 @@ def main():
                     help="instead of the benchmark line: sparse vs dense latency over context x budget x draft length")
     ap.add_argument("--configs", action="store_true",
                     help="timing lines for the batched (16 ragged sequences) and long-context (4 x 128K, tree) configurations")
+    ap.add_argument("--only", default="", help="with --configs: comma-separated configuration names (profiling aid: no dense pass)")
     ap.add_argument("--variants", action="store_true",
                     help="instead of the benchmark line: timings of the retrieval variants (shared budget, every token)")
     args = ap.parse_args()

@@ -29,6 +29,14 @@ inline int row_tiles(const sv_geom *g)
     return (g->n_draft + tt - 1) / tt;
 }
 
+// CTAs per (sequence, KV head, split): one per row tile, or one per pair of row tiles when there are several (a CTA
+// then serves two tiles from one gather of the kept K/V)
+inline int row_groups(const sv_geom *g)
+{
+    const int t = row_tiles(g);
+    return t > 1 ? (t + 1) / 2 : 1;
+}
+
 inline sv_status check_geom(const sv_geom *g)
 {
     if (!g) return SV_ERR_NULL;

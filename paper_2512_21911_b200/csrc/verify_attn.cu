@@ -153,7 +153,7 @@ using svh::sm_count;
 // that out (16 ragged sequences of 4.8-15K tokens, dense: 138 -> 90 us).
 int choose_splits(const sv_geom *g, int n_blocks, bool balance = true)
 {
-    const int pairs = g->n_seq * g->n_kv_heads * svh::row_tiles(g);
+    const int pairs = g->n_seq * g->n_kv_heads * svh::row_groups(g);
     const int per_pair = sm_count() / pairs;
     if (n_blocks <= 1) return 1;
     if (per_pair <= 1) {
@@ -245,7 +245,7 @@ static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_k
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     dim3 grid(splits, geom->n_kv_heads, geom->n_seq);
-    grid.x = splits * p.tiles;   // one CTA per (row tile, split)
+    grid.x = splits * svh::row_groups(geom);   // one CTA per (row tile or pair of row tiles, split)
     if (launch_attn_tc(tk, tv, p, grid, cs) != cudaSuccess) return SV_ERR_CUDA;
     if (splits > 1) {
         cudaLaunchConfig_t cfg = {};

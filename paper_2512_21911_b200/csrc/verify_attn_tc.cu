@@ -38,16 +38,16 @@ constexpr int kThreads = 384;
 constexpr int kUnit = 64;                        // keys per unit
 constexpr int kTile = kUnit * 128;               // bytes of one [64 rows][64 bf16] half tile (8 KB)
 constexpr int kStageBytes = 4 * kTile;           // K lo/hi + V lo/hi
-constexpr int kStages = 5;
-constexpr int kQBytes = 2 * 128 * 128;           // Q: two halves [128 rows][64 bf16]
+constexpr int kStages = 5;                       // ring stages; a CTA that serves two row tiles has two Q tiles and four stages
+constexpr int kQBytes = 2 * 128 * 128;           // Q of one row tile: two halves [128 rows][64 bf16]
 constexpr int kPBytes = 128 * 128;               // P: [128 rows][64 bf16]
-constexpr int kOffQ = kStages * kStageBytes;
-constexpr int kOffP = kOffQ + kQBytes;
+constexpr int kOffP = kStages * kStageBytes + kQBytes;   // (= 4 stages + 2 Q tiles)
 constexpr int kOffDraft = 0;                     // the draft unit is the first occupant of ring stage 0 (last split only)
 constexpr int kOffMisc = kOffP + 2 * kPBytes;
 constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 static_assert(2 * kStages + 10 <= 32, "one lane of the producer warp per barrier");
+static_assert((kStages - 1) * kStageBytes + 2 * kQBytes == kOffP, "both layouts put P at the same offset");
 constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns
 
 // barrier slots (8 bytes each) inside the misc area
@@ -67,7 +67,10 @@ enum Bar {
 // kWide: more than one row tile per (sequence, KV head) or more than 32 draft tokens (64-bit ancestor masks).  The
 // common case keeps split = blockIdx.x, plain row arithmetic and 32-bit masks: deriving the split from a division
 // costs 3 % on long loops, and the wider mask code 7 % at 128 rows.
-template <int NH, bool kWide>
+// kPair (with kWide, NH = 4): the CTA serves two row tiles of its (sequence, KV head) from one gather: warpgroup w owns
+// row tile 2 * pair + w -- its own Q tile, S / P / O buffers -- and takes every unit instead of every other one, so the
+// kept K/V cross HBM once per pair of tiles (240 query rows, a 60-token draft tree on a GQA-4 model: once in all).
+template <int NH, bool kWide, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
     verify_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                           const AttnParams p)
@@ -84,16 +87,27 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 456);
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
-    // blockIdx.x = row tile * splits + split: the query rows of draft tokens i0 .. i0 + Tq - 1, a slice of the blocks
-    const int tile = kWide ? blockIdx.x / p.splits : 0;
-    const int split = kWide ? blockIdx.x - tile * p.splits : blockIdx.x, h = blockIdx.y, s = blockIdx.z;
-    const int i0 = kWide ? tile * p.Tt : 0, Tq = kWide ? min(p.Tt, p.T - i0) : p.T;
+    static_assert(!kPair || (kWide && NH == 4), "row-tile pairs exist only where one tile is full (more than 64 rows)");
+    constexpr int NS = kPair ? kStages - 1 : kStages;        // ring stages
+    constexpr int OFFQ = NS * kStageBytes;                   // the Q tile (kPair: of warpgroup 0; warpgroup 1's follows)
+    // blockIdx.x = group * splits + split.  A group is a row tile (kWide), or a pair of row tiles (kPair) of which
+    // softmax warpgroup w owns tile 2 * group + w; `tile`, `i0`, `Tq`, `rows` are those of the executing warpgroup
+    // (the query rows of draft tokens i0 .. i0 + Tq - 1).  The split selects a slice of the blocks.
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int group = kWide ? blockIdx.x / p.splits : 0;
+    const int split = kWide ? blockIdx.x - group * p.splits : blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+    const int tile = kPair ? 2 * group + ((warp >> 2) & 1) : group;
+    const int i0 = kWide ? tile * p.Tt : 0, Tq = kWide ? max(0, min(p.Tt, p.T - i0)) : p.T;
     const int upb = p.B / kUnit;
     const bool has_draft = split == p.splits - 1;
-    const int rows = p.G * Tq;                               // query rows of this tile
+    const int rows = p.G * Tq;                               // query rows of this tile (0: the pair's second tile does not exist)
     constexpr int RPQ = 8 * NH;                              // query rows per TMEM lane quadrant
-    const int n_active = min(4, (rows + RPQ - 1) / RPQ);     // warps per softmax warpgroup that own real rows
+    const int n_active = min(4, (rows + RPQ - 1) / RPQ);     // warps of this softmax warpgroup that own real rows
+    // the same for either warpgroup, for the roles that serve both
+    const int rows_w1 = kPair ? p.G * max(0, min(p.Tt, p.T - (2 * group + 1) * p.Tt)) : 0;
+    const int rows_w0 = kPair ? p.G * min(p.Tt, p.T - 2 * group * p.Tt) : rows;
+    const int na0 = min(4, (rows_w0 + RPQ - 1) / RPQ), na1 = kPair ? min(4, (rows_w1 + RPQ - 1) / RPQ) : na0;
+    const int n_wg = (kPair && rows_w1 == 0) ? 1 : 2;        // warpgroups that take part
 
     // r / G for the small row indices of this kernel (0 <= r < 8192, 1 <= G <= 128) without an integer division:
     // (r + 0.5) / G is at least 0.5 / G >= 2^-8 away from the next integer, far more than the fp32 rounding error
@@ -117,10 +131,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (warp == 8) {
         if (lane < kNumBars) {
             uint32_t count = 1;
-            if (lane >= kSFree && lane < kSFree + 2) count = n_active;
-            if (lane >= kPReady && lane < kPReady + 2) count = n_active;
+            if (lane == kSFree || lane == kPReady) count = na0;
+            if (lane == kSFree + 1 || lane == kPReady + 1) count = max(1, na1);
             if (lane == kStaged) count = 8;
-            if (lane == kTmemDone) count = 2 * n_active;
+            if (lane == kTmemDone) count = na0 + (n_wg == 2 ? na1 : 0);
             mbar_init(bar(lane), count);
             mbar_fence_init();
         }
@@ -187,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (lane == 0 && !dead) {
                         for (int uo = 0; uo < upb; ++uo) {
                             const int u = (base - j0 + i) * upb + uo;   // ring unit; the draft unit (if any) came first
-                            const int stage = (u + off) % kStages, it = (u + off) / kStages;
+                            const int stage = (u + off) % NS, it = (u + off) / NS;
                             if (it > 0 && (*abort_flag || !mbar_wait_bounded(bar(kEmpty + stage), (it - 1) & 1))) {
                                 dead = true;
                                 *abort_flag = 1;
@@ -226,13 +240,16 @@ __global__ void __launch_bounds__(kThreads, 1)
                 bool dead = !mbar_wait_bounded(bar(kStaged), 0);
                 if (warp == 9) {
                     constexpr uint32_t idesc_s = umma_idesc_bf16(128, kUnit, false);
-                    const uint64_t dq = umma_desc_sw128(smem0 + kOffQ, 16, 1024);
+                    const uint64_t dq = umma_desc_sw128(smem0 + OFFQ, 16, 1024);
                     const uint64_t dk = umma_desc_sw128(smem0, 16, 1024);
                     const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk;
                     const uint64_t d_hi = dq & 0xFFFFFFFF00000000ull;
-                    for (int u = 0; u < n_total && !dead; ++u) {
-                        const int g = u & 1, k = u >> 1;
-                        const int stage = u % kStages, it = u / kStages;
+                    // one S per (unit, warpgroup that takes it): the warpgroups alternate units, or (kPair) each takes all
+                    const int n_issue = kPair ? n_total * n_wg : n_total;
+                    for (int x = 0; x < n_issue && !dead; ++x) {
+                        const int u = kPair ? (n_wg == 2 ? x >> 1 : x) : x;
+                        const int g = kPair ? (n_wg == 2 ? (x & 1) : 0) : (u & 1), k = kPair ? u : (u >> 1);
+                        const int stage = u % NS, it = u / NS;
                         if (*abort_flag || !mbar_wait_bounded(bar(kFull + stage), it & 1) ||
                             (k > 0 && !mbar_wait_bounded(bar(kSFree + g), (k - 1) & 1))) {
                             dead = true;
@@ -245,7 +262,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const uint32_t d = tmem_base + g * kUnit;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
-                            const uint32_t qo = (uint32_t)(((ks >> 2) * (kQBytes / 2) + (ks & 3) * 32) >> 4);
+                            const uint32_t qo = (uint32_t)(((kPair ? g * kQBytes : 0) + (ks >> 2) * (kQBytes / 2) + (ks & 3) * 32) >> 4);
                             const uint32_t ko = (uint32_t)(((ks >> 2) * kTile + (ks & 3) * 32) >> 4);
                             tc_mma_bf16(d, d_hi | (dq_lo + qo), d_hi | (k_lo + ko), idesc_s, ks > 0);
                         }
@@ -259,9 +276,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint64_t dv = umma_desc_sw128(smem0 + 2 * kTile, kTile, 1024);
                     const uint32_t dp_lo = (uint32_t)dp, dv_lo = (uint32_t)dv;
                     const uint64_t dp_hi = dp & 0xFFFFFFFF00000000ull, dv_hi = dv & 0xFFFFFFFF00000000ull;
-                    for (int u = 0; u < n_total && !dead; ++u) {
-                        const int g = u & 1, k = u >> 1;
-                        const int stage = u % kStages;
+                    const int n_issue = kPair ? n_total * n_wg : n_total;
+                    for (int x = 0; x < n_issue && !dead; ++x) {
+                        const int u = kPair ? (n_wg == 2 ? x >> 1 : x) : x;
+                        const int g = kPair ? (n_wg == 2 ? (x & 1) : 0) : (u & 1), k = kPair ? u : (u >> 1);
+                        const int stage = u % NS;
                         if (*abort_flag || !mbar_wait_bounded(bar(kPReady + g), k & 1)) {
                             dead = true;
                             *abort_flag = 1;
@@ -277,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             tc_mma_bf16(d, dp_hi | (p_lo + (uint32_t)((kk * 32) >> 4)), dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)),
                                         idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);   // the warpgroup's first unit starts O
                         tc_commit(bar(kOReady + g));
-                        tc_commit(bar(kEmpty + stage));
+                        if (!kPair || g == n_wg - 1) tc_commit(bar(kEmpty + stage));   // the last reader of the stage
                     }
                 }
             }
@@ -297,11 +316,15 @@ __global__ void __launch_bounds__(kThreads, 1)
     // (r / RPQ)*32 + r % RPQ: RPQ rows per TMEM lane quadrant, so that all four warps of a warpgroup
     // share the softmax work even when only a few of the 128 tile rows are real.
     // The zero padding needs no input and is written while the previous kernel in the stream drains.
-    for (int idx = tid; idx < 128 * 16; idx += 256) {
+    // kPair: each warpgroup stages the Q tile of its own row tile (128 threads each); otherwise all 256 threads share one
+    constexpr int kQThreads = kPair ? 128 : 256;
+    const int qtid = kPair ? (tid & 127) : tid;
+    uint8_t *q_tile = smem + OFFQ + (kPair ? ((warp >> 2) & 1) * kQBytes : 0);
+    for (int idx = qtid; idx < 128 * 16; idx += kQThreads) {
         const int tr = idx >> 4, c = idx & 15;
         const int r = (tr >> 5) * RPQ + (tr & 31);
         if (!((tr & 31) < RPQ && r < rows))
-            *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = make_uint4(0u, 0u, 0u, 0u);
     }
     if (has_draft) {
         for (int idx = tid; idx < 2 * kUnit * 16; idx += 256) {
@@ -316,12 +339,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     {
         // real rows: all loads of a thread are in flight together (16-byte chunks: Q up to 128 rows x 16, draft K and
         // V up to 64 tokens x 16 each)
-        constexpr int kQB = NH == 4 ? 8 : 4, kDB = kWide ? 8 : 4;
+        constexpr int kQB = (NH == 4 ? 8 : 4) * (kPair ? 2 : 1), kDB = kWide ? 8 : 4;
         const int n_q = rows * 16, n_d = has_draft ? 2 * p.T * 16 : 0;
         uint4 v[kQB];
 #pragma unroll
         for (int x = 0; x < kQB; ++x) {
-            const int idx = tid + x * 256;
+            const int idx = qtid + x * kQThreads;
             if (idx < n_q) {
                 const int r = idx >> 4, c = idx & 15;
                 const int i = div_g(r), g = r - i * p.G;
@@ -372,11 +395,11 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
 #pragma unroll
         for (int x = 0; x < kQB; ++x) {
-            const int idx = tid + x * 256;
+            const int idx = qtid + x * kQThreads;
             if (idx < n_q) {
                 const int r = idx >> 4, c = idx & 15;
                 const int tr = (r / RPQ) * 32 + (r % RPQ);
-                *reinterpret_cast<uint4 *>(smem + kOffQ + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = v[x];
+                *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = v[x];
             }
         }
 #pragma unroll
@@ -454,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     };
 
     int k = 0;
-    for (int u = wg; u < n_total; u += 2, ++k) {
+    for (int u = kPair ? 0 : wg; u < n_total; u += kPair ? 1 : 2, ++k) {   // kPair: every unit, for this warpgroup's row tile
         if (!dead && __any_sync(0xffffffffu, *abort_flag || !mbar_wait_bounded(bar(kSReady + wg), k & 1))) {
             dead = true;
             *abort_flag = 1;
@@ -463,7 +486,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (dead) break;
         tc_fence_after_sync();
         const bool is_draft = u < off;
-        const int stage = u % kStages;
+        const int stage = u % NS;
         const int nvalid = is_draft ? p.T : min(meta[stage], kUnit);
         uint8_t *pbuf = smem + kOffP + wg * kPBytes;
         if constexpr (NH == 4) {
@@ -669,7 +692,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------------ combine the two warpgroups, write out
     // Warp q of either warpgroup owns TMEM lane quadrant q, so each warpgroup can read the other's accumulator straight
     // from TMEM: both wait for their last PV, exchange (m, l) through their own (now idle) P tiles, and then each merges
-    // and writes one half of the 128 output columns of every row.
+    // and writes one half of the 128 output columns of every row.  (kPair: the warpgroups hold different row tiles;
+    // each writes both halves of its own rows and nothing is exchanged.)
     const int n_sm = 2 * wg_threads;
     const int t = quad * 32 + lane;
     float *ml_mine = reinterpret_cast<float *>(smem + kOffP + wg * kPBytes);          // [2 * NH][128]: m, l per slot
@@ -679,82 +703,90 @@ __global__ void __launch_bounds__(kThreads, 1)
     // they spread over the SMs that the attention CTAs are about to vacate.
     grid_launch_dependents();
     if (k > 0) wait_pv(k - 1);   // this warpgroup's accumulator is complete
+    if constexpr (!kPair) {
 #pragma unroll
-    for (int i = 0; i < NH; ++i) {
-        ml_mine[(2 * i) * 128 + t] = m[i];
-        ml_mine[(2 * i + 1) * 128 + t] = l[i];
-    }
-    tc_fence_before_sync();
-    named_bar_sync(1, n_sm);
-    tc_fence_after_sync();
-    // a warpgroup without units never wrote its accumulator
-    const bool have_mine = k > 0 && !dead, have_other = n_total >= (wg == 0 ? 2 : 1);
-    const uint32_t t_o_other = tmem_base + t_lane + 128 + (wg ^ 1) * 128;
-    // this warp's rows of O, the warpgroup's half of the columns: 16 output dims 64 wg + 8 j + 2 qd + e (index 2 j + e)
-    float o[NH][16], row_m[NH], row_l[NH];
-#pragma unroll
-    for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo) {
-        uint32_t r0[32], r1[32];
-        if (have_mine) tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + wg * 64, r0);
-        if (have_other) tmem_ld_16x256b_x8(t_o_other + ((uint32_t)(lo * 16) << 16) + wg * 64, r1);
-#pragma unroll
-        for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh) {
-            const int i = lo * 2 + hh;
-            const float m1 = ml_other[(2 * i) * 128 + t], l1 = ml_other[(2 * i + 1) * 128 + t];
-            const float M = fmaxf(m[i], m1);
-            const float M_use = (M == -INFINITY) ? 0.f : M;
-            const float w0 = fast_exp2(m[i] - M_use), w1 = fast_exp2(m1 - M_use);
-            float lsum = w0 * l[i] + w1 * l1;
-            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
-            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-            row_m[i] = M, row_l[i] = lsum;
-            if (hh == 0) tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int x = 4 * j + 2 * hh + e;
-                    const float a = have_mine ? w0 * __uint_as_float(r0[x]) : 0.f;
-                    const float b = have_other ? w1 * __uint_as_float(r1[x]) : 0.f;
-                    o[i][2 * j + e] = a + b;
-                }
+        for (int i = 0; i < NH; ++i) {
+            ml_mine[(2 * i) * 128 + t] = m[i];
+            ml_mine[(2 * i + 1) * 128 + t] = l[i];
         }
+        tc_fence_before_sync();
+        named_bar_sync(1, n_sm);
+        tc_fence_after_sync();
     }
-    tc_fence_before_sync();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar(kTmemDone));   // this warp reads TMEM no more
+    // a warpgroup without units never wrote its accumulator
+    const bool have_mine = k > 0 && !dead, have_other = !kPair && n_total >= (wg == 0 ? 2 : 1);
+    const uint32_t t_o_other = tmem_base + t_lane + 128 + (wg ^ 1) * 128;
+    for (int ch = kPair ? 0 : wg; ch < (kPair ? 2 : wg + 1); ++ch) {   // column half: 64 output dims
+        // this warp's rows of O, 16 output dims 64 ch + 8 j + 2 qd + e (index 2 j + e)
+        float o[NH][16], row_m[NH], row_l[NH];
 #pragma unroll
-    for (int i = 0; i < NH; ++i) {
-        const float M = row_m[i], lsum = row_l[i];
-        const int row = lrow[i];
-        if (row >= rows) continue;
-        if (p.splits == 1) {
-            const int ii = div_g(row), g = row - ii * p.G;
-            const size_t orow = ((size_t)s * p.T + i0 + ii) * p.Hq + h * p.G + g;
-            const float inv = 1.f / lsum;
-            uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + wg * 32 + qd;
+        for (int lo = 0; lo < (NH == 4 ? 2 : 1); ++lo) {
+            uint32_t r0[32], r1[32];
+            if (have_mine) tmem_ld_16x256b_x8(t_o + ((uint32_t)(lo * 16) << 16) + ch * 64, r0);
+            if (have_other) tmem_ld_16x256b_x8(t_o_other + ((uint32_t)(lo * 16) << 16) + ch * 64, r1);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) dst[4 * j] = pack_bf16(o[i][2 * j] * inv, o[i][2 * j + 1] * inv);
-            if (p.lse && wg == 0 && qd == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
-        } else {
-            const size_t prow = (((size_t)s * p.Hkv + h) * p.splits + split) * (p.G * p.T) + i0 * p.G + row;
-            float2 *dst = reinterpret_cast<float2 *>(p.ws_o + prow * 128) + wg * 32 + qd;
+            for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh) {
+                const int i = lo * 2 + hh;
+                const float m1 = kPair ? -INFINITY : ml_other[(2 * i) * 128 + t];
+                const float l1 = kPair ? 0.f : ml_other[(2 * i + 1) * 128 + t];
+                const float M = fmaxf(m[i], m1);
+                const float M_use = (M == -INFINITY) ? 0.f : M;
+                const float w0 = fast_exp2(m[i] - M_use), w1 = fast_exp2(m1 - M_use);
+                float lsum = w0 * l[i] + w1 * l1;
+                lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+                lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+                row_m[i] = M, row_l[i] = lsum;
+                if (hh == 0) tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) dst[4 * j] = make_float2(o[i][2 * j], o[i][2 * j + 1]);
-            if (wg == 0 && qd == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int x = 4 * j + 2 * hh + e;
+                        const float a = have_mine ? w0 * __uint_as_float(r0[x]) : 0.f;
+                        const float b = have_other ? w1 * __uint_as_float(r1[x]) : 0.f;
+                        o[i][2 * j + e] = a + b;
+                    }
+            }
+        }
+        if (!kPair || ch == 1) {
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kTmemDone));   // this warp reads TMEM no more
+        }
+#pragma unroll
+        for (int i = 0; i < NH; ++i) {
+            const float M = row_m[i], lsum = row_l[i];
+            const int row = lrow[i];
+            if (row >= rows) continue;
+            if (p.splits == 1) {
+                const int ii = div_g(row), g = row - ii * p.G;
+                const size_t orow = ((size_t)s * p.T + i0 + ii) * p.Hq + h * p.G + g;
+                const float inv = 1.f / lsum;
+                uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + orow * 128) + ch * 32 + qd;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) dst[4 * j] = pack_bf16(o[i][2 * j] * inv, o[i][2 * j + 1] * inv);
+                if (p.lse && ch == 0 && qd == 0) p.lse[orow] = (M + log2f(lsum)) * 0.69314718055994531f;
+            } else {
+                const size_t prow = (((size_t)s * p.Hkv + h) * p.splits + split) * (p.G * p.T) + i0 * p.G + row;
+                float2 *dst = reinterpret_cast<float2 *>(p.ws_o + prow * 128) + ch * 32 + qd;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) dst[4 * j] = make_float2(o[i][2 * j], o[i][2 * j + 1]);
+                if (ch == 0 && qd == 0) *reinterpret_cast<float2 *>(p.ws_ml + prow * 2) = make_float2(M, lsum);
+            }
         }
     }
 }
 
 }  // namespace
 
-template <int NH, bool kWide>
+template <int NH, bool kWide, bool kPair>
 static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                              cudaStream_t stream)
 {
     static svh::OncePerDevice once;   // function attributes belong to a device
     const cudaError_t ce = once.run([] {
-        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kSmemBytes);
     });
     if (ce != cudaSuccess) return ce;
     cudaLaunchConfig_t cfg = {};
@@ -766,21 +798,23 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
     svh::pdl_attribute(attr);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide>, tm_k, tm_v, p);
+    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide, kPair>, tm_k, tm_v, p);
 }
 
+// grid.x = splits x groups, where a group is a row tile or, with more than one row tile, a pair of them
 cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                            cudaStream_t stream)
 {
     const int rows = p.G * p.Tt;   // rows of a full row tile
-    if (p.tiles > 1 || p.T > 32) {
-        if (rows <= 32) return launch_tc<1, true>(tm_k, tm_v, p, grid, stream);
-        if (rows <= 64) return launch_tc<2, true>(tm_k, tm_v, p, grid, stream);
-        return launch_tc<4, true>(tm_k, tm_v, p, grid, stream);
+    if (p.tiles > 1) return launch_tc<4, true, true>(tm_k, tm_v, p, grid, stream);   // (a full tile has more than 64 rows)
+    if (p.T > 32) {
+        if (rows <= 32) return launch_tc<1, true, false>(tm_k, tm_v, p, grid, stream);
+        if (rows <= 64) return launch_tc<2, true, false>(tm_k, tm_v, p, grid, stream);
+        return launch_tc<4, true, false>(tm_k, tm_v, p, grid, stream);
     }
-    if (rows <= 32) return launch_tc<1, false>(tm_k, tm_v, p, grid, stream);
-    if (rows <= 64) return launch_tc<2, false>(tm_k, tm_v, p, grid, stream);
-    return launch_tc<4, false>(tm_k, tm_v, p, grid, stream);
+    if (rows <= 32) return launch_tc<1, false, false>(tm_k, tm_v, p, grid, stream);
+    if (rows <= 64) return launch_tc<2, false, false>(tm_k, tm_v, p, grid, stream);
+    return launch_tc<4, false, false>(tm_k, tm_v, p, grid, stream);
 }
 
 }  // namespace svk

@@ -165,6 +165,8 @@ SMALL = {
     "t40_chain_2seq": si.shrink(si.WORKLOADS["cfg2"], n_seq=2, seq_len=(900, 2100), budget_blocks=7, n_draft=40, planted=2),
     "g8_t24_b128": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(2000, 4000), budget_blocks=6, n_draft=24, planted=2),
     "g16_t64": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1100, 1100), budget_blocks=5, n_draft=64, tree=True, planted=2),
+    # an odd number of row tiles (3 x 128 rows: 16 + 16 + 8 draft tokens): the last CTA group serves a single tile
+    "g8_t40_tree_3tiles": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(1800, 3100), budget_blocks=6, n_draft=40, planted=2),
     # more (sequence, KV head) pairs than SMs: several waves of CTAs, one split each
     "many_seqs": si.shrink(si.WORKLOADS["cfg2"], n_seq=40, seq_len=(300, 1100), budget_blocks=6, planted=1),
     "b128_short_tail": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(128 * 9 + 30, 128 * 9 + 30), n_q_heads=16, n_kv_heads=4,

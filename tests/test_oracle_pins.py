@@ -187,6 +187,35 @@ def test_generator_plants_and_repairs_gap():
         assert sc[s, h, list(sel - {0, 63})].min() - sc[s, h, rest].max() >= c["delta"] * 0.999
 
 
+@pytest.mark.parametrize("forced", [(1, 1), (0, 0), (2, 3)])
+def test_generator_repairs_gap_on_ragged_lengths_with_partly_filled_last_blocks(forced):
+    """The generator scores blocks with its own copy of Eq. 5 to plant and repair the gap.  Where the last block
+    of a sequence is only partly filled, that copy has to divide by the tokens the block holds, as the oracle does
+    (with n_local = 0 the last block competes on its score): the oracle's own scores must show the promised gap
+    between kept and evicted blocks for every sequence of a ragged batch."""
+    w = si.shrink(si.WORKLOADS["cfg2"], n_seq=5, seq_len=(700, 3000), budget_blocks=9, n_sink=forced[0], n_local=forced[1])
+    geom = si.make_geometry(w)
+    assert any(int(L) % w.block_size for L in geom["seq_lens"])          # ragged: partly filled last blocks exist
+    c = si.make_layer(geom, sharp=True)
+    idx, cnt, sc = oracle.select_blocks(c["q"], c["k_pool"], c["block_table"], c["seq_lens"], c["budget"], forced[0],
+                                        forced[1], c["max_sel"])
+    assert c["min_gap_ratio"] >= 1.0 and c["delta"] > 0
+    gaps = []
+    for s in range(w.n_seq):
+        nb = int(c["n_blocks"][s])
+        forced_set = set(range(min(forced[0], nb))) | set(range(max(0, nb - forced[1]), nb))
+        for h in range(w.n_kv_heads):
+            sel = set(idx[s, h, :cnt[s, h]].tolist())
+            assert forced_set <= sel and set(c["planted"][(s, h)].tolist()) <= sel
+            rest = np.setdiff1d(np.arange(nb), list(sel))
+            chosen = list(sel - forced_set)
+            if len(rest) and len(chosen):     # the generator's own smallest gap must be the oracle's too
+                gap = sc[s, h, chosen].min() - sc[s, h, rest].max()
+                assert gap >= c["min_gap"] * (1 - 1e-9) - 1e-15 and gap > 0
+                gaps.append(gap)
+    assert abs(min(gaps) - c["min_gap"]) <= 1e-12 * max(1.0, abs(c["min_gap"]))
+
+
 # --------------------------------------------------------------------------- O5: inter-layer reuse (Eq. 9)
 
 def test_reuse_copies_nearest_preceding_anchor():
