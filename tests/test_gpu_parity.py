@@ -557,8 +557,9 @@ def test_commit_then_dense_verify_on_the_new_lengths(sv):
     g = np.random.default_rng(11)
     fresh = si.f32_to_bf16_bits(g.standard_normal((S, Hkv, B, 128)).astype(np.float32))
     k_pool, v_pool = np.concatenate([c["k_pool"], fresh]), np.concatenate([c["v_pool"], fresh[::-1].copy()])
-    lens = ((c["seq_lens"] // B) * B + B - 2).astype(np.int32)       # two slots left: every commit of >= 3 rows adds a block
-    lens = np.minimum(lens, c["n_blocks"] * B - 2).astype(np.int32)
+    # two slots before a block boundary inside the generated prefix (so that every cached token is real data): a
+    # commit of eight rows takes every sequence into its next block
+    lens = ((c["seq_lens"] // B) * B - 2).astype(np.int32)
     n_acc = np.full(S, T, np.int32)
     acc = np.tile(np.arange(T, dtype=np.int32), (S, 1))
     NB = bt.shape[1]
