@@ -146,6 +146,8 @@ bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
 
 using svh::sm_count;
 
+constexpr int kUnsplitUnits = 4;   // lists of at most this many 64-key units run on one CTA per (sequence, KV head)
+
 // Blocks per CTA are minimised subject to one CTA per SM; then the fewest splits that achieve it.
 // With at least one (sequence, KV head, row tile) per SM nothing needs splitting for occupancy, but long lists are
 // still cut into pieces of about 64 units when `balance` is set: the sequences of a batch differ in length, one CTA
@@ -156,6 +158,10 @@ int choose_splits(const sv_geom *g, int n_blocks, bool balance = true)
     const int pairs = g->n_seq * g->n_kv_heads * svh::row_groups(g);
     const int per_pair = sm_count() / pairs;
     if (n_blocks <= 1) return 1;
+    // A list of a few units is not worth a split: partials, the merge kernel and its boundary add 3 us to any split
+    // launch, more than one CTA per pair needs for four units in a row (1 MiB gathered: 6.5 -> 5.9 us per call; at
+    // eight units the serial chain is already slower: 7.8 against 6.5 us).
+    if (n_blocks * (g->block_size / 64) <= kUnsplitUnits) return 1;
     if (per_pair <= 1) {
         const int units = n_blocks * (g->block_size / 64);
         return (balance && units >= 128) ? (units + 63) / 64 : 1;

@@ -328,10 +328,15 @@ def test_empty_prefix_and_empty_selection(sv):
 
 def test_more_splits_than_blocks(sv):
     """One (sequence, KV head) pair: the split count is capped by the block count, some CTAs get one block."""
+    w = si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=1, seq_len=(2000, 2000), budget_blocks=10, planted=1)
+    c = si.make_layer(si.make_geometry(w), sharp=True)
+    d = run_pipeline(sv, c, what="10 blocks")[0]
+    assert sv.sv_verify_attn_splits(d.geom, 10) == 10
+    # a list of a few units is not split at all (the merge would cost more than the gather)
     w = si.shrink(si.WORKLOADS["cfg0"], n_q_heads=4, n_kv_heads=1, seq_len=(2000, 2000), budget_blocks=3, planted=1)
     c = si.make_layer(si.make_geometry(w), sharp=True)
     d = run_pipeline(sv, c, what="3 blocks")[0]
-    assert sv.sv_verify_attn_splits(d.geom, 3) == 3
+    assert sv.sv_verify_attn_splits(d.geom, 3) == 1 and sv.sv_workspace_bytes(d.geom, 3) == 0
 
 
 def test_workspace_too_small_is_rejected(sv):
