@@ -226,6 +226,23 @@ SV_API sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv_kv 
                          void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
 
 /*
+ * sv_verify_attn for a layer that reuses a block list selected by an earlier layer (Section 3.3, Eq. 9: a
+ * non-anchor layer takes the preceding anchor's blocks, so nothing has to be retrieved before it attends).
+ * Same arguments and results.  The caller vouches that nothing the gather reads -- sel_idx, sel_cnt,
+ * block_table, seq_lens and the K/V pools -- is written by the kernel that immediately precedes this call in the
+ * stream (q, draft_k, draft_v and parent may be).  The kernels of this library are chained by programmatic
+ * dependent launch, so the call's thread blocks are resident while that kernel drains; with the promise they
+ * walk the list and request the K/V tiles at once instead of waiting for it to finish, and the tiles are in
+ * shared memory when the queries may be read.  Without the promise (a list written by sv_select_blocks just
+ * before) use sv_verify_attn.  Dense verification (sel_idx == NULL) qualifies when seq_lens is not written by the
+ * preceding kernel.
+ */
+SV_API sv_status sv_verify_attn_reused(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                                const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                                const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
+                                void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
+
+/*
  * sv_verify_attn for callers that cannot provide or allocate a workspace.  (The paper has no
  * counterpart: this is a packaging variant of sv_verify_attn, not another operation.)
  *

@@ -9,5 +9,5 @@ from .binding import (EXPORTS, LIB_PATH, SV_NOALLOC_SCRATCH_BYTES, SV_OK, SV_STA
                       sv_block_reps, sv_block_reps_bf16, sv_budget_blocks, sv_geom, sv_kv, sv_kv_append,
                       sv_pick_anchors, sv_select_blocks, sv_select_blocks_bf16reps, sv_select_blocks_global,
                       sv_select_blocks_tokens, sv_status_word_check, sv_token_overlap, sv_verify_attn,
-                      sv_verify_attn_noalloc, sv_verify_attn_splits, sv_workspace_bytes)
+                      sv_verify_attn_noalloc, sv_verify_attn_reused, sv_verify_attn_splits, sv_workspace_bytes)
 from .engine import SparseVerifier  # noqa: F401

@@ -25,7 +25,7 @@ SV_STATUS_WAIT_MASK, SV_STATUS_INDEX, SV_STATUS_NO_LIST = 0x0FF, 0x100, 0x200
 SV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # size of the library's built-in scratch (sv_verify_attn_noalloc)
 
 EXPORTS = ("sv_strerror", "sv_status_word_check", "sv_budget_blocks", "sv_workspace_bytes", "sv_block_reps", "sv_select_blocks",
-           "sv_verify_attn", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
+           "sv_verify_attn", "sv_verify_attn_reused", "sv_verify_attn_splits", "sv_verify_attn_noalloc", "sv_kv_append", "sv_anchor_jaccard", "sv_pick_anchors",
            "sv_select_blocks_tokens", "sv_token_overlap", "sv_select_blocks_global", "sv_accept",
            "sv_block_reps_bf16", "sv_select_blocks_bf16reps")
 
@@ -71,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.sv_select_blocks.argtypes = [gp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
     lib.sv_verify_attn.restype = ctypes.c_int
     lib.sv_verify_attn.argtypes = [gp, vp, kp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp, vp]
+    lib.sv_verify_attn_reused.restype = ctypes.c_int
+    lib.sv_verify_attn_reused.argtypes = lib.sv_verify_attn.argtypes
     lib.sv_anchor_jaccard.restype = ctypes.c_int
     lib.sv_anchor_jaccard.argtypes = [gp, i32, vp, vp, i32, vp, vp, vp]
     lib.sv_pick_anchors.restype = ctypes.c_int
@@ -189,18 +191,27 @@ def sv_select_blocks(geom: sv_geom, q, reps, seq_lens, budget_blocks, n_sink: in
 
 
 def sv_verify_attn(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=None,
-                   workspace=None, softmax_scale: float = 0.0, status_word=None, stream=None) -> None:
+                   workspace=None, softmax_scale: float = 0.0, status_word=None, stream=None, _fn=None, _name="sv_verify_attn") -> None:
     max_sel = int(sel_idx.shape[-1]) if sel_idx is not None else int(geom.max_blocks)
     ws_ptr = workspace.data_ptr() if workspace is not None else None
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     if workspace is not None and not workspace.is_cuda:
         raise TypeError("workspace must be a CUDA tensor")
-    _check(_lib.sv_verify_attn(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), ctypes.byref(kv),
+    _check((_fn or _lib.sv_verify_attn)(ctypes.byref(geom), _ptr(q, torch.bfloat16, "q"), ctypes.byref(kv),
                                _ptr(draft_k, torch.bfloat16, "draft_k"), _ptr(draft_v, torch.bfloat16, "draft_v"),
                                _ptr(parent, torch.int32, "parent"), _ptr(sel_idx, torch.int32, "sel_idx"),
                                _ptr(sel_cnt, torch.int32, "sel_cnt"), max_sel, float(softmax_scale),
                                _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"), ws_ptr, ws_bytes,
-                               _ptr(status_word, torch.int32, "status_word"), _stream(stream)), "sv_verify_attn")
+                               _ptr(status_word, torch.int32, "status_word"), _stream(stream)), _name)
+
+
+def sv_verify_attn_reused(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=None,
+                          workspace=None, softmax_scale: float = 0.0, status_word=None, stream=None) -> None:
+    """sv_verify_attn for a layer that reuses an earlier layer's block list: the caller vouches that the list, the tables,
+    the lengths and the K/V pools are not written by the kernel just before, and the gather starts ahead of it."""
+    sv_verify_attn(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=lse, workspace=workspace,
+                   softmax_scale=softmax_scale, status_word=status_word, stream=stream, _fn=_lib.sv_verify_attn_reused,
+                   _name="sv_verify_attn_reused")
 
 
 def sv_verify_attn_noalloc(geom: sv_geom, q, kv: sv_kv, draft_k, draft_v, parent, sel_idx, sel_cnt, out, lse=None,

@@ -31,6 +31,7 @@ struct AttnParams {
     float scale_log2;
     int Tt, tiles;   // draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
     int n_pages;     // pages in each pool: page ids from the block table are clamped to it
+    int early_gather;   // 1: nothing the gather reads comes from the kernel just before; it starts ahead of the dependency wait
 };
 
 // tcgen05 / TMEM attention kernel (verify_attn_tc.cu): rows = G*T <= 128 packed as one M=128 tile.

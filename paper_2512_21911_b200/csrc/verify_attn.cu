@@ -200,7 +200,8 @@ extern "C" size_t sv_workspace_bytes(const sv_geom *geom, int32_t max_sel)
 static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
                                   const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
                                   const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out, float *lse,
-                                  void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream, bool balance)
+                                  void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream, bool balance,
+                                  bool early_gather = false)
 {
     sv_status st = svh::check_geom(geom);
     if (st != SV_OK) return st;
@@ -246,6 +247,7 @@ static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_k
     p.NBmax = geom->max_blocks, p.max_sel = max_sel, p.splits = splits;
     p.Tt = svh::tokens_per_tile(geom), p.tiles = svh::row_tiles(geom);
     p.n_pages = kv->n_pages;
+    p.early_gather = early_gather ? 1 : 0;
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;   // 1/sqrt(128)
     p.scale_log2 = scale * 1.4426950408889634f;
 
@@ -277,6 +279,16 @@ extern "C" sv_status sv_verify_attn(const sv_geom *geom, const void *q, const sv
 {
     return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
                             workspace, workspace_bytes, status_word, stream, true);
+}
+
+extern "C" sv_status sv_verify_attn_reused(const sv_geom *geom, const void *q, const sv_kv *kv, const void *draft_k,
+                                           const void *draft_v, const int32_t *parent, const int32_t *sel_idx,
+                                           const int32_t *sel_cnt, int32_t max_sel, float softmax_scale, void *out,
+                                           float *lse, void *workspace, size_t workspace_bytes, int32_t *status_word,
+                                           void *stream)
+{
+    return verify_attn_impl(geom, q, kv, draft_k, draft_v, parent, sel_idx, sel_cnt, max_sel, softmax_scale, out, lse,
+                            workspace, workspace_bytes, status_word, stream, true, true);
 }
 
 // ---------------------------------------------------------------------- sv_verify_attn_noalloc

@@ -160,7 +160,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint64_t policy = policy_evict_first();
             // pull this sequence's block-table row towards L2 while the previous kernel drains
             for (int i = lane * 32; i < p.NBmax; i += 32 * 32) prefetch_l2(p.block_table + (size_t)s * p.NBmax + i);
-            grid_dependency_wait();   // the block list is written by the kernel just before
+            // The block list is normally written by the kernel just before.  When the caller vouches that neither the
+            // list nor the tables, lengths and pools come from that kernel (a layer that reuses an earlier layer's
+            // list), the gather starts at once, while that kernel drains: the tiles are in shared memory by the time
+            // the queries, which do come from it, may be read.
+            if (!p.early_gather) grid_dependency_wait();
             // First batch of block indices speculatively, assuming the list is full (cnt == max_sel): its
             // load then overlaps the loads of the count and the length instead of following them.
             const int j0_spec = slice_begin(split, p.max_sel);

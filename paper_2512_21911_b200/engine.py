@@ -69,16 +69,21 @@ class SparseVerifier:
         """(Re)compute block representatives of a layer; a decoding loop only refreshes the tail block."""
         sv.sv_block_reps(self.geom, self.kv[layer], self.reps[layer], block_begin, block_end)
 
-    def verify_layer(self, layer: int, q, draft_k, draft_v, out, lse=None) -> None:
-        """select (anchor) or reuse (non-anchor), then sparse verification attention, on the current stream."""
+    def verify_layer(self, layer: int, q, draft_k, draft_v, out, lse=None, behind_own_layer: bool = False) -> None:
+        """select (anchor) or reuse (non-anchor), then sparse verification attention, on the current stream.
+
+        behind_own_layer: the kernel just before this call in the stream is the preceding layer's attention / merge
+        (as inside verify_step), which writes neither the block list nor the cache: a layer that reuses the list
+        then starts its gather while that kernel drains (sv_verify_attn_reused)."""
         if self.anchors[layer]:
             sv.sv_select_blocks(self.geom, q, self.reps[layer], self.seq_lens, self.budget, self.n_sink,
                                 self.n_local, self.sel_idx, self.sel_cnt)
         else:   # Eq. 9: same list as the preceding layer; in place, so nothing is launched
             sv.sv_select_blocks(self.geom, None, None, None, None, self.n_sink, self.n_local, self.sel_idx,
                                 self.sel_cnt, reuse_prev=True, prev_idx=self.sel_idx, prev_cnt=self.sel_cnt)
-        sv.sv_verify_attn(self.geom, q, self.kv[layer], draft_k, draft_v, self.parent, self.sel_idx, self.sel_cnt,
-                          out, lse=lse, workspace=self.workspace, status_word=self.status)
+        attn = sv.sv_verify_attn_reused if (behind_own_layer and not self.anchors[layer]) else sv.sv_verify_attn
+        attn(self.geom, q, self.kv[layer], draft_k, draft_v, self.parent, self.sel_idx, self.sel_cnt, out, lse=lse,
+             workspace=self.workspace, status_word=self.status)
 
     def dense_layer(self, layer: int, q, draft_k, draft_v, out, lse=None) -> None:
         """Dense ("strict") verification attention over every cached block, for comparison."""
@@ -102,7 +107,7 @@ class SparseVerifier:
                     if self.anchors[l]:
                         sv.sv_block_reps(self.geom, self.kv[l], self.reps[l], sv.SV_TAIL_BLOCK)
         for l in range(self.n_layers):
-            self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l])
+            self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l], behind_own_layer=l > 0)
 
     def accept(self, p_target, p_draft, tokens, u_accept, u_next):
         """Acceptance of the step's draft tokens (Eq. 2-3).  Returns (path [S][T], n_path [S], next_token [S]):

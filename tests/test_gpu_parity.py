@@ -281,6 +281,36 @@ def test_reuse_prev_copies_previous_layer(sv):
         sv.sv_select_blocks(d.geom, None, None, None, None, 1, 1, idx2, cnt2, reuse_prev=True)
 
 
+@pytest.mark.parametrize("name", ["cfg1_small", "cfg3_small", "t60_tree", "rows4"])
+def test_reused_list_variant_matches_oracle(sv, name):
+    """sv_verify_attn_reused (the gather starts ahead of the dependency wait; for layers that reuse a list, Eq. 9):
+    same results as the oracle on a list written well before the call, sparse and dense, called back to back so that
+    each call's gather overlaps the previous call's tail."""
+    c = si.make_layer(si.make_geometry(SMALL[name]), sharp=True)
+    d = Dev(sv, c)
+    idx, cnt, _ = gpu_select(sv, d, c["n_sink"], c["n_local"], c["max_sel"])
+    torch.cuda.synchronize()
+    idx_ref, cnt_ref, _ = oracle_select(c, c["n_sink"], c["n_local"], c["max_sel"])
+    w = d.w
+    ws = torch.empty(max(16, sv.sv_workspace_bytes(d.geom, c["max_blocks"])), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    outs = [torch.full((w.n_seq, w.n_draft, w.n_q_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+            for _ in range(4)]
+    lses = [torch.full((w.n_seq, w.n_draft, w.n_q_heads), float("nan"), device="cuda") for _ in range(4)]
+    for k in range(4):      # sparse, dense, sparse, dense
+        sparse = k % 2 == 0
+        sv.sv_verify_attn_reused(d.geom, d.q, d.kv, d.draft_k, d.draft_v, d.parent, idx if sparse else None,
+                                 cnt if sparse else None, outs[k], lse=lses[k], workspace=ws, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o_ref, lse_ref = oracle_attn(c, idx_ref, cnt_ref)
+    o_dense, lse_dense = oracle.dense_verify_attn(c["q"], c["k_pool"], c["v_pool"], c["block_table"], c["seq_lens"],
+                                                  c["draft_k"], c["draft_v"], c["parent"])
+    for k in range(4):
+        ref = (o_ref, lse_ref) if k % 2 == 0 else (o_dense, lse_dense)
+        check_attn(bf16_host(outs[k]), lses[k].cpu().numpy().astype(np.float64), ref[0], ref[1], f"reused {name} call {k}")
+
+
 def test_block_reps_range_update(sv):
     """Only the requested block range is rewritten (a decoding loop refreshes the tail block only)."""
     w = si.shrink(si.WORKLOADS["cfg2"], n_seq=3, seq_len=(900, 2000), budget_blocks=10)
