@@ -1296,6 +1296,39 @@ def test_pipeline_fuzz_random_shapes(sv):
     assert done >= 25
 
 
+def test_pipeline_fuzz_many_rows(sv):
+    """The same on shapes with more than 128 query rows per KV head or more than 32 draft tokens: one to eight row
+    tiles (served in pairs by one CTA, the last one alone when their number is odd), 64-bit ancestor masks, chain and
+    tree, one split and several."""
+    g = np.random.default_rng(4048)
+    done = 0
+    tiles_seen = set()
+    for trial in range(60):
+        Hkv = int(g.choice([1, 2]))
+        G = int(g.choice([1, 2, 4, 8, 16]))
+        T = int(g.choice([20, 33, 40, 47, 60, 64]))
+        if G * T <= 128 and T <= 32:
+            continue
+        B = int(g.choice([64, 128]))
+        S = int(g.integers(1, 3))
+        lo = int(g.integers(3 * B, 10 * B))
+        hi = lo + int(g.integers(0, 6 * B))
+        n_sink, n_local = int(g.integers(0, 2)), int(g.integers(0, 3))
+        nb_min = (lo + B - 1) // B
+        budget = int(g.integers(max(1, n_sink + n_local), nb_min + 2))
+        w = si.Workload(f"wide{trial}", S, (lo, hi), Hkv * G, Hkv, 128, B, budget, T, bool(g.integers(0, 2)), 1,
+                        max(1, min(2, budget - n_sink - n_local)), 7000 + trial, n_sink, n_local)
+        tt = T if G * T <= 128 else max(1, 128 // G)
+        tiles_seen.add(-(-T // tt))
+        geom = si.make_geometry(w)
+        c = si.make_layer(geom, sharp=bool(trial & 1))
+        run_pipeline(sv, c, what=f"wide {trial}: S={S} Hkv={Hkv} G={G} T={T} B={B} L={lo}..{hi} N={budget} sink={n_sink} local={n_local}")
+        done += 1
+        if done >= 24 and {1, 2, 3}.issubset(tiles_seen) and max(tiles_seen) >= 5:
+            break
+    assert done >= 20 and {1, 2, 3}.issubset(tiles_seen) and max(tiles_seen) >= 5, (done, tiles_seen)
+
+
 def test_accept_fuzz(sv):
     """Acceptance walk on random small cases: trees with several siblings per row, every draft length, vocabularies that
     leave ragged per-thread segments, draft models from identical to unrelated."""
