@@ -32,6 +32,18 @@ def test_exports_every_declared_symbol(svb):
         assert hasattr(lib, name), name
 
 
+def test_exports_nothing_else(svb):
+    """The library's dynamic symbol table holds the entry points of sv.h and nothing more (no development hooks)."""
+    import shutil
+    import subprocess
+    nm = shutil.which("nm")
+    if nm is None:
+        pytest.skip("binutils nm not available")
+    out = subprocess.run([nm, "-D", "--defined-only", svb.LIB_PATH], capture_output=True, text=True, check=True).stdout
+    names = {line.split()[-1] for line in out.splitlines() if line.strip()}
+    assert names == set(svb.EXPORTS), names ^ set(svb.EXPORTS)
+
+
 def test_strerror_texts(svb):
     texts = {svb._strerror(i) for i in range(10)}
     assert len(texts) == 10 and "ok" in texts and "unknown status" not in texts
