@@ -13,6 +13,8 @@
  *                     last few; or reuse the previous layer's set  (Eq. 5, Eq. 9)
  *   sv_verify_attn    attention of all draft tokens over the kept blocks
  *                     and the draft tokens' own K/V                       (Fig. 1)
+ *   sv_verify_attn_reused   the same for a layer that reuses an earlier
+ *                     layer's block list                                  (Eq. 9)
  *   sv_kv_append      commit of the accepted draft tokens to the cache, with
  *                     the representatives of the grown blocks refreshed (Section 2.1)
  *   sv_accept         acceptance of the draft tokens after verification (Eq. 2-3)
@@ -29,7 +31,11 @@
  *   - Tensor bases must be 16-byte aligned (the K/V pools 128-byte aligned).
  *   - bf16 tensors are passed as const void*.
  *   - Arguments are validated on the host; a bad argument returns an sv_status
- *     and launches nothing.  A failed launch returns SV_ERR_CUDA.
+ *     and launches nothing.  A failed launch returns SV_ERR_CUDA.  What only the
+ *     device can see (an index outside its table, a wait that gave up) goes to
+ *     the optional device status word, see sv_status_word_check.
+ *   - One process may use the library on several devices (per-device state is
+ *     kept by device index); a call works on the current device.
  *   - head_dim must be 128; block_size 64 or 128; n_q_heads a multiple of
  *     n_kv_heads; query head hq uses KV head hq / (n_q_heads / n_kv_heads).
  */
