@@ -609,6 +609,7 @@ def run_sweep(args):
                 ws = torch.zeros(max(16, sv.sv_workspace_bytes(geom, N)), dtype=torch.uint8, device=dev)
                 if not dense:
                     sv.sv_select_blocks(geom, q, reps[0], sl, bud, 1, 1, idx, cnt)
+                torch.cuda.synchronize()   # the timed calls run on another stream
 
                 def attn_all():
                     for kv in kvs:
@@ -650,9 +651,10 @@ def run_sweep(args):
 
 
 def run_configs(args):
-    """--configs: timing lines for the two other full-size configurations (their parity is covered by the tests):
-    the 16-sequence batch with ragged prefixes (block 64, 2048-token budget, 5 draft tokens as a chain) and the
-    4 x 131072-token long-context case (GQA 8, block 128, 4096-token budget, 16-node draft tree).  K/V are seeded
+    """--configs: timing lines for the other full-size configurations (their parity is covered by the tests):
+    the 16-sequence batch with ragged prefixes (block 64, 2048-token budget, 5 draft tokens as a chain), the
+    4 x 131072-token long-context case (GQA 8, block 128, 4096-token budget, 16-node draft tree), and 60-token
+    draft trees on Llama-3.1-8B geometry (240 query rows per KV head), one sequence and a batch of 12.  K/V are seeded
     device-side N(0, 1/128) tensors, lengths / page tables / the tree come from seeded host generators, the block
     lists from sv_select_blocks.  Each configuration rotates over independent KV replicas so that at least 256 MiB
     is gathered between two uses of a replica (HBM, not L2).  One JSON line per configuration."""
@@ -668,7 +670,10 @@ def run_configs(args):
              ("cfg3", dict(S=4, Hq=64, Hkv=8, B=128, lens=(131072, 131072), budget_tokens=4096, T=16, tree=True, seed=1003)),
              # the paper's own verification shape (Section 2.2, set-up of Section 4.1): a 60-token draft tree on
              # Llama-3.1-8B geometry (240 query rows per KV head), budget from Eq. 6 with rho = 0.1 and L0 = 4K
-             ("tree60", dict(S=1, Hq=32, Hkv=8, B=64, lens=(32768, 32768), budget_tokens=None, T=60, tree=True, seed=1060))]
+             ("tree60", dict(S=1, Hq=32, Hkv=8, B=64, lens=(32768, 32768), budget_tokens=None, T=60, tree=True, seed=1060)),
+             # a batch of such trees on ragged prefixes: 12 x 8 x 2 row tiles just miss fitting the SMs once, the case
+             # in which one CTA serves a pair of row tiles
+             ("tree60_batch", dict(S=12, Hq=32, Hkv=8, B=64, lens=(6000, 10000), budget_tokens=None, T=60, tree=True, seed=1061))]
     if args.only:
         cases = [c for c in cases if c[0] in args.only.split(",")]
     for name, c in cases:
@@ -715,6 +720,7 @@ def run_configs(args):
         ws = torch.zeros(max(16, sv.sv_workspace_bytes(geom, NB)), dtype=torch.uint8, device=dev)
         status = torch.zeros(1, dtype=torch.int32, device=dev)
         sv.sv_select_blocks(geom, q, reps[0], sl, bud, 1, 1, idx, cnt)
+        torch.cuda.synchronize()   # the timed calls run on another stream
 
         def sel_all():
             for r in reps:

@@ -30,6 +30,7 @@ struct AttnParams {
     int T, Hq, Hkv, G, B, NBmax, max_sel, splits;
     float scale_log2;
     int Tt, tiles;   // draft tokens per row tile (G * Tt <= 128 query rows) and number of row tiles
+    int pair;        // 1: a CTA serves two row tiles (grid.x = splits x ceil(tiles / 2)); 0: one (grid.x = splits x tiles)
     int n_pages;     // pages in each pool: page ids from the block table are clamped to it
     int early_gather;   // 1: nothing the gather reads comes from the kernel just before; it starts ahead of the dependency wait
 };

@@ -29,13 +29,6 @@ inline int row_tiles(const sv_geom *g)
     return (g->n_draft + tt - 1) / tt;
 }
 
-// CTAs per (sequence, KV head, split): one per row tile, or one per pair of row tiles when there are several (a CTA
-// then serves two tiles from one gather of the kept K/V)
-inline int row_groups(const sv_geom *g)
-{
-    const int t = row_tiles(g);
-    return t > 1 ? (t + 1) / 2 : 1;
-}
 
 inline sv_status check_geom(const sv_geom *g)
 {
@@ -114,6 +107,28 @@ inline int sm_count()
     }
     if (cached) count[dev].store(v, std::memory_order_relaxed);
     return v;
+}
+
+// CTAs per (sequence, KV head, split): one per row tile, or one per pair of row tiles (a CTA then serves both tiles
+// from one gather, each softmax warpgroup taking every unit for its own tile).  One per tile is the default: the CTAs
+// that share a slice of the blocks sit next to each other in the grid, request the same K/V tiles at about the same
+// time, and all but the first find them in L2 (240 rows, one sequence: 29.6 MB from DRAM for 29.8 MB algorithmic), and
+// the finer CTAs fill the SMs better (20.0 against 22.9 us there).  A paired CTA takes 16/9 as long as a single-tile
+// one (batches of 240-row trees: 100 against 56 us per wave of CTAs), so pairs are used where they save enough waves
+// to pay for that -- in practice when the row-tile CTAs just miss fitting the SMs once (10 to 16 such sequences of 8
+// KV heads: 100 against 112 us).
+inline bool pair_row_tiles(const sv_geom *g)
+{
+    const int t = row_tiles(g);
+    if (t < 2) return false;
+    const long long pairs = (long long)g->n_seq * g->n_kv_heads, sms = sm_count();
+    const long long waves_tile = (pairs * t + sms - 1) / sms, waves_pair = (pairs * ((t + 1) / 2) + sms - 1) / sms;
+    return 16 * waves_pair < 9 * waves_tile;
+}
+inline int row_groups(const sv_geom *g)
+{
+    const int t = row_tiles(g);
+    return pair_row_tiles(g) ? (t + 1) / 2 : t;
 }
 
 inline sv_status launch_status()

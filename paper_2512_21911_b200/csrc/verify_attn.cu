@@ -246,6 +246,7 @@ static sv_status verify_attn_impl(const sv_geom *geom, const void *q, const sv_k
     p.T = geom->n_draft, p.Hq = geom->n_q_heads, p.Hkv = geom->n_kv_heads, p.G = G, p.B = geom->block_size;
     p.NBmax = geom->max_blocks, p.max_sel = max_sel, p.splits = splits;
     p.Tt = svh::tokens_per_tile(geom), p.tiles = svh::row_tiles(geom);
+    p.pair = svh::pair_row_tiles(geom) ? 1 : 0;
     p.n_pages = kv->n_pages;
     p.early_gather = early_gather ? 1 : 0;
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.08838834764831845f;   // 1/sqrt(128)

@@ -68,8 +68,8 @@ enum Bar {
 // common case keeps split = blockIdx.x, plain row arithmetic and 32-bit masks: deriving the split from a division
 // costs 3 % on long loops, and the wider mask code 7 % at 128 rows.
 // kPair (with kWide, NH = 4): the CTA serves two row tiles of its (sequence, KV head) from one gather: warpgroup w owns
-// row tile 2 * pair + w -- its own Q tile, S / P / O buffers -- and takes every unit instead of every other one, so the
-// kept K/V cross HBM once per pair of tiles (240 query rows, a 60-token draft tree on a GQA-4 model: once in all).
+// row tile 2 * pair + w -- its own Q tile, S / P / O buffers -- and takes every unit instead of every other one.  The
+// host chooses it where it saves enough waves of CTAs (svh::pair_row_tiles).
 template <int NH, bool kWide, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
     verify_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -805,13 +805,13 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
     return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide, kPair>, tm_k, tm_v, p);
 }
 
-// grid.x = splits x groups, where a group is a row tile or, with more than one row tile, a pair of them
+// grid.x = splits x groups, where a group is a row tile or (p.pair) a pair of row tiles
 cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                            cudaStream_t stream)
 {
     const int rows = p.G * p.Tt;   // rows of a full row tile
-    if (p.tiles > 1) return launch_tc<4, true, true>(tm_k, tm_v, p, grid, stream);   // (a full tile has more than 64 rows)
-    if (p.T > 32) {
+    if (p.pair) return launch_tc<4, true, true>(tm_k, tm_v, p, grid, stream);   // (a full tile has more than 64 rows)
+    if (p.tiles > 1 || p.T > 32) {
         if (rows <= 32) return launch_tc<1, true, false>(tm_k, tm_v, p, grid, stream);
         if (rows <= 64) return launch_tc<2, true, false>(tm_k, tm_v, p, grid, stream);
         return launch_tc<4, true, false>(tm_k, tm_v, p, grid, stream);

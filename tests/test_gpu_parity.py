@@ -165,8 +165,12 @@ SMALL = {
     "t40_chain_2seq": si.shrink(si.WORKLOADS["cfg2"], n_seq=2, seq_len=(900, 2100), budget_blocks=7, n_draft=40, planted=2),
     "g8_t24_b128": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(2000, 4000), budget_blocks=6, n_draft=24, planted=2),
     "g16_t64": si.shrink(si.WORKLOADS["cfg0"], n_q_heads=32, n_kv_heads=2, seq_len=(1100, 1100), budget_blocks=5, n_draft=64, tree=True, planted=2),
-    # an odd number of row tiles (3 x 128 rows: 16 + 16 + 8 draft tokens): the last CTA group serves a single tile
+    # an odd number of row tiles (3 x 128 rows: 16 + 16 + 8 draft tokens), one CTA per row tile
     "g8_t40_tree_3tiles": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(1800, 3100), budget_blocks=6, n_draft=40, planted=2),
+    # more row-tile CTAs than SMs: one CTA serves a pair of row tiles from one gather (2 tiles: 10 x 8 x 2 = 160 CTAs
+    # otherwise; 3 tiles, the last pair holding one: 7 x 8 x 3 = 168)
+    "t24_tile_pairs": si.shrink(si.WORKLOADS["cfg3"], n_seq=10, seq_len=(700, 1900), budget_blocks=5, n_draft=24, planted=2),
+    "t40_tree_tile_pairs_odd": si.shrink(si.WORKLOADS["cfg3"], n_seq=7, seq_len=(600, 1500), budget_blocks=4, n_draft=40, tree=True, planted=1),
     # more (sequence, KV head) pairs than SMs: several waves of CTAs, one split each
     "many_seqs": si.shrink(si.WORKLOADS["cfg2"], n_seq=40, seq_len=(300, 1100), budget_blocks=6, planted=1),
     "b128_short_tail": si.shrink(si.WORKLOADS["cfg3"], n_seq=2, seq_len=(128 * 9 + 30, 128 * 9 + 30), n_q_heads=16, n_kv_heads=4,
@@ -1298,10 +1302,12 @@ def test_pipeline_fuzz_random_shapes(sv):
 
 def test_pipeline_fuzz_many_rows(sv):
     """The same on shapes with more than 128 query rows per KV head or more than 32 draft tokens: one to eight row
-    tiles (served in pairs by one CTA, the last one alone when their number is odd), 64-bit ancestor masks, chain and
-    tree, one split and several."""
+    tiles, 64-bit ancestor masks, chain and tree, one split and several; every third case has enough sequences that the
+    row-tile CTAs outnumber the SMs, where one CTA serves a pair of row tiles (the last one alone when their number is
+    odd)."""
     g = np.random.default_rng(4048)
-    done = 0
+    done = paired = 0
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
     tiles_seen = set()
     for trial in range(60):
         Hkv = int(g.choice([1, 2]))
@@ -1311,22 +1317,27 @@ def test_pipeline_fuzz_many_rows(sv):
             continue
         B = int(g.choice([64, 128]))
         S = int(g.integers(1, 3))
-        lo = int(g.integers(3 * B, 10 * B))
-        hi = lo + int(g.integers(0, 6 * B))
+        tt = T if G * T <= 128 else max(1, 128 // G)
+        tiles = -(-T // tt)
+        many = trial % 3 == 2 and tiles > 1
+        if many:
+            S = n_sm // (Hkv * tiles) + int(g.integers(1, 4))
+            paired += 1
+        lo = int(g.integers(3 * B, (5 if many else 10) * B))
+        hi = lo + int(g.integers(0, (3 if many else 6) * B))
         n_sink, n_local = int(g.integers(0, 2)), int(g.integers(0, 3))
         nb_min = (lo + B - 1) // B
         budget = int(g.integers(max(1, n_sink + n_local), nb_min + 2))
         w = si.Workload(f"wide{trial}", S, (lo, hi), Hkv * G, Hkv, 128, B, budget, T, bool(g.integers(0, 2)), 1,
                         max(1, min(2, budget - n_sink - n_local)), 7000 + trial, n_sink, n_local)
-        tt = T if G * T <= 128 else max(1, 128 // G)
-        tiles_seen.add(-(-T // tt))
+        tiles_seen.add(tiles)
         geom = si.make_geometry(w)
         c = si.make_layer(geom, sharp=bool(trial & 1))
         run_pipeline(sv, c, what=f"wide {trial}: S={S} Hkv={Hkv} G={G} T={T} B={B} L={lo}..{hi} N={budget} sink={n_sink} local={n_local}")
         done += 1
-        if done >= 24 and {1, 2, 3}.issubset(tiles_seen) and max(tiles_seen) >= 5:
+        if done >= 27 and paired >= 6 and {1, 2, 3}.issubset(tiles_seen) and max(tiles_seen) >= 5:
             break
-    assert done >= 20 and {1, 2, 3}.issubset(tiles_seen) and max(tiles_seen) >= 5, (done, tiles_seen)
+    assert done >= 20 and paired >= 5 and {1, 2, 3}.issubset(tiles_seen) and max(tiles_seen) >= 5, (done, paired, tiles_seen)
 
 
 def test_accept_fuzz(sv):
