@@ -105,8 +105,9 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// Tensor map over a pool viewed as a 2-D bf16 matrix [n_pages*Hkv*B rows][128 cols]; box = 64 rows x 64 cols
-// (128 bytes wide, 128-byte swizzle).  Encoding costs microseconds of host time, so maps are kept in a
+// Tensor map over a pool viewed as a bf16 tensor [2 column halves][n_pages*Hkv*B rows][64 cols] (the halves 128 bytes
+// apart inside a 256-byte row); box = 2 halves x 64 rows x 64 cols (128 bytes wide, 128-byte swizzle), so that one copy
+// brings a 64-row unit as the two half tiles the tensor cores read.  Encoding costs microseconds of host time, so maps are kept in a
 // small fixed table keyed by (pool, rows) (no heap use; a full table is overwritten round-robin).
 bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
 {
@@ -127,12 +128,12 @@ bool pool_tensor_map(const void *pool, int64_t n_rows, CUtensorMap *out)
         }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {128, (cuuint64_t)n_rows};
-    const cuuint64_t strides[1] = {256};
-    const cuuint32_t box[2] = {64, kUnit};
-    const cuuint32_t estr[2] = {1, 1};
+    const cuuint64_t dims[3] = {64, (cuuint64_t)n_rows, 2};
+    const cuuint64_t strides[2] = {256, 128};
+    const cuuint32_t box[3] = {64, kUnit, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMap tm;
-    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
+    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims, strides, box, estr,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;

@@ -220,10 +220,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                             // an empty unit (block 128, tail of at most 64 tokens) is still loaded:
                             // it keeps the unit sequence uniform and is fully masked downstream
                             mbar_arrive_expect_tx(fb, kStageBytes);
-                            tma_load_2d(dst, &tm_k, 0, y, fb, policy);
-                            tma_load_2d(dst + kTile, &tm_k, 64, y, fb, policy);
-                            tma_load_2d(dst + 2 * kTile, &tm_v, 0, y, fb, policy);
-                            tma_load_2d(dst + 3 * kTile, &tm_v, 64, y, fb, policy);
+                            // one copy per operand: the box spans both 64-column halves (third coordinate), which
+                            // land as two consecutive [64 rows][128 bytes] swizzled tiles
+                            tma_load_3d(dst, &tm_k, 0, y, 0, fb, policy);
+                            tma_load_3d(dst + 2 * kTile, &tm_v, 0, y, 0, fb, policy);
                         }
                     }
                 }
