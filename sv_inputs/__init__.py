@@ -85,6 +85,11 @@ WORKLOADS = {
     "cfg2": Workload("cfg2", 16, (4096, 16384), 32, 8, 128, 64, 32, 5, False, 1, 0.05, 1002),
     # long context, GQA 8, 16-node draft tree, 4096-token budget
     "cfg3": Workload("cfg3", 4, (131072, 131072), 64, 8, 128, 128, 32, 16, True, 1, 0.02, 1003),
+    # the paper's verification shape (Section 2.2, Section 4.1): a 60-node draft tree on Llama-3.1-8B geometry, 240 query
+    # rows per KV head; the budgets are Eq. 6 with rho = 0.1, L0 = 4K at 32768 and at 10000 cached tokens.  Alone, and
+    # as a batch of 12 on ragged prefixes.
+    "tree60": Workload("tree60", 1, (32768, 32768), 32, 8, 128, 64, 109, 60, True, 1, 0.05, 1060),
+    "tree60_batch": Workload("tree60_batch", 12, (6000, 10000), 32, 8, 128, 64, 74, 60, True, 1, 0.05, 1061),
 }
 
 

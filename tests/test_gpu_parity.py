@@ -481,6 +481,16 @@ def test_full_size_cfg3_sampled(sv):
     _sampled_check(sv, c, 64, "cfg3")
 
 
+@pytest.mark.parametrize("name", ["tree60", "tree60_batch"])
+def test_full_size_tree60_sampled(sv, name):
+    """The 60-node draft tree on Llama-3.1-8B geometry at full size: alone (two row tiles, one CTA each) and as a batch of
+    12 (one CTA per pair of row tiles); lists bit-exact, attention on sampled rows of both row tiles."""
+    w = si.WORKLOADS[name]
+    assert w.budget_blocks == sv.sv_budget_blocks(max(w.seq_len), 4096, 0.1, 64, 1, 1)
+    c = si.make_layer(si.make_geometry(w), sharp=True)
+    _sampled_check(sv, c, 64, name)
+
+
 @pytest.mark.parametrize("point", [(8192, 1 / 32, 1), (32768, 1 / 8, 16), (131072, 1 / 4, 4)])
 def test_sweep_points(sv, point):
     c = si.make_layer(si.make_geometry(si.sweep_workload(*point)), sharp=True)
