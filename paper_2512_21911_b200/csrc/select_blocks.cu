@@ -2,8 +2,8 @@
 // first draft token's query, then the top-N blocks with the first/last few kept (Section 3.1), in one
 // launch.  reuse_prev copies the previous layer's set (Section 3.3, Eq. 9).
 //
-// One thread-block cluster (up to 8 CTAs) per (sequence, KV head).  Each CTA of the cluster scores a
-// contiguous slice of the blocks (a GEMV over the representatives: one warp per block row, 128-bit loads,
+// One thread-block cluster (up to 8 CTAs; 16 for a few very long block lists) per (sequence, KV head).  Each CTA of
+// the cluster scores a contiguous slice of the blocks (a GEMV over the representatives: one warp per block row, 128-bit loads,
 // several rows in flight per warp), turns the scores into order-preserving 32-bit keys and pushes them
 // straight into CTA 0's shared memory with st.async stores that count their bytes on an mbarrier there;
 // the senders then exit.  CTA 0 waits (bounded) for the expected byte count and selects exactly: the
@@ -181,6 +181,38 @@ __global__ void copy_selection_kernel(const int32_t *__restrict__ prev_idx, cons
 
 }  // namespace
 
+// Whether this device can hold clusters of 16 CTAs of the select kernel (asked once per device and instantiation).
+static bool clusters_of_16_fit(bool reps_bf16)
+{
+    static std::atomic<int> state[2][svh::kMaxDevices];   // 0: not asked, 1: yes, 2: no
+    const int dev = svh::current_device();
+    if (dev < 0 || dev >= svh::kMaxDevices) return false;
+    int v = state[reps_bf16][dev].load(std::memory_order_acquire);
+    if (v == 0) {
+        const void *fn = reps_bf16 ? reinterpret_cast<const void *>(select_kernel<true>)
+                                   : reinterpret_cast<const void *>(select_kernel<false>);
+        v = 2;
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(16, 8, 1);
+            cfg.blockDim = dim3(kThreads);
+            cfg.dynamicSmemBytes = 16 * 128 * sizeof(uint32_t);
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 16;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) == cudaSuccess && n >= 8) v = 1;
+        }
+        (void)cudaGetLastError();   // a refusal is an answer, not an error of the call that asked
+        state[reps_bf16][dev].store(v, std::memory_order_release);
+    }
+    return v == 1;
+}
+
 static sv_status select_impl(const sv_geom *geom, const void *q, const void *reps, bool reps_bf16, const int32_t *seq_lens,
                              const int32_t *budget_blocks, int32_t n_sink, int32_t n_local, int32_t reuse_prev,
                              const int32_t *prev_idx, const int32_t *prev_cnt, int32_t *out_idx, int32_t *out_cnt,
@@ -212,6 +244,10 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     const int pairs = geom->n_seq * geom->n_kv_heads;
     int CL = 1;
     while (CL < 8 && geom->max_blocks / (CL * 2) >= 32 && pairs * CL * 2 <= 2 * svh::sm_count()) CL *= 2;
+    // Few pairs with very long block lists (one sequence of 128K tokens: 8 pairs x 2048 blocks) leave most SMs idle at
+    // 8 CTAs per pair, and reading the representatives (128 KB per CTA) is what the kernel then waits for: clusters of
+    // 16 (beyond the portable size, so the device is asked first whether it can hold them)
+    if (CL == 8 && geom->max_blocks >= 2048 && pairs * 16 <= svh::sm_count() && clusters_of_16_fit(reps_bf16)) CL = 16;
     const int per = (geom->max_blocks + CL - 1) / CL;
     const int chunk = (per + kWarps * kRowsPerIter - 1) / (kWarps * kRowsPerIter) * (kWarps * kRowsPerIter);
 
