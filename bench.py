@@ -413,9 +413,12 @@ def run_gpu(args):
 
     ms_e2e_pipelined = time_e2e(side, 4)
 
-    def time_e2e_serial(steps, warmup):
-        """Copy in, run the step, copy out, one step after the other on one stream: the next step's queries depend on
-        what this step accepts, so a decoding loop cannot overlap the copies of neighbouring steps."""
+    def time_e2e_serial(steps, warmup, g_host):
+        """One step after the other: the next step's queries depend on what this step accepts, so a decoding loop cannot
+        overlap neighbouring steps.  g_host None: copy in, the step graph, copy out, all on one stream.  Otherwise g_host
+        is the graph of SparseVerifier.verify_step_from_host, which moves the same bytes in chunks of a few layers on two
+        side streams inside the step (a chunk's layers start when its inputs have arrived, its outputs leave while the
+        next chunk computes)."""
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         with torch.cuda.stream(stream):
             for i in range(warmup + steps):
@@ -423,6 +426,9 @@ def run_gpu(args):
                     stream.synchronize()
                     barrier()
                     e0.record(stream)
+                if g_host is not None:
+                    g_host.replay()
+                    continue
                 q.copy_(q_h, non_blocking=True)
                 dk.copy_(dk_h, non_blocking=True)
                 dv.copy_(dv_h, non_blocking=True)
@@ -433,7 +439,12 @@ def run_gpu(args):
         barrier()
         return e0.elapsed_time(e1) / steps
 
-    ms_e2e = time_e2e_serial(side, 4)
+    ms_e2e_one_stream = time_e2e_serial(side, 4, None)
+    out_h.zero_()
+    g_host = capture(lambda: eng.verify_step_from_host(q_h, dk_h, dv_h, q, dk, dv, out, out_h,
+                                                       layers_per_chunk=args.e2e_chunk, refresh_tail=True))
+    ms_e2e = time_e2e_serial(side, 4, g_host)
+    assert torch.equal(out_h, out.cpu()), "the host-fed step did not deliver the step's outputs"
     assert int(eng.status.item()) == 0 and int(eng_reuse.status.item()) == 0 and int(eng_chain.status.item()) == 0, \
         "a kernel gave up on a bounded wait"
 
@@ -444,9 +455,9 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps, ms_e2e_pipelined = (
+    ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps, ms_e2e_pipelined, ms_e2e_one_stream = (
         aggregate_over_ranks(x, world, allmax)[0]
-        for x in (ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps, ms_e2e_pipelined))
+        for x in (ms_step, ms_reuse, ms_chain, ms_attn, ms_dense, ms_e2e, ms_reps, ms_e2e_pipelined, ms_e2e_one_stream))
 
     # algorithmic bytes of one sv_verify_attn launch (K+V of the kept tokens and draft tokens, Q in, O out)
     S, T, Hq, Hkv, D, B, N = w.n_seq, w.n_draft, w.n_q_heads, w.n_kv_heads, w.head_dim, w.block_size, w.budget_blocks
@@ -469,9 +480,14 @@ def run_gpu(args):
         "clocks": sampler.summary(),
         "e2e": {"value": ms_e2e * 1e3 / (w.n_layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
-                "note": "per step, one after the other on one stream: Q and draft K/V of all layers copied from pinned host "
-                        "memory, the step, the outputs copied back (a decoding loop cannot overlap neighbouring steps: the "
-                        "next queries depend on this step's acceptance); the KV cache is device-resident state",
+                "note": "steps one after the other (a decoding loop cannot overlap neighbouring steps: the next queries "
+                        "depend on this step's acceptance); every step is one call of SparseVerifier.verify_step_from_host: "
+                        "Q and draft K/V of all layers from pinned host memory, the step, the outputs back to pinned host "
+                        "memory, the copies in chunks of a few layers on two side streams so that all but the first upload "
+                        "and the last download run under the step's kernels; the KV cache is device-resident state",
+                "layers_per_chunk": args.e2e_chunk,
+                "one_stream_value": ms_e2e_one_stream * 1e3 / (w.n_layers * world),
+                "one_stream_note": "the same bytes copied whole before and after the step on the step's own stream",
                 "pipelined_value": ms_e2e_pipelined * 1e3 / (w.n_layers * world),
                 "pipelined_note": "the same copies with two buffer sets and three streams, so that the copies of steps "
                                   "i+1 / i-1 run under the kernels of step i (an upper bound no real loop reaches)"},
@@ -884,6 +900,7 @@ def main():
                     help="instead of the benchmark line: sparse vs dense latency over context x budget x draft length")
     ap.add_argument("--configs", action="store_true",
                     help="timing lines for the batched (16 ragged sequences) and long-context (4 x 128K, tree) configurations")
+    ap.add_argument("--e2e-chunk", type=int, default=4, help="layers per copy chunk of the end-to-end step")
     ap.add_argument("--only", default="", help="with --configs: comma-separated configuration names (profiling aid: no dense pass)")
     ap.add_argument("--variants", action="store_true",
                     help="instead of the benchmark line: timings of the retrieval variants (shared budget, every token)")

@@ -37,6 +37,7 @@ class SparseVerifier:
         self.kv: List[Optional[sv.sv_kv]] = [None] * n_layers
         self._pools = [None] * n_layers   # keep the tensors alive
         self._stack_kv = None
+        self._copy_streams = None
 
     def set_layer_kv(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
         self._pools[layer] = (k_pool, v_pool)
@@ -108,6 +109,50 @@ class SparseVerifier:
                         sv.sv_block_reps(self.geom, self.kv[l], self.reps[l], sv.SV_TAIL_BLOCK)
         for l in range(self.n_layers):
             self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l], behind_own_layer=l > 0)
+
+    def verify_step_from_host(self, q_host, draft_k_host, draft_v_host, q, draft_k, draft_v, out, out_host,
+                              layers_per_chunk: int = 4, refresh_tail: bool = False) -> None:
+        """verify_step with the step's inputs in pinned host memory and its outputs wanted there.  The copies go in chunks
+        of a few layers on two side streams: a chunk's layers start as soon as its inputs have arrived, its outputs leave
+        while the next chunk computes, so only the first upload and the last download are not hidden behind kernels.
+        q/draft_k/draft_v/out are the device staging tensors (shapes as for verify_step); the *_host tensors the pinned
+        ones.  Returns with everything enqueued; the current stream ends behind the last download.  Capturable in a
+        CUDA graph (the side streams fork from and join the current stream)."""
+        main = torch.cuda.current_stream()
+        if self._copy_streams is None:
+            self._copy_streams = (torch.cuda.Stream(device=q.device), torch.cuda.Stream(device=q.device))
+        s_in, s_out = self._copy_streams
+        s_in.wait_stream(main)
+        s_out.wait_stream(main)
+        chunks = [(c0, min(c0 + layers_per_chunk, self.n_layers)) for c0 in range(0, self.n_layers, layers_per_chunk)]
+        arrived = []
+        with torch.cuda.stream(s_in):
+            for c0, c1 in chunks:
+                q[c0:c1].copy_(q_host[c0:c1], non_blocking=True)
+                draft_k[c0:c1].copy_(draft_k_host[c0:c1], non_blocking=True)
+                draft_v[c0:c1].copy_(draft_v_host[c0:c1], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(s_in)
+                arrived.append(ev)
+        if refresh_tail:
+            if self._stack_kv is not None:
+                self.refresh_tail_all()
+            else:
+                for l in range(self.n_layers):
+                    if self.anchors[l]:
+                        sv.sv_block_reps(self.geom, self.kv[l], self.reps[l], sv.SV_TAIL_BLOCK)
+        for (c0, c1), ev in zip(chunks, arrived):
+            main.wait_event(ev)
+            for l in range(c0, c1):
+                # the kernel before a chunk's first layer is not this stream's previous layer alone (the upload joins there)
+                self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l], behind_own_layer=l > c0)
+            done = torch.cuda.Event()
+            done.record(main)
+            s_out.wait_event(done)
+            with torch.cuda.stream(s_out):
+                out_host[c0:c1].copy_(out[c0:c1], non_blocking=True)
+        main.wait_stream(s_in)
+        main.wait_stream(s_out)
 
     def accept(self, p_target, p_draft, tokens, u_accept, u_next):
         """Acceptance of the step's draft tokens (Eq. 2-3).  Returns (path [S][T], n_path [S], next_token [S]):

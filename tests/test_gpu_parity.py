@@ -415,6 +415,27 @@ def test_layer_stack_with_reuse_matches_oracle(sv):
     np.testing.assert_array_equal(eng.sel_idx.cpu().numpy(), ref_sel[2][0])
     assert eng.kernels_per_step() == 2 + 4 * (2 if sv.sv_verify_attn_splits(eng.geom, geom["max_sel"]) > 1 else 1)
 
+    # the same step fed from pinned host memory, its copies in chunks on side streams: the same bits, eagerly and as a graph
+    q_h, dk_h, dv_h = q.cpu().pin_memory(), dk.cpu().pin_memory(), dv.cpu().pin_memory()
+    want = out.cpu()
+    for chunk in (1, 3, 4):
+        q2, dk2, dv2, out2 = torch.zeros_like(q), torch.zeros_like(dk), torch.zeros_like(dv), torch.zeros_like(out)
+        out_h = torch.zeros_like(want).pin_memory()
+        eng.verify_step_from_host(q_h, dk_h, dv_h, q2, dk2, dv2, out2, out_h, layers_per_chunk=chunk)
+        torch.cuda.synchronize()
+        assert torch.equal(out_h, want), chunk
+    side = torch.cuda.Stream()
+    out_h = torch.zeros_like(want).pin_memory()
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            eng.verify_step_from_host(q_h, dk_h, dv_h, q2, dk2, dv2, out2, out_h, layers_per_chunk=2)
+        q2.zero_(), out2.zero_()
+        g.replay()
+        g.replay()
+        side.synchronize()
+    assert torch.equal(out_h, want) and int(eng.status.item()) == 0
+
 
 # ------------------------------------------------------------------ full-size configurations
 
