@@ -70,7 +70,7 @@ enum Bar {
 // kPair (with kWide, NH = 4): the CTA serves two row tiles of its (sequence, KV head) from one gather: warpgroup w owns
 // row tile 2 * pair + w -- its own Q tile, S / P / O buffers -- and takes every unit instead of every other one.  The
 // host chooses it where it saves enough waves of CTAs (svh::pair_row_tiles).
-template <int NH, bool kWide, bool kPair>
+template <int NH, bool kWide, bool kPair, bool kUnitSlices>
 __global__ void __launch_bounds__(kThreads, 1)
     verify_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                           const AttnParams p)
@@ -116,15 +116,25 @@ __global__ void __launch_bounds__(kThreads, 1)
     // First block of split k's slice of a list of n blocks.  With 65-128 rows the draft tokens' unit of the last split
     // costs about as much as three ordinary units (masking 64 columns per thread, a first pass through that code), so
     // there the list is cut as if it were that much longer and the last slice comes out shorter.
+    // kUnitSlices (128 rows, blocks of 128 tokens): the slices are cut at 64-key units instead, so that two neighbouring
+    // splits may share a block (32 blocks over 4 splits: 17 / 17 / 17 / 13 + draft units instead of 16 / 18 / 16 / 14 +
+    // draft); slice_begin then returns a unit.  A compile-time variant because the extra index arithmetic costs the
+    // other shapes 2-4 %.
     // (Up to 64 rows: 32-bit products -- k <= 148 splits, n <= 32768 blocks -- because a 64-bit division here costs every
     // CTA of a short launch 0.3 us before its first load; the 128-row instantiation measured faster with the 64-bit form.)
     auto slice_begin = [&](int k, int n) {
-        if constexpr (NH == 4) {
+        if constexpr (kUnitSlices) {
+            return min(2 * n, (int)((long long)k * (2 * n + 3) / p.splits));
+        } else if constexpr (NH == 4) {
             const int w_draft = (3 + upb - 1) / upb;
             return min(n, (int)((long long)k * (n + w_draft) / p.splits));
         } else {
             return (int)((uint32_t)k * (uint32_t)n / (uint32_t)p.splits);
         }
+    };
+    // units of split k's slice
+    auto slice_units = [&](int k, int n) {
+        return kUnitSlices ? slice_begin(k + 1, n) - slice_begin(k, n) : (slice_begin(k + 1, n) - slice_begin(k, n)) * upb;
     };
     const float inv_g = 1.f / (float)p.G;
     auto div_g = [&](int r) { return (int)(((float)r + 0.5f) * inv_g); };
@@ -169,7 +179,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (!p.early_gather) grid_dependency_wait();
             // First batch of block indices speculatively, assuming the list is full (cnt == max_sel): its
             // load then overlaps the loads of the count and the length instead of following them.
-            const int j0_spec = slice_begin(split, p.max_sel);
+            const int j0_spec = kUnitSlices ? slice_begin(split, p.max_sel) >> 1 : slice_begin(split, p.max_sel);
             int blk_spec = 0;
             if (p.sel_idx && j0_spec + lane < p.max_sel)
                 blk_spec = p.sel_idx[((size_t)s * p.Hkv + h) * p.max_sel + j0_spec + lane];
@@ -180,8 +190,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             // only, and say so
             if (cnt_in < 0 && lane == 0 && p.status) atomicOr(p.status, kStatusNoList);
             const int n_sel = p.sel_idx ? max(0, min(cnt_in, p.max_sel)) : nb;
-            const int j0 = slice_begin(split, n_sel);
-            const int j1 = slice_begin(split + 1, n_sel);
+            // blocks j0 .. j1 - 1 of the list; kUnitSlices: units u0 .. u1 - 1 of the list, which those blocks hold
+            const int u0 = slice_begin(split, n_sel), u1 = slice_begin(split + 1, n_sel);
+            const int j0 = kUnitSlices ? u0 >> 1 : u0, j1 = kUnitSlices ? (u1 + 1) >> 1 : u1;
             const int off = has_draft ? 1 : 0;
             bool dead = false;
             for (int base = j0; base < j1; base += 32) {
@@ -205,8 +216,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const int r0 = __shfl_sync(0xffffffffu, row0, i);
                     const int t0 = __shfl_sync(0xffffffffu, tok0, i);
                     if (lane == 0 && !dead) {
-                        for (int uo = 0; uo < upb; ++uo) {
-                            const int u = (base - j0 + i) * upb + uo;   // ring unit; the draft unit (if any) came first
+                        const int ub = 2 * (base + i);   // (kUnitSlices) first unit of the block
+                        for (int uo = kUnitSlices ? max(0, u0 - ub) : 0; uo < (kUnitSlices ? min(2, u1 - ub) : upb); ++uo) {
+                            // ring unit; the draft unit (if any) came first
+                            const int u = kUnitSlices ? ub + uo - u0 : (base - j0 + i) * upb + uo;
                             const int stage = (u + off) % NS, it = (u + off) / NS;
                             if (it > 0 && (*abort_flag || !mbar_wait_bounded(bar(kEmpty + stage), (it - 1) & 1))) {
                                 dead = true;
@@ -239,10 +252,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int L = p.seq_lens[s];
                 const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
                 const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-                const int j0 = slice_begin(split, n_sel);
-                const int j1 = slice_begin(split + 1, n_sel);
                 const int off = has_draft ? 1 : 0;
-                const int n_total = (j1 - j0) * upb + off;
+                const int n_total = slice_units(split, n_sel) + off;
                 bool dead = !mbar_wait_bounded(bar(kStaged), 0);
                 if (warp == 9) {
                     constexpr uint32_t idesc_s = umma_idesc_bf16(128, kUnit, false);
@@ -457,10 +468,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int L = p.seq_lens[s];
     const int nb = min(p.B == 128 ? (L + 127) >> 7 : (L + 63) >> 6, p.NBmax);
     const int n_sel = p.sel_idx ? max(0, min(p.sel_cnt[(size_t)s * p.Hkv + h], p.max_sel)) : nb;
-    const int j0 = slice_begin(split, n_sel);
-    const int j1 = slice_begin(split + 1, n_sel);
     const int off = has_draft ? 1 : 0;
-    const int n_total = (j1 - j0) * upb + off;
+    const int n_total = slice_units(split, n_sel) + off;
 
     // per slot (row): reference maximum of the exponentials (log2 units) and partial row sum
     float m[NH], l[NH];
@@ -785,13 +794,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 }  // namespace
 
-template <int NH, bool kWide, bool kPair>
+template <int NH, bool kWide, bool kPair, bool kUnitSlices = false>
 static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, dim3 grid,
                              cudaStream_t stream)
 {
     static svh::OncePerDevice once;   // function attributes belong to a device
     const cudaError_t ce = once.run([] {
-        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        return cudaFuncSetAttribute(verify_attn_tc_kernel<NH, kWide, kPair, kUnitSlices>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     kSmemBytes);
     });
     if (ce != cudaSuccess) return ce;
@@ -804,7 +813,7 @@ static cudaError_t launch_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, c
     svh::pdl_attribute(attr);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide, kPair>, tm_k, tm_v, p);
+    return cudaLaunchKernelEx(&cfg, verify_attn_tc_kernel<NH, kWide, kPair, kUnitSlices>, tm_k, tm_v, p);
 }
 
 // grid.x = splits x groups, where a group is a row tile or (p.pair) a pair of row tiles
@@ -812,15 +821,21 @@ cudaError_t launch_attn_tc(const CUtensorMap &tm_k, const CUtensorMap &tm_v, con
                            cudaStream_t stream)
 {
     const int rows = p.G * p.Tt;   // rows of a full row tile
-    if (p.pair) return launch_tc<4, true, true>(tm_k, tm_v, p, grid, stream);   // (a full tile has more than 64 rows)
+    const bool units = p.B == 128;   // 128-row tiles over blocks of 128 tokens: slices cut at 64-key units
+    if (p.pair) {   // (a full tile has more than 64 rows)
+        return units ? launch_tc<4, true, true, true>(tm_k, tm_v, p, grid, stream)
+                     : launch_tc<4, true, true>(tm_k, tm_v, p, grid, stream);
+    }
     if (p.tiles > 1 || p.T > 32) {
         if (rows <= 32) return launch_tc<1, true, false>(tm_k, tm_v, p, grid, stream);
         if (rows <= 64) return launch_tc<2, true, false>(tm_k, tm_v, p, grid, stream);
-        return launch_tc<4, true, false>(tm_k, tm_v, p, grid, stream);
+        return units ? launch_tc<4, true, false, true>(tm_k, tm_v, p, grid, stream)
+                     : launch_tc<4, true, false>(tm_k, tm_v, p, grid, stream);
     }
     if (rows <= 32) return launch_tc<1, false, false>(tm_k, tm_v, p, grid, stream);
     if (rows <= 64) return launch_tc<2, false, false>(tm_k, tm_v, p, grid, stream);
-    return launch_tc<4, false, false>(tm_k, tm_v, p, grid, stream);
+    return units ? launch_tc<4, false, false, true>(tm_k, tm_v, p, grid, stream)
+                 : launch_tc<4, false, false>(tm_k, tm_v, p, grid, stream);
 }
 
 }  // namespace svk
