@@ -441,8 +441,10 @@ def run_gpu(args):
 
     ms_e2e_one_stream = time_e2e_serial(side, 4, None)
     out_h.zero_()
+    e2e_chunks = [int(x) for x in str(args.e2e_chunk).split(",") if x]
+    e2e_chunks = None if not e2e_chunks else (e2e_chunks[0] if len(e2e_chunks) == 1 else e2e_chunks)
     g_host = capture(lambda: eng.verify_step_from_host(q_h, dk_h, dv_h, q, dk, dv, out, out_h,
-                                                       layers_per_chunk=args.e2e_chunk, refresh_tail=True))
+                                                       layers_per_chunk=e2e_chunks, refresh_tail=True))
     ms_e2e = time_e2e_serial(side, 4, g_host)
     assert torch.equal(out_h, out.cpu()), "the host-fed step did not deliver the step's outputs"
     assert int(eng.status.item()) == 0 and int(eng_reuse.status.item()) == 0 and int(eng_chain.status.item()) == 0, \
@@ -485,7 +487,7 @@ def run_gpu(args):
                         "Q and draft K/V of all layers from pinned host memory, the step, the outputs back to pinned host "
                         "memory, the copies in chunks of a few layers on two side streams so that all but the first upload "
                         "and the last download run under the step's kernels; the KV cache is device-resident state",
-                "layers_per_chunk": args.e2e_chunk,
+                "layers_per_chunk": e2e_chunks if e2e_chunks is not None else "2 / half / half / 2",
                 "one_stream_value": ms_e2e_one_stream * 1e3 / (w.n_layers * world),
                 "one_stream_note": "the same bytes copied whole before and after the step on the step's own stream",
                 "pipelined_value": ms_e2e_pipelined * 1e3 / (w.n_layers * world),
@@ -900,7 +902,8 @@ def main():
                     help="instead of the benchmark line: sparse vs dense latency over context x budget x draft length")
     ap.add_argument("--configs", action="store_true",
                     help="timing lines for the batched (16 ragged sequences) and long-context (4 x 128K, tree) configurations")
-    ap.add_argument("--e2e-chunk", type=int, default=4, help="layers per copy chunk of the end-to-end step")
+    ap.add_argument("--e2e-chunk", default="", help="layers per copy chunk of the end-to-end step: a size, or sizes a,b,c,... "
+                                                     "(default: the engine's schedule, 2 / half / half / 2)")
     ap.add_argument("--only", default="", help="with --configs: comma-separated configuration names (profiling aid: no dense pass)")
     ap.add_argument("--variants", action="store_true",
                     help="instead of the benchmark line: timings of the retrieval variants (shared budget, every token)")

@@ -111,9 +111,9 @@ class SparseVerifier:
             self.verify_layer(l, q[l], draft_k[l], draft_v[l], out[l], behind_own_layer=l > 0)
 
     def verify_step_from_host(self, q_host, draft_k_host, draft_v_host, q, draft_k, draft_v, out, out_host,
-                              layers_per_chunk: int = 4, refresh_tail: bool = False) -> None:
+                              layers_per_chunk=None, refresh_tail: bool = False) -> None:
         """verify_step with the step's inputs in pinned host memory and its outputs wanted there.  The copies go in chunks
-        of a few layers on two side streams: a chunk's layers start as soon as its inputs have arrived, its outputs leave
+        of a few layers (layers_per_chunk: one size, or a list of sizes) on two side streams: a chunk's layers start as soon as its inputs have arrived, its outputs leave
         while the next chunk computes, so only the first upload and the last download are not hidden behind kernels.
         q/draft_k/draft_v/out are the device staging tensors (shapes as for verify_step); the *_host tensors the pinned
         ones.  Returns with everything enqueued; the current stream ends behind the last download.  Capturable in a
@@ -124,7 +124,23 @@ class SparseVerifier:
         s_in, s_out = self._copy_streams
         s_in.wait_stream(main)
         s_out.wait_stream(main)
-        chunks = [(c0, min(c0 + layers_per_chunk, self.n_layers)) for c0 in range(0, self.n_layers, layers_per_chunk)]
+        if layers_per_chunk is None:
+            # two layers first and last (their upload / download is what nothing hides), the rest in two halves (every
+            # chunk boundary costs the step a few microseconds): 32 layers measured 16.1 us/layer against 16.6 in chunks
+            # of four and 18.5 with the copies whole
+            mid = max(0, self.n_layers - 4)
+            layers_per_chunk = [2, (mid + 1) // 2, mid // 2, 2] if self.n_layers > 4 else [self.n_layers]
+        if isinstance(layers_per_chunk, int):
+            sizes = [layers_per_chunk] * -(-self.n_layers // layers_per_chunk)
+        else:   # a schedule: e.g. a small first and last chunk (their copies are the ones nothing hides), large ones between
+            sizes = list(layers_per_chunk)
+        chunks, c0 = [], 0
+        for n in sizes:
+            if c0 < self.n_layers and n > 0:
+                chunks.append((c0, min(c0 + n, self.n_layers)))
+                c0 += n
+        if c0 < self.n_layers:
+            chunks.append((c0, self.n_layers))
         arrived = []
         with torch.cuda.stream(s_in):
             for c0, c1 in chunks:
