@@ -52,8 +52,10 @@ class SparseVerifier:
         for l in range(n_layers):
             self.set_layer_kv(l, k_all[l], v_all[l])
         g = self.geom
-        offs = (torch.arange(n_layers, device=k_all.device, dtype=torch.int32) * n_pages).view(n_layers, 1, 1)
-        self._stack_table = (self.block_table.unsqueeze(0) + offs).reshape(n_layers * g.n_seq, g.max_blocks).contiguous()
+        self._stack_offs = (torch.arange(n_layers, device=k_all.device, dtype=torch.int32) * n_pages).view(n_layers, 1, 1)
+        self._stack_table = torch.empty((n_layers * g.n_seq, g.max_blocks), dtype=torch.int32, device=k_all.device)
+        self._stack_pages = n_pages
+        self.sync_block_table()
         self._stack_lens = self.seq_lens.repeat(n_layers).contiguous()
         self._stack_geom = sv.make_geom(g.n_seq * n_layers, g.n_q_heads, g.n_kv_heads, g.head_dim, g.block_size,
                                         g.max_blocks, g.n_draft)
@@ -61,6 +63,13 @@ class SparseVerifier:
         self._stack_kv = sv.make_kv(k_all.view(n_layers * n_pages, *k_all.shape[2:]),
                                     v_all.view(n_layers * n_pages, *v_all.shape[2:]), self._stack_table,
                                     self._stack_lens)
+
+    def sync_block_table(self) -> None:
+        """Rebuild the stacked page table from block_table (call after assigning pages to a sequence; commit does it
+        itself).  Entries that are not pages of a layer's pool stay invalid in every layer."""
+        bt = self.block_table.unsqueeze(0)
+        ok = (bt >= 0) & (bt < self._stack_pages)
+        self._stack_table.copy_(torch.where(ok, bt + self._stack_offs, -1).reshape(self._stack_table.shape))
 
     def refresh_tail_all(self) -> None:
         """Recompute the representative of every sequence's last block in all layers (one launch)."""
@@ -182,17 +191,28 @@ class SparseVerifier:
         return path, n_path, next_token
 
     def commit(self, draft_k, draft_v, path, n_path) -> None:
-        """Append the kept rows' K/V of every layer to the paged cache (one sv_kv_append per layer, which also
-        refreshes the representatives of the blocks that grew) and advance the sequence lengths.  The block table
+        """Append the kept rows' K/V of every layer to the paged cache (sv_kv_append, which also refreshes the
+        representatives of the blocks that grew: one launch for all layers when the pools were given with
+        set_kv_stack, else one per layer) and advance the sequence lengths.  The block table
         must already hold pages for the blocks the sequences grow into.  draft_k/v: [layers][S][T][Hkv][D]."""
+        if self._stack_kv is not None:   # one launch for all layers: (layer, sequence) is the batch dimension
+            self.sync_block_table()
+            L, g = self.n_layers, self.geom
+            k_all, v_all = self._stack_pools
+            new_len = torch.empty_like(self._stack_lens)
+            sv.sv_kv_append(self._stack_geom, k_all.view(-1, *k_all.shape[2:]), v_all.view(-1, *v_all.shape[2:]),
+                            self._stack_table, self._stack_lens, draft_k.reshape(L * g.n_seq, *draft_k.shape[2:]),
+                            draft_v.reshape(L * g.n_seq, *draft_v.shape[2:]), path.repeat(L, 1), n_path.repeat(L), new_len,
+                            self.reps.view(-1, *self.reps.shape[2:]))
+            self._stack_lens.copy_(new_len)
+            self.seq_lens.copy_(new_len[:g.n_seq])
+            return
         new_len = torch.empty_like(self.seq_lens)
         for l in range(self.n_layers):
             k_pool, v_pool = self._pools[l]
             sv.sv_kv_append(self.geom, k_pool, v_pool, self.block_table, self.seq_lens, draft_k[l], draft_v[l], path,
                             n_path, new_len, self.reps[l])
         self.seq_lens.copy_(new_len)          # every layer has read the old lengths by now (same stream)
-        if self._stack_kv is not None:
-            self._stack_lens.copy_(self.seq_lens.repeat(self.n_layers))
 
     def check_status(self) -> None:
         """Read the device status word back (this synchronises with the stream) and raise if a kernel gave up
