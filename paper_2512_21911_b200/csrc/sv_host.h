@@ -113,17 +113,17 @@ inline int sm_count()
 // from one gather, each softmax warpgroup taking every unit for its own tile).  One per tile is the default: the CTAs
 // that share a slice of the blocks sit next to each other in the grid, request the same K/V tiles at about the same
 // time, and all but the first find them in L2 (240 rows, one sequence: 29.6 MB from DRAM for 29.8 MB algorithmic), and
-// the finer CTAs fill the SMs better (20.0 against 22.9 us there).  A paired CTA takes 16/9 as long as a single-tile
-// one (batches of 240-row trees: 100 against 56 us per wave of CTAs), so pairs are used where they save enough waves
-// to pay for that -- in practice when the row-tile CTAs just miss fitting the SMs once (10 to 16 such sequences of 8
-// KV heads: 100 against 112 us).
+// the finer CTAs fill the SMs better.  A paired CTA takes 1.93 times as long as a single-tile one (batches of 240-row
+// trees: 99.5 against 51.6 us per wave of CTAs), so pairs are used where they save enough waves to pay for that -- in
+// practice when the row-tile CTAs just miss fitting the SMs once or twice (10 to 16 such sequences of 8 KV heads:
+// 99 against 103 us).
 inline bool pair_row_tiles(const sv_geom *g)
 {
     const int t = row_tiles(g);
     if (t < 2) return false;
     const long long pairs = (long long)g->n_seq * g->n_kv_heads, sms = sm_count();
     const long long waves_tile = (pairs * t + sms - 1) / sms, waves_pair = (pairs * ((t + 1) / 2) + sms - 1) / sms;
-    return 16 * waves_pair < 9 * waves_tile;
+    return 29 * waves_pair < 15 * waves_tile;
 }
 inline int row_groups(const sv_geom *g)
 {

@@ -38,7 +38,9 @@ constexpr int kThreads = 384;
 constexpr int kUnit = 64;                        // keys per unit
 constexpr int kTile = kUnit * 128;               // bytes of one [64 rows][64 bf16] half tile (8 KB)
 constexpr int kStageBytes = 4 * kTile;           // K lo/hi + V lo/hi
-constexpr int kStages = 5;                       // ring stages; a CTA that serves two row tiles has two Q tiles and four stages
+constexpr int kStages = 5;                       // ring stages; a CTA that serves two row tiles has two Q tiles and four stages;
+                                                 // 128-row tiles keep P in tensor memory and use its 32 KB as one more stage
+constexpr int kMaxStages = kStages + 1;
 constexpr int kQBytes = 2 * 128 * 128;           // Q of one row tile: two halves [128 rows][64 bf16]
 constexpr int kPBytes = 128 * 128;               // P: [128 rows][64 bf16]
 constexpr int kOffP = kStages * kStageBytes + kQBytes;   // (= 4 stages + 2 Q tiles)
@@ -46,15 +48,18 @@ constexpr int kOffDraft = 0;                     // the draft unit is the first 
 constexpr int kOffMisc = kOffP + 2 * kPBytes;
 constexpr int kSmemBytes = 1024 + kOffMisc + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
-static_assert(2 * kStages + 10 <= 32, "one lane of the producer warp per barrier");
+static_assert(2 * kMaxStages + 10 <= 32, "one lane of the producer warp per barrier");
 static_assert((kStages - 1) * kStageBytes + 2 * kQBytes == kOffP, "both layouts put P at the same offset");
-constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns
+constexpr int kTmemCols = 512;                   // S: 2 x 64 columns, O: 2 x 128 columns; 128-row tiles also P: 2 x 32 and
+                                                 // Q: 64, or (two row tiles per CTA) Q: 2 x 64
+constexpr int kTmemP = 384;                      // first column of P: [warpgroup][32 packed columns]
+constexpr int kTmemQ = 448;                      // Q of a single row tile: 128 dims = 64 packed columns (two row tiles: 384, 448)
 
 // barrier slots (8 bytes each) inside the misc area
 enum Bar {
-    kFull = 0,                  // [kStages] TMA landed
-    kEmpty = kFull + kStages,   // [kStages] PV of the unit finished reading the stage
-    kSReady = kEmpty + kStages, // [2] S of the warpgroup's unit is in TMEM
+    kFull = 0,                  // [kMaxStages] TMA landed
+    kEmpty = kFull + kMaxStages,   // [kStages] PV of the unit finished reading the stage
+    kSReady = kEmpty + kMaxStages, // [2] S of the warpgroup's unit is in TMEM
     kSFree = kSReady + 2,       // [2] the warpgroup has read S
     kPReady = kSFree + 2,       // [2] P is in shared memory
     kOReady = kPReady + 2,      // [2] the warpgroup's latest PV has been added to O in TMEM
@@ -88,7 +93,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
     static_assert(!kPair || (kWide && NH == 4), "row-tile pairs exist only where one tile is full (more than 64 rows)");
-    constexpr int NS = kPair ? kStages - 1 : kStages;        // ring stages
+    // 128-row tiles are bound by the tensor pipe when every MMA fetches both operands from shared memory (S = Q K^T: eight
+    // 128 x 64 x 16 MMAs, each re-reading 4 KB of Q), so their Q lives in tensor memory (A operand from TMEM), and with a
+    // single row tile P does too (one tile per warpgroup), which frees 32 KB for a sixth ring stage.
+    constexpr bool kQTmem = NH == 4;
+    constexpr bool kPTmem = NH == 4 && !kPair;
+    constexpr int NS = kPair ? kStages - 1 : kPTmem ? kStages + 1 : kStages;   // ring stages
     constexpr int OFFQ = NS * kStageBytes;                   // the Q tile (kPair: of warpgroup 0; warpgroup 1's follows)
     // blockIdx.x = split * groups + group: the CTAs that gather the same slice of the blocks are neighbours in the grid
     // (they share those K/V tiles through L2; 1-2 % faster than group-major order).  A group is a row tile (kWide), or
@@ -281,7 +291,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                         for (int ks = 0; ks < 8; ++ks) {
                             const uint32_t qo = (uint32_t)(((kPair ? g * kQBytes : 0) + (ks >> 2) * (kQBytes / 2) + (ks & 3) * 32) >> 4);
                             const uint32_t ko = (uint32_t)(((ks >> 2) * kTile + (ks & 3) * 32) >> 4);
-                            tc_mma_bf16(d, d_hi | (dq_lo + qo), d_hi | (k_lo + ko), idesc_s, ks > 0);
+                            if constexpr (kQTmem)   // 16 dims = 8 packed columns of Q per instruction
+                                tc_mma_bf16_ta(d, tmem_base + (kPair ? kTmemP + g * 64 : kTmemQ) + ks * 8, d_hi | (k_lo + ko), idesc_s, ks > 0);
+                            else
+                                tc_mma_bf16(d, d_hi | (dq_lo + qo), d_hi | (k_lo + ko), idesc_s, ks > 0);
                         }
                         tc_commit(bar(kSReady + g));
                     }
@@ -309,9 +322,14 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const uint32_t p_lo = dp_lo + (uint32_t)((g * kPBytes) >> 4);
                         const uint32_t d = tmem_base + 128 + g * 128;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            tc_mma_bf16(d, dp_hi | (p_lo + (uint32_t)((kk * 32) >> 4)), dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)),
-                                        idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);   // the warpgroup's first unit starts O
+                        for (int kk = 0; kk < 4; ++kk) {   // (the warpgroup's first unit starts O)
+                            if constexpr (kPTmem)   // A = P from tensor memory: 16 keys = 8 packed columns per instruction
+                                tc_mma_bf16_ta(d, tmem_base + kTmemP + g * 32 + kk * 8,
+                                               dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)), idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);
+                            else
+                                tc_mma_bf16(d, dp_hi | (p_lo + (uint32_t)((kk * 32) >> 4)), dv_hi | (v_lo + (uint32_t)((kk * 2048) >> 4)),
+                                            idesc_pv, (k > 0 || kk > 0) ? 1u : 0u);
+                        }
                         tc_commit(bar(kOReady + g));
                         if (!kPair || g == n_wg - 1) tc_commit(bar(kEmpty + stage));   // the last reader of the stage
                     }
@@ -430,6 +448,26 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     fence_proxy_async();   // the tensor cores read these tiles through the async proxy
     named_bar_sync(2, 256);
+    if constexpr (kQTmem) {
+        // Q goes on to tensor memory (thread = tile row = TMEM lane; the 64 32-bit words of the row are the 64 packed
+        // columns): every S = Q K^T then reads only the K tile from shared memory, which is what bounds a
+        // 128 x 64 x 16 MMA whose two operands both come from there.
+        if (kPair || warp < 4) {   // (two row tiles: either warpgroup copies its own)
+            const int tr = (warp & 3) * 32 + lane;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t w[32];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(q_tile + half * (kQBytes / 2) + swz128(tr, c));
+                    w[4 * c] = v.x, w[4 * c + 1] = v.y, w[4 * c + 2] = v.z, w[4 * c + 3] = v.w;
+                }
+                tmem_st_x32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (kPair ? kTmemP + (warp >> 2) * 64 : kTmemQ) + half * 32, w);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+        }
+    }
     if (lane == 0) mbar_arrive(bar(kStaged));
     if (has_draft && tid == 0) mbar_arrive(bar(kFull + 0));   // the draft unit fills stage 0 in place of a TMA load
 
@@ -567,19 +605,34 @@ __global__ void __launch_bounds__(kThreads, 1)
             const float m_use = (m[0] == -INFINITY) ? 0.f : m[0];
             const unsigned long long scale2 = f2_pack(p.scale_log2, p.scale_log2), neg_m2 = f2_pack(-m_use, -m_use);
             unsigned long long lsum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
-            const uint32_t row = (uint32_t)(quad * 32 + lane);
+            if constexpr (kPTmem) {
+                uint32_t pk[32];   // this row of P: keys 2c, 2c + 1 are packed column c
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
+                for (int c = 0; c < 32; ++c) {
                     float x0, x1;
-                    f2_unpack(f2_fma(f2_pack(sc[8 * j + 2 * e], sc[8 * j + 2 * e + 1]), scale2, neg_m2), x0, x1);
+                    f2_unpack(f2_fma(f2_pack(sc[2 * c], sc[2 * c + 1]), scale2, neg_m2), x0, x1);
                     const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                    lsum2[e & 1] = f2_add(lsum2[e & 1], f2_pack(p0, p1));
-                    pk[e] = pack_bf16(p0, p1);
+                    lsum2[c & 1] = f2_add(lsum2[c & 1], f2_pack(p0, p1));
+                    pk[c] = pack_bf16(p0, p1);
                 }
-                *reinterpret_cast<uint4 *>(pbuf + swz128(row, j)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                tmem_st_x32(tmem_base + t_lane + kTmemP + wg * 32, pk);
+                tmem_st_wait();   // P is in tensor memory
+                tc_fence_before_sync();
+            } else {
+                const uint32_t row = (uint32_t)(quad * 32 + lane);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float x0, x1;
+                        f2_unpack(f2_fma(f2_pack(sc[8 * j + 2 * e], sc[8 * j + 2 * e + 1]), scale2, neg_m2), x0, x1);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        lsum2[e & 1] = f2_add(lsum2[e & 1], f2_pack(p0, p1));
+                        pk[e] = pack_bf16(p0, p1);
+                    }
+                    *reinterpret_cast<uint4 *>(pbuf + swz128(row, j)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
             }
             float ls0, ls1;
             f2_unpack(f2_add(lsum2[0], lsum2[1]), ls0, ls1);
@@ -718,7 +771,21 @@ __global__ void __launch_bounds__(kThreads, 1)
     // they spread over the SMs that the attention CTAs are about to vacate.
     grid_launch_dependents();
     if (k > 0) wait_pv(k - 1);   // this warpgroup's accumulator is complete
-    if constexpr (!kPair) {
+    uint32_t ml_theirs[8] = {};   // (kPTmem) the other warpgroup's m, l of this thread's slots
+    if constexpr (!kPair && kPTmem) {
+        // no P tiles in shared memory: the exchange goes through the warpgroup's own (now idle) S columns, thread for
+        // thread (this thread's slots live on TMEM lane quad * 32 + lane in either warpgroup)
+        uint32_t ml_ours[8];
+#pragma unroll
+        for (int i = 0; i < NH; ++i) ml_ours[2 * i] = __float_as_uint(m[i]), ml_ours[2 * i + 1] = __float_as_uint(l[i]);
+        tmem_st_x8(tmem_base + t_lane + wg * kUnit, ml_ours);
+        tmem_st_wait();
+        tc_fence_before_sync();
+        named_bar_sync(1, n_sm);
+        tc_fence_after_sync();
+        tmem_ld_x8(tmem_base + t_lane + (wg ^ 1) * kUnit, ml_theirs);
+        tmem_ld_wait();
+    } else if constexpr (!kPair) {
 #pragma unroll
         for (int i = 0; i < NH; ++i) {
             ml_mine[(2 * i) * 128 + t] = m[i];
@@ -742,8 +809,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
             for (int hh = 0; hh < (NH == 1 ? 1 : 2); ++hh) {
                 const int i = lo * 2 + hh;
-                const float m1 = kPair ? -INFINITY : ml_other[(2 * i) * 128 + t];
-                const float l1 = kPair ? 0.f : ml_other[(2 * i + 1) * 128 + t];
+                const float m1 = kPair ? -INFINITY : kPTmem ? __uint_as_float(ml_theirs[2 * i]) : ml_other[(2 * i) * 128 + t];
+                const float l1 = kPair ? 0.f : kPTmem ? __uint_as_float(ml_theirs[2 * i + 1]) : ml_other[(2 * i + 1) * 128 + t];
                 const float M = fmaxf(m[i], m1);
                 const float M_use = (M == -INFINITY) ? 0.f : M;
                 const float w0 = fast_exp2(m[i] - M_use), w1 = fast_exp2(m1 - M_use);
