@@ -97,6 +97,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     // 128 x 64 x 16 MMAs, each re-reading 4 KB of Q), so their Q lives in tensor memory (A operand from TMEM), and with a
     // single row tile P does too (one tile per warpgroup), which frees 32 KB for a sixth ring stage.
     constexpr bool kQTmem = NH == 4;
+    // Up to 64 query rows run as M = 64 MMAs (half the tensor time of the zero-padded M = 128 tile): matrix row m is
+    // TMEM lane (m / 16) * 32 + m % 16, the 16 lanes per quadrant that the NH <= 2 softmax layout uses anyway.
+    constexpr int MT = NH == 4 ? 128 : 64;                   // rows of the Q and P tiles and of the MMAs
+    constexpr int QR = NH == 4 ? 32 : 16;                    // tile rows per TMEM lane quadrant
     constexpr bool kPTmem = NH == 4 && !kPair;
     constexpr int NS = kPair ? kStages - 1 : kPTmem ? kStages + 1 : kStages;   // ring stages
     constexpr int OFFQ = NS * kStageBytes;                   // the Q tile (kPair: of warpgroup 0; warpgroup 1's follows)
@@ -266,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int n_total = slice_units(split, n_sel) + off;
                 bool dead = !mbar_wait_bounded(bar(kStaged), 0);
                 if (warp == 9) {
-                    constexpr uint32_t idesc_s = umma_idesc_bf16(128, kUnit, false);
+                    constexpr uint32_t idesc_s = umma_idesc_bf16(MT, kUnit, false);
                     const uint64_t dq = umma_desc_sw128(smem0 + OFFQ, 16, 1024);
                     const uint64_t dk = umma_desc_sw128(smem0, 16, 1024);
                     const uint32_t dq_lo = (uint32_t)dq, dk_lo = (uint32_t)dk;
@@ -301,7 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     // free TMEM only after every softmax warp has finished reading it
                     if (!mbar_wait_bounded(bar(kTmemDone), 0) && p.status) atomicOr(p.status, 16);
                 } else {
-                    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, true);
+                    constexpr uint32_t idesc_pv = umma_idesc_bf16(MT, 128, true);
                     const uint64_t dp = umma_desc_sw128(smem0 + kOffP, 16, 1024);
                     const uint64_t dv = umma_desc_sw128(smem0 + 2 * kTile, kTile, 1024);
                     const uint32_t dp_lo = (uint32_t)dp, dv_lo = (uint32_t)dv;
@@ -355,10 +359,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     constexpr int kQThreads = kPair ? 128 : 256;
     const int qtid = kPair ? (tid & 127) : tid;
     uint8_t *q_tile = smem + OFFQ + (kPair ? ((warp >> 2) & 1) * kQBytes : 0);
-    for (int idx = qtid; idx < 128 * 16; idx += kQThreads) {
+    for (int idx = qtid; idx < MT * 16; idx += kQThreads) {
         const int tr = idx >> 4, c = idx & 15;
-        const int r = (tr >> 5) * RPQ + (tr & 31);
-        if (!((tr & 31) < RPQ && r < rows))
+        const int r = (tr / QR) * RPQ + (tr % QR);
+        if (!((tr % QR) < RPQ && r < rows))
             *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = make_uint4(0u, 0u, 0u, 0u);
     }
     if (has_draft) {
@@ -433,7 +437,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int idx = qtid + x * kQThreads;
             if (idx < n_q) {
                 const int r = idx >> 4, c = idx & 15;
-                const int tr = (r / RPQ) * 32 + (r % RPQ);
+                const int tr = (r / RPQ) * QR + (r % RPQ);
                 *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * (kQBytes / 2) + swz128(tr, c & 7)) = v[x];
             }
         }
@@ -489,7 +493,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
     for (int i = 0; i < NH; ++i) {
         lrow[i] = quad * RPQ + 8 * i + lr;
-        trow[i] = quad * 32 + 8 * i + lr;
+        trow[i] = quad * QR + 8 * i + lr;
         if constexpr (kWide) {
             const unsigned long long all_t = (p.T == 64) ? ~0ull : ((1ull << p.T) - 1ull);
             const unsigned long long row_vis = (has_draft && lrow[i] < rows) ? anc[i0 + div_g(lrow[i])] : all_t;
