@@ -2,14 +2,17 @@
 //
 // Grid (split [x row tile], KV head, sequence); a CTA owns
 // a contiguous slice of the ascending block list of its (sequence, KV head) and all G*T query rows of
-// that KV head, padded to one M = 128 tile.  Per 64-key unit (32 KB of K and V gathered by TMA):
+// that KV head, padded to one M = 64 (up to 64 rows) or M = 128 tile.  Per 64-key unit (32 KB of K and V gathered
+// by TMA), with M = 128:
 //
-//   S[128 x 64]  = Q[128 x 128] . K^T     8 x tcgen05.mma (M128 N64 K16), operands in shared memory
-//                                         (Q, K: K-major, 128-byte swizzle), accumulator in TMEM
+//   S[128 x 64]  = Q[128 x 128] . K^T     8 x tcgen05.mma (M128 N64 K16), K from shared memory (K-major, 128-byte
+//                                         swizzle), Q from shared memory (same layout) or, for 128-row tiles,
+//                                         from tensor memory; accumulator in TMEM
 //   softmax      up to 64 query rows: four threads per row (tcgen05.ld 16x256b, the mma.sync accumulator
 //                fragment layout, rows spread over all four lane quadrants): mask, running max / sum in
-//                fp32 with quad shuffles; 65-128 rows: one thread per row (tcgen05.ld 32x32b), no shuffles,
-//                16-byte P stores.  P rounded to bf16 into shared memory (K-major, 128-byte swizzle)
+//                fp32 with quad shuffles; 65-128 rows: one thread per row (tcgen05.ld 32x32b), no shuffles.
+//                P rounded to bf16 into shared memory (K-major, 128-byte swizzle) or, for a single 128-row
+//                tile, into tensor memory (two keys per 32-bit column)
 //   O[128x128]  += P[128 x 64] . V        4 x tcgen05.mma (M128 N128 K16), V read MN-major from the
 //                                         tile exactly as TMA stored it; O stays in TMEM for the whole
 //                                         kernel.  The exponentials use a reference maximum that is only
