@@ -131,6 +131,19 @@ def test_workspace_size_formula(svb):
     assert svb.sv_workspace_bytes(svb.make_geom(1, 8, 3, 128, 64, 64, 4), 16) == 0
 
 
+def test_split_rule_on_a_148_sm_device(svb):
+    """The split counts of the shapes the profiles quote (the library assumes 148 SMs when it has no device to ask, and a
+    B200 has 148): few units unsplit; the benchmark layer 16 splits; 240-row trees one CTA per row tile while those fit
+    the SMs (1 / 2 / 4 / 8 sequences: 9 / 4 / 2 / 1 splits -- with a pair of row tiles per CTA it would be 18 / 9 / 4 / 2),
+    and no split once there are more row-tile CTAs than SMs; the workspace follows the split count."""
+    assert svb.sv_verify_attn_splits(svb.make_geom(1, 32, 8, 128, 64, 128, 8), 4) == 1
+    assert svb.sv_verify_attn_splits(svb.make_geom(1, 32, 8, 128, 64, 512, 8), 64) == 16
+    for n_seq, want in ((1, 9), (2, 4), (4, 2), (8, 1), (12, 1), (24, 1)):
+        g = svb.make_geom(n_seq, 32, 8, 128, 64, 512, 60)
+        assert svb.sv_verify_attn_splits(g, 70) == want, n_seq
+        assert svb.sv_workspace_bytes(g, 70) == (0 if want == 1 else n_seq * 8 * want * 240 * 130 * 4 + 256)
+
+
 def test_pick_anchors_matches_oracle_on_host(svb):
     import numpy as np
     g = np.random.default_rng(2)
