@@ -672,7 +672,8 @@ def run_configs(args):
     """--configs: timing lines for the other full-size configurations (their parity is covered by the tests):
     the 16-sequence batch with ragged prefixes (block 64, 2048-token budget, 5 draft tokens as a chain), the
     4 x 131072-token long-context case (GQA 8, block 128, 4096-token budget, 16-node draft tree), and 60-token
-    draft trees on Llama-3.1-8B geometry (240 query rows per KV head), one sequence and a batch of 12.  K/V are seeded
+    draft trees on Llama-3.1-8B geometry (240 query rows per KV head), one sequence and a batch of 12, and a batch of
+    128 ragged sequences (several waves of CTAs).  K/V are seeded
     device-side N(0, 1/128) tensors, lengths / page tables / the tree come from seeded host generators, the block
     lists from sv_select_blocks.  Each configuration rotates over independent KV replicas so that at least 256 MiB
     is gathered between two uses of a replica (HBM, not L2).  One JSON line per configuration."""
@@ -691,7 +692,9 @@ def run_configs(args):
              ("tree60", dict(S=1, Hq=32, Hkv=8, B=64, lens=(32768, 32768), budget_tokens=None, T=60, tree=True, seed=1060)),
              # a batch of such trees on ragged prefixes: 12 x 8 x 2 row tiles just miss fitting the SMs once, the case
              # in which one CTA serves a pair of row tiles
-             ("tree60_batch", dict(S=12, Hq=32, Hkv=8, B=64, lens=(6000, 10000), budget_tokens=None, T=60, tree=True, seed=1061))]
+             ("tree60_batch", dict(S=12, Hq=32, Hkv=8, B=64, lens=(6000, 10000), budget_tokens=None, T=60, tree=True, seed=1061)),
+             # the 16-sequence batch eight times over: seven waves of CTAs, one per (sequence, KV head)
+             ("batch128", dict(S=128, Hq=32, Hkv=8, B=64, lens=(4096, 16384), budget_tokens=2048, T=5, tree=False, seed=1005))]
     if args.only:
         cases = [c for c in cases if c[0] in args.only.split(",")]
     for name, c in cases:
