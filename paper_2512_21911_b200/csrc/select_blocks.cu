@@ -26,7 +26,8 @@ namespace {
 
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
-constexpr int kRowsPerIter = 4;   // independent representative rows a warp has in flight
+constexpr int kRowsPerIter = 4;   // consecutive representative rows a warp scores per pass (one 16-byte store of keys)
+constexpr int kStride = kWarps * kRowsPerIter;   // blocks the CTA covers per pass
 
 using svsel::kForcedKey;
 using svsel::order_key;
@@ -47,8 +48,10 @@ struct SelectParams {
 // on an mbarrier there, and exits; CTA 0 waits for the expected number of bytes and selects.  The only cluster-wide barrier is split (arrive early, wait late) so that
 // its latency hides behind the loads.
 // kBf16: the representatives are stored in bfloat16 (storage variant); scores are fp32 either way.
-template <bool kBf16>
-__global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
+// kDepth: passes whose rows a warp loads together (1, or 2 for slices of more than 64 blocks: eight rows in flight per
+// warp, half as many trips to DRAM; more would cost the second CTA per SM its registers).
+template <bool kBf16, int kDepth>
+__global__ void __launch_bounds__(kThreads, 2) select_kernel(const SelectParams p)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
@@ -86,8 +89,10 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     };
     int b = b0 + warp * kRowsPerIter;
 #pragma unroll
-    for (int i = 0; i < kRowsPerIter; ++i)
-        if (b + i < min(b0 + p.chunk, p.NBmax)) svk::prefetch_l2(row_ptr(b + i));
+    for (int d = 0; d < kDepth; ++d)
+#pragma unroll
+        for (int i = 0; i < kRowsPerIter; ++i)
+            if (b + d * kStride + i < min(b0 + p.chunk, p.NBmax)) svk::prefetch_l2(row_ptr(b + d * kStride + i));
     const int G = p.Hq / p.Hkv;
     const __nv_bfloat16 *q0 = p.q + ((size_t)s * p.T * p.Hq + (size_t)h * G) * 128;
     if (tid < G * 2) svk::prefetch_l2(q0 + tid * 64);
@@ -97,11 +102,13 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     // every load below is issued before the first use
     const int L = p.seq_lens[s];
     const int budget = p.budget[s];
-    float4 r[kRowsPerIter];
+    float4 r[kDepth][kRowsPerIter];
     auto load_rows = [&](int bb, int hi) {
 #pragma unroll
-        for (int i = 0; i < kRowsPerIter; ++i)
-            r[i] = (bb + i < hi) ? load_row(bb + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int d = 0; d < kDepth; ++d)
+#pragma unroll
+            for (int i = 0; i < kRowsPerIter; ++i)
+                r[d][i] = (bb + d * kStride + i < hi) ? load_row(bb + d * kStride + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     };
     load_rows(b, min(b0 + p.chunk, p.NBmax));
     float qsum = 0.f;
@@ -133,21 +140,27 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
     }
     if (need_scores) {
         const float4 qv = reinterpret_cast<const float4 *>(qbar)[lane];
-        for (; b < b1; b += kWarps * kRowsPerIter) {
-            uint32_t kk[kRowsPerIter];
+        for (; b < b1; b += kDepth * kStride) {
 #pragma unroll
-            for (int i = 0; i < kRowsPerIter; ++i) {
-                float d = r[i].x * qv.x + r[i].y * qv.y + r[i].z * qv.z + r[i].w * qv.w;
+            for (int d = 0; d < kDepth; ++d) {
+                const int bd = b + d * kStride;
+                if (bd >= b1) break;   // (warp-uniform)
+                uint32_t kk[kRowsPerIter];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-                const int bb = b + i;
-                const bool is_forced = bb < p.n_sink || bb >= nb - p.n_local;
-                kk[i] = is_forced ? kForcedKey : order_key(d);
-                if (p.out_scores && lane == 0 && bb < b1) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = d;
+                for (int i = 0; i < kRowsPerIter; ++i) {
+                    float dot = r[d][i].x * qv.x + r[d][i].y * qv.y + r[d][i].z * qv.z + r[d][i].w * qv.w;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                    const int bb = bd + i;
+                    const bool is_forced = bb < p.n_sink || bb >= nb - p.n_local;
+                    kk[i] = is_forced ? kForcedKey : order_key(dot);
+                    if (p.out_scores && lane == 0 && bb < b1) p.out_scores[((size_t)s * p.Hkv + h) * p.NBmax + bb] = dot;
+                }
+                // rows bd .. bd+3 are 4 consecutive keys: one 16-byte store into CTA 0 (entries past nb are never read)
+                if (lane == 0 && !keep_all)
+                    svk::st_async_cluster_v4(keys0 + 4u * (uint32_t)bd, make_uint4(kk[0], kk[1], kk[2], kk[3]), ready0);
             }
-            // rows b .. b+3 are 4 consecutive keys: one 16-byte store into CTA 0 (entries past nb are never read)
-            if (lane == 0 && !keep_all) svk::st_async_cluster_v4(keys0 + 4u * (uint32_t)b, make_uint4(kk[0], kk[1], kk[2], kk[3]), ready0);
-            if (b + kWarps * kRowsPerIter < b1) load_rows(b + kWarps * kRowsPerIter, b1);
+            if (b + kDepth * kStride < b1) load_rows(b + kDepth * kStride, b1);
         }
     }
     if (rank != 0) return;
@@ -189,8 +202,8 @@ static bool clusters_of_16_fit(bool reps_bf16)
     if (dev < 0 || dev >= svh::kMaxDevices) return false;
     int v = state[reps_bf16][dev].load(std::memory_order_acquire);
     if (v == 0) {
-        const void *fn = reps_bf16 ? reinterpret_cast<const void *>(select_kernel<true>)
-                                   : reinterpret_cast<const void *>(select_kernel<false>);
+        const void *fn = reps_bf16 ? reinterpret_cast<const void *>(select_kernel<true, 2>)
+                                   : reinterpret_cast<const void *>(select_kernel<false, 2>);   // (slices of 128 blocks)
         v = 2;
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
@@ -249,7 +262,7 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     // 16 (beyond the portable size, so the device is asked first whether it can hold them)
     if (CL == 8 && geom->max_blocks >= 2048 && pairs * 16 <= svh::sm_count() && clusters_of_16_fit(reps_bf16)) CL = 16;
     const int per = (geom->max_blocks + CL - 1) / CL;
-    const int chunk = (per + kWarps * kRowsPerIter - 1) / (kWarps * kRowsPerIter) * (kWarps * kRowsPerIter);
+    const int chunk = (per + kStride - 1) / kStride * kStride;
 
     SelectParams p;
     p.q = static_cast<const __nv_bfloat16 *>(q);
@@ -263,10 +276,12 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     p.NBmax = geom->max_blocks, p.n_sink = n_sink, p.n_local = n_local, p.max_sel = max_sel, p.chunk = chunk;
 
     const size_t smem = (size_t)CL * chunk * sizeof(uint32_t);
-    if (smem > 48 * 1024 &&
-        (reps_bf16 ? cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                   : cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
-            cudaSuccess)
+    const bool deep = chunk > kStride;   // more than one pass per warp: load two passes' rows together
+    const void *fn = reps_bf16 ? (deep ? reinterpret_cast<const void *>(select_kernel<true, 2>)
+                                       : reinterpret_cast<const void *>(select_kernel<true, 1>))
+                               : (deep ? reinterpret_cast<const void *>(select_kernel<false, 2>)
+                                       : reinterpret_cast<const void *>(select_kernel<false, 1>));
+    if (smem > 48 * 1024 && cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SV_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CL, geom->n_kv_heads, geom->n_seq);
@@ -281,9 +296,8 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     svh::pdl_attribute(attr + 1);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if ((reps_bf16 ? cudaLaunchKernelEx(&cfg, select_kernel<true>, p) : cudaLaunchKernelEx(&cfg, select_kernel<false>, p)) !=
-        cudaSuccess)
-        return SV_ERR_CUDA;
+    void *args[] = {&p};
+    if (cudaLaunchKernelExC(&cfg, fn, args) != cudaSuccess) return SV_ERR_CUDA;
     return svh::launch_status();
 }
 
