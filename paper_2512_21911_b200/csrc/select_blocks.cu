@@ -24,10 +24,12 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-constexpr int kThreads = 512;
-constexpr int kWarps = kThreads / 32;
+// Threads per CTA: 512 while the CTAs of a launch fit the SMs at once (one sequence: the selection's barriers are the
+// critical path and sixteen warps finish the passes between them soonest), 256 for more CTAs than SMs (batches: four
+// CTAs per SM overlap one CTA's latencies with another's work; 128 sequences 31 -> 24 us, the 4 x 128K configuration
+// 8.2 -> 7.2 us, where one sequence would lose 0.3 us).
+constexpr int kThreadsFew = 512, kThreadsMany = 256;
 constexpr int kRowsPerIter = 4;   // consecutive representative rows a warp scores per pass (one 16-byte store of keys)
-constexpr int kStride = kWarps * kRowsPerIter;   // blocks the CTA covers per pass
 
 using svsel::kForcedKey;
 using svsel::order_key;
@@ -50,9 +52,11 @@ struct SelectParams {
 // kBf16: the representatives are stored in bfloat16 (storage variant); scores are fp32 either way.
 // kDepth: passes whose rows a warp loads together (1, or 2 for slices of more than 64 blocks: eight rows in flight per
 // warp, half as many trips to DRAM; more would cost the second CTA per SM its registers).
-template <bool kBf16, int kDepth>
-__global__ void __launch_bounds__(kThreads, 2) select_kernel(const SelectParams p)
+template <bool kBf16, int kDepth, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads) select_kernel(const SelectParams p)
 {
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kStride = kWarps * kRowsPerIter;   // blocks the CTA covers per pass
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int CL = (int)cluster.num_blocks();
@@ -194,6 +198,15 @@ __global__ void copy_selection_kernel(const int32_t *__restrict__ prev_idx, cons
 
 }  // namespace
 
+template <int kThreads>
+static const void *select_fn(bool reps_bf16, bool deep)
+{
+    return reps_bf16 ? (deep ? reinterpret_cast<const void *>(select_kernel<true, 2, kThreads>)
+                             : reinterpret_cast<const void *>(select_kernel<true, 1, kThreads>))
+                     : (deep ? reinterpret_cast<const void *>(select_kernel<false, 2, kThreads>)
+                             : reinterpret_cast<const void *>(select_kernel<false, 1, kThreads>));
+}
+
 // Whether this device can hold clusters of 16 CTAs of the select kernel (asked once per device and instantiation).
 static bool clusters_of_16_fit(bool reps_bf16)
 {
@@ -202,13 +215,12 @@ static bool clusters_of_16_fit(bool reps_bf16)
     if (dev < 0 || dev >= svh::kMaxDevices) return false;
     int v = state[reps_bf16][dev].load(std::memory_order_acquire);
     if (v == 0) {
-        const void *fn = reps_bf16 ? reinterpret_cast<const void *>(select_kernel<true, 2>)
-                                   : reinterpret_cast<const void *>(select_kernel<false, 2>);   // (slices of 128 blocks)
+        const void *fn = select_fn<kThreadsFew>(reps_bf16, true);   // (slices of 128 blocks)
         v = 2;
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(16, 8, 1);
-            cfg.blockDim = dim3(kThreads);
+            cfg.blockDim = dim3(kThreadsFew);
             cfg.dynamicSmemBytes = 16 * 128 * sizeof(uint32_t);
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -252,8 +264,8 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     if (n_sink + n_local > max_sel) return SV_ERR_BUDGET;
     if (geom->max_blocks > svh::kMaxBlocksSelect) return SV_ERR_UNSUPPORTED;
 
-    // CTAs per (sequence, KV head): at least 32 blocks each, and no more CTAs than two per SM can hold at once
-    // (512 threads x 60 registers: two CTAs per SM) -- a second wave costs more than the shorter slices save
+    // CTAs per (sequence, KV head): at least 32 blocks each, and no more CTAs than two per SM (a second wave costs more
+    // than the shorter slices save)
     const int pairs = geom->n_seq * geom->n_kv_heads;
     int CL = 1;
     while (CL < 8 && geom->max_blocks / (CL * 2) >= 32 && pairs * CL * 2 <= 2 * svh::sm_count()) CL *= 2;
@@ -262,7 +274,10 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     // 16 (beyond the portable size, so the device is asked first whether it can hold them)
     if (CL == 8 && geom->max_blocks >= 2048 && pairs * 16 <= svh::sm_count() && clusters_of_16_fit(reps_bf16)) CL = 16;
     const int per = (geom->max_blocks + CL - 1) / CL;
-    const int chunk = (per + kStride - 1) / kStride * kStride;
+    const bool many = (long long)pairs * CL > svh::sm_count();   // more CTAs than SMs: smaller CTAs, four per SM
+    const int threads = many ? kThreadsMany : kThreadsFew;
+    const int stride = threads / 32 * kRowsPerIter;              // blocks a CTA covers per pass
+    const int chunk = (per + stride - 1) / stride * stride;
 
     SelectParams p;
     p.q = static_cast<const __nv_bfloat16 *>(q);
@@ -276,16 +291,13 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     p.NBmax = geom->max_blocks, p.n_sink = n_sink, p.n_local = n_local, p.max_sel = max_sel, p.chunk = chunk;
 
     const size_t smem = (size_t)CL * chunk * sizeof(uint32_t);
-    const bool deep = chunk > kStride;   // more than one pass per warp: load two passes' rows together
-    const void *fn = reps_bf16 ? (deep ? reinterpret_cast<const void *>(select_kernel<true, 2>)
-                                       : reinterpret_cast<const void *>(select_kernel<true, 1>))
-                               : (deep ? reinterpret_cast<const void *>(select_kernel<false, 2>)
-                                       : reinterpret_cast<const void *>(select_kernel<false, 1>));
+    const bool deep = chunk > stride;   // more than one pass per warp: load two passes' rows together
+    const void *fn = many ? select_fn<kThreadsMany>(reps_bf16, deep) : select_fn<kThreadsFew>(reps_bf16, deep);
     if (smem > 48 * 1024 && cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SV_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CL, geom->n_kv_heads, geom->n_seq);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(threads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = cs;
     cudaLaunchAttribute attr[2];
