@@ -24,10 +24,11 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-// Threads per CTA: 512 while the CTAs of a launch fit the SMs at once (one sequence: the selection's barriers are the
-// critical path and sixteen warps finish the passes between them soonest), 256 for more CTAs than SMs (batches: four
-// CTAs per SM overlap one CTA's latencies with another's work; 128 sequences 31 -> 24 us, the 4 x 128K configuration
-// 8.2 -> 7.2 us, where one sequence would lose 0.3 us).
+// Threads per CTA: 512 while the CTAs of a launch are resident together (two per SM: the selection's barriers are
+// the critical path, sixteen warps finish the passes between them soonest, and the attention kernel behind waits for
+// the last CTA), 256 for launches of several waves (four CTAs per SM overlap one CTA's latencies with another's work:
+// 128 sequences 31 -> 24 us per call and 216 -> 208 us with the attention behind it; with one wave the smaller CTAs
+// finish a stand-alone call sooner too, but the attention behind them starts later -- 4 x 128K: 31.0 against 29.8 us).
 constexpr int kThreadsFew = 512, kThreadsMany = 256;
 constexpr int kRowsPerIter = 4;   // consecutive representative rows a warp scores per pass (one 16-byte store of keys)
 
@@ -274,7 +275,7 @@ static sv_status select_impl(const sv_geom *geom, const void *q, const void *rep
     // 16 (beyond the portable size, so the device is asked first whether it can hold them)
     if (CL == 8 && geom->max_blocks >= 2048 && pairs * 16 <= svh::sm_count() && clusters_of_16_fit(reps_bf16)) CL = 16;
     const int per = (geom->max_blocks + CL - 1) / CL;
-    const bool many = (long long)pairs * CL > svh::sm_count();   // more CTAs than SMs: smaller CTAs, four per SM
+    const bool many = (long long)pairs * CL > 2 * svh::sm_count();   // more CTAs than fit at once: smaller CTAs, four per SM
     const int threads = many ? kThreadsMany : kThreadsFew;
     const int stride = threads / 32 * kRowsPerIter;              // blocks a CTA covers per pass
     const int chunk = (per + stride - 1) / stride * stride;
