@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // 128 x 64 x 16 MMAs, each re-reading 4 KB of Q), so their Q lives in tensor memory (A operand from TMEM), and with a
     // single row tile P does too (one tile per warpgroup), which frees 32 KB for a sixth ring stage.
     constexpr bool kQTmem = NH == 4;
-    // Up to 64 query rows run as M = 64 MMAs (half the tensor time of the zero-padded M = 128 tile): matrix row m is
+    // Up to 64 query rows run as M = 64 MMAs (half the Q and P bytes of the zero-padded M = 128 tile): matrix row m is
     // TMEM lane (m / 16) * 32 + m % 16, the 16 lanes per quadrant that the NH <= 2 softmax layout uses anyway.
     constexpr int MT = NH == 4 ? 128 : 64;                   // rows of the Q and P tiles and of the MMAs
     constexpr int QR = NH == 4 ? 32 : 16;                    // tile rows per TMEM lane quadrant
